@@ -1,0 +1,144 @@
+/*
+ * kdkl - fused chunked KL distillation loss for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * The loss is the forward KL divergence between a cached top-K teacher and the student's
+ * softmax over the LM head, evaluated with the output projection fused into the loss so the
+ * [T, V] logit tensor never exists (paper, section "Full Chunked KL Computation",
+ * Algorithm 1). Per token, with z = W h the student logits, q = softmax(z / tau), p the teacher
+ * probabilities on the support S (|S| = K), M = sum_S p the retained mass (not renormalised):
+ *
+ *     L = sum_S p log p  -  sum_S p z / tau  +  M log Z          (Eq. "decomp")
+ *     dL/dz_v = (M q_v - p_v) / tau                              (Eq. "grad"; 1/tau = chain rule)
+ *
+ * and the reported loss is the mean of L over the tokens whose mask is 1 (text under Eq. "kl").
+ *
+ * Conventions for every entry point unless stated otherwise
+ *   - all data pointers are DEVICE pointers owned by the caller; the library allocates no
+ *     device memory, keeps no global state, and only enqueues work on the given stream
+ *     (no host synchronisation);
+ *   - matrices are row-major and contiguous; hidden, weight and the workspace must be
+ *     16-byte aligned; H must be a multiple of 8;
+ *   - return value: KDKL_OK or a negative KDKL_ERR_* detected on the host before anything
+ *     was enqueued (outputs untouched). Conditions only the device can see are recorded in
+ *     the workspace and read with kdkl_status().
+ */
+#ifndef KDKL_H_
+#define KDKL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KDKL_OK 0
+#define KDKL_ERR_NULL (-1)      /* a required pointer is NULL */
+#define KDKL_ERR_SHAPE (-2)     /* T, H, V, K < 1; K > KDKL_MAX_K; H % 8 != 0; V >= 2^31 */
+#define KDKL_ERR_ALIGN (-3)     /* hidden / weight / workspace / outputs not 16-byte aligned */
+#define KDKL_ERR_WORKSPACE (-4) /* workspace smaller than kdkl_workspace_bytes() */
+#define KDKL_ERR_ARG (-5)       /* temperature <= 0, chunk < 0, bad option value */
+#define KDKL_ERR_ARCH (-6)      /* current device is not compute capability 10.x */
+#define KDKL_ERR_CUDA (-7)      /* a CUDA call failed; kdkl_last_error() has the text */
+/* device-detected, reported by kdkl_status(): */
+#define KDKL_ERR_TIMEOUT (-8)   /* a bounded wait inside a kernel expired */
+#define KDKL_ERR_STATE (-9)     /* backward called on a workspace forward did not fill for this shape */
+#define KDKL_ERR_INDEX (-10)    /* a teacher index >= V was seen (the entry was ignored) */
+#define KDKL_ERR_NONFINITE (-11)/* a counted token's loss is not finite */
+
+#define KDKL_MAX_K 1024
+
+typedef struct kdkl_options {
+  int32_t struct_size;        /* sizeof(kdkl_options), for versioning */
+  int32_t teacher_mode;       /* 0: values are logits, p = exp(l/tau - Lambda), Lambda = teacher_lse[t] if given
+                                    (retained mass M < 1 possible, as in the paper) else logsumexp over the
+                                    row's K values (M = 1);
+                                 1: values are log-probabilities, p = exp(l), tau must be 1 */
+  int32_t accumulate_dweight; /* 0: dweight is overwritten; 1: dweight += */
+  int32_t dhidden_dtype;      /* 0: bf16; 1: fp32 */
+  float denom_override;       /* <= 0: mean over this call's counted tokens; > 0: divide by this instead */
+} kdkl_options;
+
+/* Bytes of device workspace forward and backward need for this shape (chunk 0 = default 4096).
+ * The same workspace must be passed to forward and then to backward: it carries the saved
+ * state of Algorithm 1 (log Z, M, the prepared teacher) and the transient per-chunk buffers. */
+size_t kdkl_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk,
+                            const kdkl_options* opt);
+
+/* Forward (Algorithm 1, "Forward"; Eq. "decomp"). One tensor-core sweep per chunk computes the
+ * online max / sum-exp over the vocabulary and gathers z at the teacher's indices.
+ *   hidden_bf16   [T, H]  bf16   student final hidden states
+ *   weight_bf16   [V, H]  bf16   LM-head weight
+ *   topk_idx      [T, K]  int32  teacher support; < 0 = empty slot; >= V = ignored + KDKL_ERR_INDEX;
+ *                                duplicates within a row add
+ *   topk_val      [T, K]  fp32   teacher values (see teacher_mode)
+ *   teacher_lse   [T] fp32 or NULL   full-vocabulary teacher logsumexp at temperature tau
+ *   loss_mask     [T] uint8 or NULL  1 = counted, 0 = ignored (teacher row is never read)
+ *   chunk         tokens per chunk, 0 = default; the result does not depend on it
+ *   loss_out      [1] fp32  mean loss
+ *   loss_per_token [T] fp32 or NULL  (0 at ignored tokens)
+ *   gathered_logits [T, K] fp32 or NULL  z at topk_idx, caller's slot order (NaN where not gathered)
+ *   gathered_idx  [T, K] int32 or NULL   the vocabulary column the kernel read for each slot (-1 where none)
+ */
+int kdkl_forward(const void* hidden_bf16, const void* weight_bf16, const int32_t* topk_idx,
+                 const float* topk_val, const float* teacher_lse, const uint8_t* loss_mask,
+                 int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, float temperature,
+                 const kdkl_options* opt, void* workspace, size_t workspace_bytes,
+                 float* loss_out, float* loss_per_token, float* gathered_logits,
+                 int32_t* gathered_idx, void* cuda_stream);
+
+/* Backward (Algorithm 1, "Backward"; Eq. "grad"). Per chunk: recompute the logit tile in tensor
+ * memory, form G = (M q - p) g / tau in registers, then dhidden = G W and dweight += G^T h.
+ * Same hidden / weight / mask / shape / chunk / temperature / opt as the forward call, and the
+ * workspace that call filled.
+ *   grad_loss  d(total)/d(loss_out), usually 1
+ *   dhidden    [T, H] bf16 (or fp32, see options); rows of ignored tokens are exact zeros
+ *   dweight    [V, H] fp32
+ */
+int kdkl_backward(const void* hidden_bf16, const void* weight_bf16, const uint8_t* loss_mask,
+                  int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, float temperature,
+                  const kdkl_options* opt, float grad_loss, void* workspace, size_t workspace_bytes,
+                  void* dhidden, float* dweight, void* cuda_stream);
+
+/* Synchronises the stream and reads the device status of the last forward/backward on this
+ * workspace: *code = KDKL_OK or a device-detected KDKL_ERR_*; detail[0] = site/row of the error,
+ * detail[1] = number of counted tokens, detail[2] = number of ignored (>= V) teacher indices.
+ * detail may be NULL. */
+int kdkl_status(const void* workspace, void* cuda_stream, int32_t* code, int64_t* detail);
+
+/* Saved per-token scalars of Algorithm 1 inside a workspace forward has filled (device pointers
+ * into the workspace; valid until the workspace is reused): log Z of z/tau and the retained mass M. */
+int kdkl_saved_state(void* workspace, int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk,
+                     const kdkl_options* opt, const float** logZ, const float** mass);
+
+/* Forward + backward with HOST buffers (the end-to-end call): copies the inputs to the device
+ * arena, runs both passes, copies loss, dhidden and dweight back, and synchronises the stream.
+ * Host pointers: hidden, weight, topk_idx, topk_val, teacher_lse (or NULL), loss_mask (or NULL),
+ * loss_out [1], dhidden_out [T,H] (dtype per options), dweight_out [V,H] fp32 (either may be NULL
+ * to skip that copy). device_arena is a device buffer of at least kdkl_host_arena_bytes(). */
+size_t kdkl_host_arena_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk,
+                             const kdkl_options* opt);
+int kdkl_forward_backward_host(const void* hidden_bf16, const void* weight_bf16, const int32_t* topk_idx,
+                               const float* topk_val, const float* teacher_lse, const uint8_t* loss_mask,
+                               int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, float temperature,
+                               const kdkl_options* opt, float grad_loss, void* device_arena,
+                               size_t arena_bytes, float* loss_out, void* dhidden_out, float* dweight_out,
+                               void* cuda_stream);
+
+/* The tensor-core mainloop on its own: C[M,N] (fp32, row-major) = A * B^T with bf16 operands.
+ * a_mn = 0: A is [M, K] row-major; 1: A is stored [K, M]. b_mn likewise for B ([N, K] or [K, N]).
+ * M, N, K multiples of 8. status: device int32[2] the caller zeroed, receives {KDKL_ERR_TIMEOUT, site}
+ * if a bounded wait expires, or NULL. Used to validate and time the GEMM under the fused epilogues. */
+int kdkl_gemm_bf16(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K,
+                   int32_t a_mn, int32_t b_mn, int32_t* status, void* cuda_stream);
+
+/* Text of the last KDKL_ERR_CUDA on this thread. */
+const char* kdkl_last_error(void);
+
+/* Number of kernels the last forward / backward / host call on this thread enqueued. */
+int64_t kdkl_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KDKL_H_ */

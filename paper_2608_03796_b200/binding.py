@@ -1,0 +1,209 @@
+"""ctypes binding over the kdkl C ABI (include/kdkl.h): argument marshalling only.
+
+Every step of the loss runs in the library's CUDA kernels. torch is used here for device
+memory and the current stream, nothing else. If the shared library has not been built the
+first call raises: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libkdkl.so")
+
+KDKL_OK = 0
+ERRORS = {
+    -1: "KDKL_ERR_NULL", -2: "KDKL_ERR_SHAPE", -3: "KDKL_ERR_ALIGN", -4: "KDKL_ERR_WORKSPACE",
+    -5: "KDKL_ERR_ARG", -6: "KDKL_ERR_ARCH", -7: "KDKL_ERR_CUDA", -8: "KDKL_ERR_TIMEOUT",
+    -9: "KDKL_ERR_STATE", -10: "KDKL_ERR_INDEX", -11: "KDKL_ERR_NONFINITE",
+}
+
+EXPORTS = [
+    "kdkl_workspace_bytes", "kdkl_forward", "kdkl_backward", "kdkl_status", "kdkl_saved_state",
+    "kdkl_host_arena_bytes", "kdkl_forward_backward_host", "kdkl_gemm_bf16", "kdkl_last_error",
+    "kdkl_last_launch_count",
+]
+
+
+class KdklError(RuntimeError):
+    def __init__(self, code: int, text: str = ""):
+        self.code = code
+        super().__init__(f"{ERRORS.get(code, code)} {text}".strip())
+
+
+class kdkl_options(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_int32), ("teacher_mode", ctypes.c_int32),
+                ("accumulate_dweight", ctypes.c_int32), ("dhidden_dtype", ctypes.c_int32),
+                ("denom_override", ctypes.c_float)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the shared library (once). Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it first (python -c 'import __graft_entry__ as g; g.build()')")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i64, i32, f32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_float, ctypes.c_size_t
+    L.kdkl_workspace_bytes.restype = sz
+    L.kdkl_workspace_bytes.argtypes = [i64, i64, i64, i32, i64, vp]
+    L.kdkl_forward.restype = ctypes.c_int
+    L.kdkl_forward.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, vp, sz, vp, vp, vp, vp, vp]
+    L.kdkl_backward.restype = ctypes.c_int
+    L.kdkl_backward.argtypes = [vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, f32, vp, sz, vp, vp, vp]
+    L.kdkl_status.restype = ctypes.c_int
+    L.kdkl_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)]
+    L.kdkl_saved_state.restype = ctypes.c_int
+    L.kdkl_saved_state.argtypes = [vp, i64, i64, i64, i32, i64, vp, ctypes.POINTER(vp), ctypes.POINTER(vp)]
+    L.kdkl_host_arena_bytes.restype = sz
+    L.kdkl_host_arena_bytes.argtypes = [i64, i64, i64, i32, i64, vp]
+    L.kdkl_forward_backward_host.restype = ctypes.c_int
+    L.kdkl_forward_backward_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, f32, vp, sz,
+                                             vp, vp, vp, vp]
+    L.kdkl_gemm_bf16.restype = ctypes.c_int
+    L.kdkl_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, vp, vp]
+    L.kdkl_last_error.restype = ctypes.c_char_p
+    L.kdkl_last_error.argtypes = []
+    L.kdkl_last_launch_count.restype = ctypes.c_int64
+    L.kdkl_last_launch_count.argtypes = []
+    _lib = L
+    return L
+
+
+def _check(rc: int):
+    if rc != KDKL_OK:
+        raise KdklError(rc, lib().kdkl_last_error().decode() if rc == -7 else "")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def make_options(teacher_mode=0, accumulate_dweight=0, dhidden_dtype=0, denom_override=0.0) -> kdkl_options:
+    return kdkl_options(ctypes.sizeof(kdkl_options), teacher_mode, accumulate_dweight, dhidden_dtype, denom_override)
+
+
+def _opt_ptr(opt: Optional[kdkl_options]):
+    return None if opt is None else ctypes.cast(ctypes.pointer(opt), ctypes.c_void_p)
+
+
+def kdkl_workspace_bytes(T, H, V, K, chunk=0, opt=None) -> int:
+    return lib().kdkl_workspace_bytes(T, H, V, K, chunk, _opt_ptr(opt))
+
+
+def kdkl_forward(hidden, weight, topk_idx, topk_val, workspace, loss_out, *, teacher_lse=None, loss_mask=None,
+                 chunk=0, temperature=1.0, opt=None, loss_per_token=None, gathered_logits=None,
+                 gathered_idx=None) -> None:
+    T, H = hidden.shape
+    V = weight.shape[0]
+    K = topk_idx.shape[1]
+    _check(lib().kdkl_forward(_ptr(hidden), _ptr(weight), _ptr(topk_idx), _ptr(topk_val), _ptr(teacher_lse),
+                              _ptr(loss_mask), T, H, V, K, chunk, temperature, _opt_ptr(opt), _ptr(workspace),
+                              workspace.numel() * workspace.element_size(), _ptr(loss_out), _ptr(loss_per_token),
+                              _ptr(gathered_logits), _ptr(gathered_idx), _stream()))
+
+
+def kdkl_backward(hidden, weight, K, workspace, dhidden, dweight, *, loss_mask=None, chunk=0, temperature=1.0,
+                  opt=None, grad_loss=1.0) -> None:
+    T, H = hidden.shape
+    V = weight.shape[0]
+    _check(lib().kdkl_backward(_ptr(hidden), _ptr(weight), _ptr(loss_mask), T, H, V, K, chunk, temperature,
+                               _opt_ptr(opt), grad_loss, _ptr(workspace),
+                               workspace.numel() * workspace.element_size(), _ptr(dhidden), _ptr(dweight), _stream()))
+
+
+def kdkl_status(workspace):
+    """(code, [site_or_row, counted_tokens, ignored_indices]); synchronises the current stream."""
+    code = ctypes.c_int32(0)
+    detail = (ctypes.c_int64 * 3)()
+    _check(lib().kdkl_status(_ptr(workspace), _stream(), ctypes.byref(code), detail))
+    return code.value, list(detail)
+
+
+def kdkl_saved_state(workspace, T, H, V, K, chunk=0, opt=None):
+    """Views of the saved log Z [T] and retained mass M [T] inside the workspace."""
+    a, b = ctypes.c_void_p(), ctypes.c_void_p()
+    _check(lib().kdkl_saved_state(_ptr(workspace), T, H, V, K, chunk, _opt_ptr(opt), ctypes.byref(a), ctypes.byref(b)))
+    base = workspace.data_ptr()
+    ws_f = workspace.view(torch.uint8)
+    def view(p):
+        off = p.value - base
+        return ws_f[off:off + 4 * T].view(torch.float32)
+    return view(a), view(b)
+
+
+def kdkl_host_arena_bytes(T, H, V, K, chunk=0, opt=None) -> int:
+    return lib().kdkl_host_arena_bytes(T, H, V, K, chunk, _opt_ptr(opt))
+
+
+def kdkl_forward_backward_host(hidden, weight, topk_idx, topk_val, arena, loss_out, dhidden_out, dweight_out, *,
+                               teacher_lse=None, loss_mask=None, chunk=0, temperature=1.0, opt=None,
+                               grad_loss=1.0) -> None:
+    """All tensors except ``arena`` are HOST tensors (pinned for full copy speed)."""
+    T, H = hidden.shape
+    V = weight.shape[0]
+    K = topk_idx.shape[1]
+    _check(lib().kdkl_forward_backward_host(_ptr(hidden), _ptr(weight), _ptr(topk_idx), _ptr(topk_val),
+                                            _ptr(teacher_lse), _ptr(loss_mask), T, H, V, K, chunk, temperature,
+                                            _opt_ptr(opt), grad_loss, _ptr(arena),
+                                            arena.numel() * arena.element_size(), _ptr(loss_out), _ptr(dhidden_out),
+                                            _ptr(dweight_out), _stream()))
+
+
+def kdkl_gemm_bf16(A, B, C, M, N, K, a_mn=0, b_mn=0, status=None) -> None:
+    _check(lib().kdkl_gemm_bf16(_ptr(A), _ptr(B), _ptr(C), M, N, K, a_mn, b_mn, _ptr(status), _stream()))
+
+
+def kdkl_last_launch_count() -> int:
+    return lib().kdkl_last_launch_count()
+
+
+class FusedChunkedKL:
+    """Convenience holder: allocates workspace and outputs with torch once, then runs the two calls."""
+
+    def __init__(self, T, H, V, K, chunk=0, temperature=1.0, opt=None, device="cuda", want_gathered=False,
+                 want_per_token=False):
+        self.T, self.H, self.V, self.K = T, H, V, K
+        self.chunk, self.temperature, self.opt = chunk, temperature, opt
+        nbytes = kdkl_workspace_bytes(T, H, V, K, chunk, opt)
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        self.loss = torch.zeros(1, dtype=torch.float32, device=device)
+        dh_dtype = torch.float32 if (opt is not None and opt.dhidden_dtype == 1) else torch.bfloat16
+        self.dhidden = torch.empty(T, H, dtype=dh_dtype, device=device)
+        self.dweight = torch.empty(V, H, dtype=torch.float32, device=device)
+        self.loss_per_token = torch.empty(T, dtype=torch.float32, device=device) if want_per_token else None
+        self.gathered_logits = torch.empty(T, K, dtype=torch.float32, device=device) if want_gathered else None
+        self.gathered_idx = torch.empty(T, K, dtype=torch.int32, device=device) if want_gathered else None
+        self.launches = 0
+
+    def forward(self, hidden, weight, topk_idx, topk_val, teacher_lse=None, loss_mask=None):
+        kdkl_forward(hidden, weight, topk_idx, topk_val, self.workspace, self.loss, teacher_lse=teacher_lse,
+                     loss_mask=loss_mask, chunk=self.chunk, temperature=self.temperature, opt=self.opt,
+                     loss_per_token=self.loss_per_token, gathered_logits=self.gathered_logits,
+                     gathered_idx=self.gathered_idx)
+        self.launches = kdkl_last_launch_count()
+        return self.loss
+
+    def backward(self, hidden, weight, loss_mask=None, grad_loss=1.0):
+        kdkl_backward(hidden, weight, self.K, self.workspace, self.dhidden, self.dweight, loss_mask=loss_mask,
+                      chunk=self.chunk, temperature=self.temperature, opt=self.opt, grad_loss=grad_loss)
+        self.launches += kdkl_last_launch_count()
+        return self.dhidden, self.dweight
+
+    def status(self):
+        return kdkl_status(self.workspace)
+
+    def saved_state(self):
+        return kdkl_saved_state(self.workspace, self.T, self.H, self.V, self.K, self.chunk, self.opt)

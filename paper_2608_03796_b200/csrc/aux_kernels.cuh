@@ -1,0 +1,283 @@
+// The small kernels around the GEMMs: teacher preparation, partial log-sum-exp combine,
+// loss reduction and backward coefficients. All are bandwidth-trivial
+// next to the tensor-core phases; they use warp-shuffle reductions and fixed-order sums
+// (no floating-point atomics), so results are reproducible run to run.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace kdkl {
+
+constexpr int KDKL_MAGIC = 0x4b444b4c;  // "KDKL"
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kLog2e = 1.4426950408889634f;
+
+// Head of the workspace (256 bytes). Written by forward, read by backward.
+struct WsHeader {
+  int status;        // 0 or the first device-detected error code
+  int where;         // detail for the error (wait site, row, ...)
+  int magic;         // KDKL_MAGIC once forward has completed its last kernel
+  int go;            // backward gate: 1 when the state matches the call, else 0
+  long long T, H, V;
+  int K;
+  int n_bad_idx;     // teacher indices >= V seen by prep (ignored entries)
+  long long n_tokens;  // number of counted tokens (mask = 1)
+  float denom;       // divisor of the mean actually used
+  float tau;
+  double loss_sum;   // sum of counted per-token losses
+};
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__global__ void header_reset_kernel(WsHeader* hdr) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    hdr->status = 0; hdr->where = 0; hdr->magic = 0; hdr->go = 0;
+    hdr->n_bad_idx = 0; hdr->n_tokens = 0; hdr->denom = 0.f; hdr->loss_sum = 0.0;
+  }
+}
+
+// ------------------------------------------------------------------------------------ prep
+// One warp per token. From the cached teacher values l[t,k] and tau:
+//   p_k = exp(l_k/tau - Lambda_t), Lambda_t = teacher_lse[t] | logsumexp_k(l_k/tau) | 0 (log-prob mode)
+//   M_t = sum_k p_k (retained mass, never renormalised), Hent_t = sum_v p_v log p_v
+// and an index-sorted copy of the row (idx ascending, p merged over duplicate indices, the
+// original slot of every entry) that the GEMM epilogues walk with a cursor.
+// Ignored tokens (mask = 0) get an empty row: their teacher entries are never read.
+constexpr int PREP_WARPS = 4;
+__global__ void __launch_bounds__(PREP_WARPS * 32)
+prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val,
+            const float* __restrict__ teacher_lse, const uint8_t* __restrict__ mask, long long T, int V, int K,
+            int Kpad, float inv_tau, int teacher_mode, int* __restrict__ idx_sorted, float* __restrict__ p_sorted,
+            uint16_t* __restrict__ perm, int* __restrict__ nvalid, float* __restrict__ Mout,
+            float* __restrict__ Hent, WsHeader* hdr) {
+  extern __shared__ uint8_t prep_smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int* keys = reinterpret_cast<int*>(prep_smem) + warp * Kpad;
+  float* pv = reinterpret_cast<float*>(prep_smem + sizeof(int) * PREP_WARPS * Kpad) + warp * Kpad;
+  uint16_t* slot = reinterpret_cast<uint16_t*>(prep_smem + 2 * sizeof(int) * PREP_WARPS * Kpad) + warp * Kpad;
+
+  const long long t = (long long)blockIdx.x * PREP_WARPS + warp;
+  if (t >= T) return;
+  const bool counted = mask == nullptr || mask[t] != 0;
+  int* out_idx = idx_sorted + t * K;
+  float* out_p = p_sorted + t * K;
+  uint16_t* out_perm = perm + t * K;
+  if (!counted) {
+    for (int k = lane; k < K; k += 32) { out_idx[k] = 0x7fffffff; out_p[k] = 0.f; out_perm[k] = (uint16_t)k; }
+    if (lane == 0) { nvalid[t] = 0; Mout[t] = 0.f; Hent[t] = 0.f; }
+    return;
+  }
+  // load, validate, scaled values
+  float mx = -INFINITY;
+  int bad = 0;
+  for (int k = lane; k < Kpad; k += 32) {
+    int key = 0x7fffffff;
+    float u = -INFINITY;
+    if (k < K) {
+      const int id = topk_idx[t * K + k];
+      if (id >= 0 && id < V) { key = id; u = topk_val[t * K + k] * inv_tau; }
+      else if (id >= V) bad++;
+    }
+    keys[k] = key; pv[k] = u; slot[k] = (uint16_t)k;
+    mx = fmaxf(mx, u);
+  }
+  bad = (int)warp_sum((float)bad);
+  if (bad && lane == 0) { atomicAdd(&hdr->n_bad_idx, bad); atomicCAS(&hdr->status, 0, -10); }
+  float lam;
+  if (teacher_mode == 1) lam = 0.f;
+  else if (teacher_lse != nullptr) lam = teacher_lse[t];
+  else {
+    mx = warp_max(mx);
+    if (!(mx > -INFINITY)) mx = 0.f;
+    __syncwarp();
+    float s = 0.f;
+    for (int k = lane; k < Kpad; k += 32) s += expf(pv[k] - mx);
+    s = warp_sum(s);
+    lam = mx + logf(s);
+  }
+  __syncwarp();
+  for (int k = lane; k < Kpad; k += 32) pv[k] = keys[k] != 0x7fffffff ? expf(pv[k] - lam) : 0.f;
+  __syncwarp();
+  // bitonic sort by key, (p, slot) carried along
+  for (int size = 2; size <= Kpad; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int i = lane; i < (Kpad >> 1); i += 32) {
+        const int lo = 2 * i - (i & (stride - 1));
+        const int hi = lo + stride;
+        const bool up = (lo & size) == 0;
+        const int a = keys[lo], b = keys[hi];
+        if ((a > b) == up) {
+          keys[lo] = b; keys[hi] = a;
+          const float pa = pv[lo]; pv[lo] = pv[hi]; pv[hi] = pa;
+          const uint16_t sa = slot[lo]; slot[lo] = slot[hi]; slot[hi] = sa;
+        }
+      }
+      __syncwarp();
+    }
+  }
+  // merge duplicate indices into the head of each run (scatter-add semantics)
+  float msum = 0.f, hsum = 0.f;
+  int nv = 0;
+  for (int j = lane; j < Kpad; j += 32) {
+    const int key = keys[j];
+    float pj = 0.f;
+    if (key != 0x7fffffff) {
+      nv++;
+      if (j == 0 || keys[j - 1] != key) {
+        pj = pv[j];
+        for (int q = j + 1; q < Kpad && keys[q] == key; ++q) pj += pv[q];
+        msum += pj;
+        if (pj > 0.f) hsum += pj * logf(pj);
+      }
+    }
+    if (j < K) { out_idx[j] = key; out_p[j] = pj; out_perm[j] = slot[j]; }
+  }
+  msum = warp_sum(msum); hsum = warp_sum(hsum);
+  nv = (int)warp_sum((float)nv);
+  if (lane == 0) { nvalid[t] = nv; Mout[t] = msum; Hent[t] = hsum; }
+}
+
+// ------------------------------------------------------------------------------------ combine
+// Per chunk. Merges the per-vocab-tile (max, sum) partials of every row into the log-normaliser,
+// adds the sparse terms and writes the per-token loss  L_t = Hent_t - C_t + M_t log Z_t
+// (Eq. "decomp"), with C_t = sum_k p_k z_k / tau from the gathered logits. Also un-permutes the
+// gathered logits / columns into the caller's slot order.
+// Block = 32 rows x 8 partial lanes; partial arrays are [n_tiles, part_stride] so reads coalesce.
+__global__ void __launch_bounds__(256)
+combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_s, long long part_stride,
+               int n_tiles, int rows, long long row0, int K, float inv_tau, const int* __restrict__ nvalid,
+               const float* __restrict__ p_sorted, const uint16_t* __restrict__ perm, const float* __restrict__ zg,
+               const int* __restrict__ colread, const float* __restrict__ Mv, const float* __restrict__ Hent,
+               const uint8_t* __restrict__ mask, float* __restrict__ lz2, float* __restrict__ logZ_nat,
+               float* __restrict__ loss_tok, float* __restrict__ loss_tok_user, float* __restrict__ g_logits,
+               int* __restrict__ g_idx, WsHeader* hdr) {
+  __shared__ float sm_m[8][32], sm_s[8][32];
+  __shared__ float sm_lz[32];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int r = blockIdx.x * 32 + tx;       // row within the chunk
+  float m = -INFINITY, s = 0.f;
+  if (r < rows) {
+    for (int nt = ty; nt < n_tiles; nt += 8) {
+      const float pm = part_m[(long long)nt * part_stride + r];
+      const float ps = part_s[(long long)nt * part_stride + r];
+      const float mn = fmaxf(m, pm);
+      s = s * exp2f(m - mn) + ps * exp2f(pm - mn);
+      m = mn;
+    }
+  }
+  sm_m[ty][tx] = m; sm_s[ty][tx] = s;
+  __syncthreads();
+  if (ty == 0 && r < rows) {
+    float mm = sm_m[0][tx], ss = sm_s[0][tx];
+    for (int i = 1; i < 8; ++i) {           // fixed order
+      const float pm = sm_m[i][tx], ps = sm_s[i][tx];
+      if (pm == -INFINITY) continue;
+      const float mn = fmaxf(mm, pm);
+      ss = ss * exp2f(mm - mn) + ps * exp2f(pm - mn);
+      mm = mn;
+    }
+    const float l2 = mm + log2f(ss);
+    sm_lz[tx] = l2;
+    lz2[row0 + r] = l2;
+    logZ_nat[row0 + r] = l2 * kLn2;
+  }
+  __syncthreads();
+  // sparse terms: warp ty handles rows ty*4 .. ty*4+3 of this block
+  for (int i = 0; i < 4; ++i) {
+    const int rr = blockIdx.x * 32 + ty * 4 + i;
+    if (rr >= rows) break;
+    const long long t = row0 + rr;
+    const int nv = nvalid[t];
+    float c = 0.f;
+    for (int j = tx; j < K; j += 32) {
+      const int sl = perm[t * K + j];
+      if (j < nv) {
+        const float z = zg[t * K + j];
+        c += p_sorted[t * K + j] * z;
+        if (g_logits) g_logits[t * K + sl] = z;
+        if (g_idx) g_idx[t * K + sl] = colread[t * K + j];
+      } else {
+        if (g_logits) g_logits[t * K + sl] = __int_as_float(0x7fc00000);
+        if (g_idx) g_idx[t * K + sl] = -1;
+      }
+    }
+    c = warp_sum(c) * inv_tau;
+    if (tx == 0) {
+      const bool counted = mask == nullptr || mask[t] != 0;
+      const float lz = sm_lz[ty * 4 + i] * kLn2;
+      float L = 0.f;
+      if (counted) {
+        L = Hent[t] - c + Mv[t] * lz;
+        if (!isfinite(L)) { atomicCAS(&hdr->status, 0, -11); atomicCAS(&hdr->where, 0, (int)t); }
+      }
+      loss_tok[t] = L;
+      if (loss_tok_user) loss_tok_user[t] = L;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------ loss reduce
+// One block: loss = sum_t mask_t L_t / denom, summed in double in a fixed order. Marks the
+// workspace as complete for backward.
+__global__ void __launch_bounds__(1024)
+loss_reduce_kernel(const float* __restrict__ loss_tok, const uint8_t* __restrict__ mask, long long T,
+                   float denom_override, float tau, long long H, long long V, int K, float* loss_out,
+                   WsHeader* hdr) {
+  __shared__ double sm_sum[1024];
+  __shared__ long long sm_cnt[1024];
+  double acc = 0.0;
+  long long cnt = 0;
+  for (long long t = threadIdx.x; t < T; t += 1024) {
+    const bool counted = mask == nullptr || mask[t] != 0;
+    if (counted) { acc += (double)loss_tok[t]; cnt++; }
+  }
+  sm_sum[threadIdx.x] = acc; sm_cnt[threadIdx.x] = cnt;
+  __syncthreads();
+  for (int o = 512; o > 0; o >>= 1) {
+    if (threadIdx.x < o) { sm_sum[threadIdx.x] += sm_sum[threadIdx.x + o]; sm_cnt[threadIdx.x] += sm_cnt[threadIdx.x + o]; }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const long long n = sm_cnt[0];
+    const float denom = denom_override > 0.f ? denom_override : (float)n;
+    hdr->n_tokens = n; hdr->denom = denom; hdr->loss_sum = sm_sum[0]; hdr->tau = tau;
+    hdr->T = T; hdr->H = H; hdr->V = V; hdr->K = K;
+    *loss_out = denom > 0.f ? (float)(sm_sum[0] / (double)denom) : 0.f;
+    __threadfence();
+    hdr->magic = KDKL_MAGIC;
+  }
+}
+
+// ------------------------------------------------------------------------------------ backward prep
+// coefA_t = g_t M_t / tau, coefB_t = g_t / tau with g_t = grad_loss * mask_t / denom
+// (Algorithm 1 backward: G = (M g) q, G -= p g; the 1/tau is the chain rule through z/tau).
+// Also checks that the workspace was filled by a forward call of the same shape.
+__global__ void bwd_coef_kernel(const float* __restrict__ Mv, const uint8_t* __restrict__ mask, long long T,
+                                long long H, long long V, int K, float grad_loss, float inv_tau,
+                                float* __restrict__ coefA, float* __restrict__ coefB, WsHeader* hdr) {
+  const bool state_ok = hdr->magic == KDKL_MAGIC && hdr->T == T && hdr->H == H && hdr->V == V && hdr->K == K;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    hdr->go = state_ok ? 1 : 0;
+    if (!state_ok) atomicCAS(&hdr->status, 0, -9);
+  }
+  if (!state_ok) return;
+  const float denom = hdr->denom;
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= T) return;
+  const bool counted = mask == nullptr || mask[t] != 0;
+  const float g = (counted && denom > 0.f) ? grad_loss / denom : 0.f;
+  coefA[t] = g * Mv[t] * inv_tau;
+  coefB[t] = g * inv_tau;
+}
+
+}  // namespace kdkl

@@ -1,0 +1,386 @@
+// Persistent, warp-specialised bf16 GEMM for sm_100a: D[M,N] = A[M,K] * B[N,K]^T with fp32
+// accumulation in tensor memory, operands staged by TMA into 128-byte-swizzled shared memory.
+//
+//   warp 0      TMA producer (one lane): fills a ring of STAGES shared-memory stages
+//   warp 1      allocates TMEM; one lane issues tcgen05.mma and commits to mbarriers
+//   warps 2..5  epilogue: tcgen05.ld gives each thread one accumulator row (32 columns at
+//               a time); two TMEM accumulator stages let tile i's epilogue overlap tile
+//               i+1's MMAs
+//
+// One CTA per SM (grid = min(tiles, SM count)), tiles of 128 x 256, k-blocks of 64.
+// Either operand may be K-major (its rows are contiguous along K) or MN-major (stored
+// [K, M] / [K, N], contiguous along M / N); the difference is confined to the TMA boxes
+// and the shared-memory descriptors.
+//
+// Epilogues (the fused parts of the loss):
+//   EPI_STORE_F32   plain fp32 store or += (dWeight accumulation, Algorithm 1 "dW += G^T h")
+//   EPI_STORE_BF16  bf16 store (dHidden, Algorithm 1 "dh = G W")
+//   EPI_LSE         forward: per (row, vocab tile) online max / sum-exp of z/tau and gather of
+//                   z at the teacher's indices; logits never leave the SM (Algorithm 1,
+//                   forward passes 1 and 2 in one sweep; Eq. "decomp")
+//   EPI_DLOGITS     backward: G = a_t * exp(z/tau - logZ) - b_t * p at the support, cast to
+//                   bf16 (Eq. "grad", Algorithm 1 backward)
+#pragma once
+#include <cuda_bf16.h>
+
+#include "sm100_prims.cuh"
+
+namespace kdkl {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int UMMA_K = 16;
+constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KiB
+constexpr int B_STAGE_BYTES = BN * BK * 2;   // 32 KiB
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int GEMM_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr int GEMM_SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+enum { EPI_STORE_F32 = 0, EPI_STORE_BF16 = 1, EPI_LSE = 2, EPI_DLOGITS = 3 };
+
+struct GemmParams {
+  int M, N, K;               // valid extents of this launch
+  int m_tiles, n_tiles;
+  int m_inner;               // 1: consecutive tile ids walk M first (B panel shared), 0: N first
+  int* status;               // device status word pair {code, where}
+  const int* go;             // optional: kernel returns at once when *go == 0
+  // EPI_STORE_*
+  void* C;                   // fp32 or bf16 [M, ldc]
+  long long ldc;
+  int accumulate;            // fp32 only: 1 -> C += D
+  // EPI_LSE / EPI_DLOGITS: all row-indexed pointers are already offset to this chunk's row 0
+  float scale_log2;          // log2(e) / tau
+  int Ktop;                  // teacher slots per row
+  const int* idx_sorted;     // [rows, Ktop] ascending, first nvalid[row] entries valid
+  const int* nvalid;         // [rows]
+  float* part_m;             // [n_tiles, part_stride] running max (log2 domain)
+  float* part_s;             // [n_tiles, part_stride] sum of 2^(s - max)
+  long long part_stride;
+  float* zg;                 // [rows, Ktop] gathered logits, sorted order
+  int* colread;              // [rows, Ktop] column actually read, sorted order
+  const float* lz2;          // [rows] log2-domain log-normaliser
+  const float* coefA;        // [rows] g_t * M_t / tau
+  const float* coefB;        // [rows] g_t / tau
+  const float* p_sorted;     // [rows, Ktop]
+  __nv_bfloat16* G;          // [rows, ldg]
+  long long ldg;
+};
+
+__device__ __forceinline__ int lower_bound_i32(const int* a, int n, int key) {
+  int lo = 0, hi = n;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (a[mid] < key) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ float sel32(const uint32_t (&r)[32], int off) {
+  float v = 0.f;
+#pragma unroll
+  for (int j = 0; j < 32; ++j) v = (off == j) ? __uint_as_float(r[j]) : v;
+  return v;
+}
+
+// 2^x by the special-function unit (relative error about 2^-22; 2^-inf = 0)
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int EPI, bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+  // barriers and bookkeeping live after the stage ring
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * STAGE_BYTES);
+  const uint32_t bar0 = smem_base + STAGES * STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (p.go != nullptr && *p.go == 0) return;   // uniform across the grid
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    *abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int num_tiles = p.m_tiles * p.n_tiles;
+  const int kblocks = (p.K + BK - 1) / BK;
+
+  auto tile_coords = [&](int tile, int& mt, int& nt) {
+    if (p.m_inner) { mt = tile % p.m_tiles; nt = tile / p.m_tiles; }
+    else           { nt = tile % p.n_tiles; mt = tile / p.n_tiles; }
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0, issued = 0, last_par = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        int mt, nt;
+        tile_coords(tile, mt, nt);
+        const int m0 = mt * BM, n0 = nt * BN;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
+          const uint32_t sa = smem_base + s * STAGE_BYTES;
+          const uint32_t sb = sa + A_STAGE_BYTES;
+          mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES);
+          const int k0 = kb * BK;
+          if (!A_MN) {
+            tma_load_2d(sa, &tmA, k0, m0, full_bar(s));
+          } else {
+#pragma unroll
+            for (int i = 0; i < BM / 64; ++i) tma_load_2d(sa + i * (BK * 128), &tmA, m0 + 64 * i, k0, full_bar(s));
+          }
+          if (!B_MN) {
+            tma_load_2d(sb, &tmB, k0, n0, full_bar(s));
+          } else {
+#pragma unroll
+            for (int i = 0; i < BN / 64; ++i) tma_load_2d(sb + i * (BK * 128), &tmB, n0 + 64 * i, k0, full_bar(s));
+          }
+          issued |= 1u << s;
+          last_par = (last_par & ~(1u << s)) | (ph << s);
+        }
+      }
+      if (!ok) {
+        // aborted: give the copies still in flight a bounded time to land before the CTA exits
+        for (int s = 0; s < STAGES; ++s) {
+          if (!((issued >> s) & 1u)) continue;
+          const uint64_t t0 = globaltimer_ns();
+          while (!mbar_try_wait(full_bar(s), (last_par >> s) & 1u) && globaltimer_ns() - t0 < 2000000ull) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc_bf16(BM, BN, A_MN ? 1u : 0u, B_MN ? 1u : 0u);
+      uint32_t it = 0, lt = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+        const uint32_t acc = lt & 1u;
+        const uint32_t aph = (lt >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + acc * BN;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, 3)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + s * STAGE_BYTES;
+          const uint32_t sb = sa + A_STAGE_BYTES;
+#pragma unroll
+          for (int j = 0; j < BK / UMMA_K; ++j) {
+            const uint64_t ad = A_MN ? make_smem_desc(sa + j * (UMMA_K * 128), BK * 128, 1024)
+                                     : make_smem_desc(sa + j * (UMMA_K * 2), 0, 1024);
+            const uint64_t bd = B_MN ? make_smem_desc(sb + j * (UMMA_K * 128), BK * 128, 1024)
+                                     : make_smem_desc(sb + j * (UMMA_K * 2), 0, 1024);
+            umma_bf16(tmem_d, ad, bd, idesc, (kb > 0 || j > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(s));           // frees the stage when these MMAs have read it
+        }
+        if (ok) umma_commit(tfull_bar(acc));   // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int lg = warp & 3;                   // TMEM lane group this warp may read
+    const int row_in_tile = lg * 32 + lane;
+    uint32_t lt = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+      int mt, nt;
+      tile_coords(tile, mt, nt);
+      const int m0 = mt * BM, n0 = nt * BN;
+      const int row = m0 + row_in_tile;
+      const bool row_ok = row < p.M;
+      const uint32_t acc = lt & 1u;
+      const uint32_t aph = (lt >> 1) & 1u;
+
+      // per-row state that does not need the accumulator: fetched before the wait
+      int cur = 0, nv = 0, next_idx = 0x7fffffff;
+      const int* idxrow = nullptr;
+      float row_a = 0.f, row_b = 0.f, row_lz2 = 0.f;
+      if (EPI == EPI_LSE || EPI == EPI_DLOGITS) {
+        if (row_ok) {
+          idxrow = p.idx_sorted + (long long)row * p.Ktop;
+          nv = p.nvalid[row];
+          cur = lower_bound_i32(idxrow, nv, n0);
+          next_idx = cur < nv ? idxrow[cur] : 0x7fffffff;
+          if (EPI == EPI_DLOGITS) { row_a = p.coefA[row]; row_b = p.coefB[row]; row_lz2 = p.lz2[row]; }
+        }
+      }
+
+      // the decision to go on is taken by the whole warp: tcgen05.ld below is warp-collective
+      const bool arrived = mbar_wait(tfull_bar(acc), aph, abort_flag, p.status, 4);
+      if (!__all_sync(0xffffffffu, arrived)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + (uint32_t(lg * 32) << 16) + acc * BN;
+
+      float m_run = -INFINITY, s_run = 0.f;
+#pragma unroll 1
+      for (int w = 0; w < BN / 32; ++w) {
+        const int col0 = n0 + w * 32;
+        if (col0 >= p.N) break;                // uniform: whole window past the edge
+        uint32_t r[32];
+        __syncwarp();
+        tmem_ld32(taddr + w * 32, r);
+        tmem_ld_wait();
+        const bool full_w = col0 + 32 <= p.N;
+
+        if (EPI == EPI_STORE_F32) {
+          if (row_ok) {
+            float* dst = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col0;
+            if (full_w && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                       __uint_as_float(r[j + 3]));
+                if (p.accumulate) {
+                  const float4 o = *reinterpret_cast<const float4*>(dst + j);
+                  v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                }
+                *reinterpret_cast<float4*>(dst + j) = v;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.N) dst[j] = __uint_as_float(r[j]) + (p.accumulate ? dst[j] : 0.f);
+            }
+          }
+        } else if (EPI == EPI_STORE_BF16) {
+          if (row_ok) {
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col0;
+            if (full_w && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                uint4 v;
+                v.x = pack_bf16x2(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+                v.y = pack_bf16x2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                v.z = pack_bf16x2(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
+                v.w = pack_bf16x2(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
+                *reinterpret_cast<uint4*>(dst + j) = v;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(r[j]));
+            }
+          }
+        } else if (EPI == EPI_LSE) {
+          if (row_ok) {
+            // gather the student logit at every teacher index that falls in this window
+            while (next_idx < col0 + 32) {
+              const float zsel = sel32(r, next_idx - col0);
+              p.zg[(long long)row * p.Ktop + cur] = zsel;
+              p.colread[(long long)row * p.Ktop + cur] = next_idx;
+              ++cur;
+              next_idx = cur < nv ? idxrow[cur] : 0x7fffffff;
+            }
+            // online max / sum-exp in the log2 domain
+            float t[32];
+            float wmax = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              t[j] = (full_w || col0 + j < p.N) ? __uint_as_float(r[j]) * p.scale_log2 : -INFINITY;
+              wmax = fmaxf(wmax, t[j]);
+            }
+            const float m_new = fmaxf(m_run, wmax);
+            float acc_s = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) acc_s += ex2_approx(t[j] - m_new);
+            s_run = s_run * ex2_approx(m_run - m_new) + acc_s;
+            m_run = m_new;
+          }
+        } else {  // EPI_DLOGITS
+          if (row_ok) {
+            float g[32];
+            const bool live = (row_a != 0.f) || (row_b != 0.f);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float q = ex2_approx(fmaf(__uint_as_float(r[j]), p.scale_log2, -row_lz2));
+              g[j] = live ? row_a * q : 0.f;
+            }
+            while (next_idx < col0 + 32) {
+              const int off = next_idx - col0;
+              const float bp = row_b * p.p_sorted[(long long)row * p.Ktop + cur];
+#pragma unroll
+              for (int j = 0; j < 32; ++j) g[j] -= (off == j) ? bp : 0.f;
+              ++cur;
+              next_idx = cur < nv ? idxrow[cur] : 0x7fffffff;
+            }
+            __nv_bfloat16* dst = p.G + (long long)row * p.ldg + col0;
+            if (full_w) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                uint4 v;
+                v.x = pack_bf16x2(g[j], g[j + 1]);
+                v.y = pack_bf16x2(g[j + 2], g[j + 3]);
+                v.z = pack_bf16x2(g[j + 4], g[j + 5]);
+                v.w = pack_bf16x2(g[j + 6], g[j + 7]);
+                *reinterpret_cast<uint4*>(dst + j) = v;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(g[j]);
+            }
+          }
+        }
+      }
+      // accumulator stage is free again
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+
+      if (EPI == EPI_LSE) {
+        if (row_ok) {
+          p.part_m[(long long)nt * p.part_stride + row] = m_run;
+          p.part_s[(long long)nt * p.part_stride + row] = s_run;
+        }
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+}
+
+}  // namespace kdkl

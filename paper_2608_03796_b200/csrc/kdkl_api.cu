@@ -1,0 +1,443 @@
+// Host side of the C ABI: argument checks, workspace carving, tensor-map encoding and the
+// per-chunk launch schedule of Algorithm 1. Enqueue-only: nothing here synchronises except
+// kdkl_status() and the host-buffer entry point, which say so.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "../../include/kdkl.h"
+#include "aux_kernels.cuh"
+#include "gemm_tcgen05.cuh"
+
+namespace kdkl {
+
+static thread_local char g_err[512] = "";
+static thread_local int64_t g_launches = 0;
+
+static int cuda_fail(const char* what, cudaError_t e) {
+  snprintf(g_err, sizeof(g_err), "%s: %s", what, cudaGetErrorString(e));
+  return KDKL_ERR_CUDA;
+}
+#define KDKL_CUDA(call)                                   \
+  do {                                                    \
+    cudaError_t e__ = (call);                             \
+    if (e__ != cudaSuccess) return cuda_fail(#call, e__); \
+  } while (0)
+#define KDKL_LAUNCHED(name)                               \
+  do {                                                    \
+    cudaError_t e__ = cudaGetLastError();                 \
+    if (e__ != cudaSuccess) return cuda_fail(name, e__);  \
+    ++g_launches;                                         \
+  } while (0)
+
+// ------------------------------------------------------------------ tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(p);
+  return fn;
+}
+
+// 2-D bf16 tensor, `inner` contiguous elements per row, `outer` rows of `pitch_bytes`;
+// boxes of box_inner x box_outer written to shared memory with the 128-byte swizzle;
+// out-of-bounds elements read as zero.
+static int make_tmap_bf16(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_bytes,
+                          uint32_t box_inner, uint32_t box_outer) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) { snprintf(g_err, sizeof(g_err), "cuTensorMapEncodeTiled entry point not found"); return KDKL_ERR_CUDA; }
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {pitch_bytes};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(g_err, sizeof(g_err), "cuTensorMapEncodeTiled failed (%d): inner=%llu outer=%llu pitch=%llu box=%ux%u",
+             (int)r, (unsigned long long)inner, (unsigned long long)outer, (unsigned long long)pitch_bytes, box_inner,
+             box_outer);
+    return KDKL_ERR_CUDA;
+  }
+  return KDKL_OK;
+}
+
+// ------------------------------------------------------------------ device / launch helpers
+struct DeviceInfo { int sm_count; int cc_major; bool ok; };
+static int device_info(DeviceInfo* di) {
+  int dev = 0;
+  KDKL_CUDA(cudaGetDevice(&dev));
+  KDKL_CUDA(cudaDeviceGetAttribute(&di->sm_count, cudaDevAttrMultiProcessorCount, dev));
+  KDKL_CUDA(cudaDeviceGetAttribute(&di->cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+  return KDKL_OK;
+}
+
+template <int EPI, bool A_MN, bool B_MN>
+static int launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int sm_count,
+                       cudaStream_t st) {
+  auto kern = gemm_tcgen05_kernel<EPI, A_MN, B_MN>;
+  static bool attr_set = false;   // per instantiation
+  if (!attr_set) {
+    KDKL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES));
+    attr_set = true;
+  }
+  const int tiles = p.m_tiles * p.n_tiles;
+  const int grid = tiles < sm_count ? tiles : sm_count;
+  kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ta, tb, p);
+  KDKL_LAUNCHED("gemm_tcgen05_kernel");
+  return KDKL_OK;
+}
+
+// ------------------------------------------------------------------ workspace
+static inline size_t up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WsLayout {
+  long long C, Cpad, Vpad, n_tiles_v;
+  size_t hdr, idx_sorted, p_sorted, perm, zg, colread, nvalid, M, Hent, lz2, logZ, loss_tok, coefA, coefB;
+  size_t part_m, part_s, G, total;
+};
+
+static WsLayout ws_layout(long long T, long long H, long long V, int K, long long chunk) {
+  WsLayout L;
+  L.C = chunk <= 0 ? 4096 : chunk;
+  if (L.C > T) L.C = T;
+  L.Cpad = (long long)up((size_t)L.C, 128);
+  L.Vpad = (long long)up((size_t)V, 64);
+  L.n_tiles_v = (V + BN - 1) / BN;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = up(o + bytes, 256); return at; };
+  L.hdr = take(256);
+  L.idx_sorted = take((size_t)T * K * 4);
+  L.p_sorted = take((size_t)T * K * 4);
+  L.perm = take((size_t)T * K * 2);
+  L.zg = take((size_t)T * K * 4);
+  L.colread = take((size_t)T * K * 4);
+  L.nvalid = take((size_t)T * 4);
+  L.M = take((size_t)T * 4);
+  L.Hent = take((size_t)T * 4);
+  L.lz2 = take((size_t)T * 4);
+  L.logZ = take((size_t)T * 4);
+  L.loss_tok = take((size_t)T * 4);
+  L.coefA = take((size_t)T * 4);
+  L.coefB = take((size_t)T * 4);
+  L.part_m = take((size_t)L.n_tiles_v * L.Cpad * 4);
+  L.part_s = take((size_t)L.n_tiles_v * L.Cpad * 4);
+  L.G = take((size_t)L.Cpad * L.Vpad * 2);
+  L.total = o;
+  return L;
+}
+
+static int check_common(const void* hidden, const void* weight, long long T, long long H, long long V, int K,
+                        long long chunk, float tau, const kdkl_options* opt, const void* ws, size_t ws_bytes,
+                        kdkl_options* eff, WsLayout* L) {
+  if (!hidden || !weight || !ws) return KDKL_ERR_NULL;
+  if (T < 1 || H < 1 || V < 1 || K < 1 || K > KDKL_MAX_K || (H % 8) != 0 || V >= (1ll << 31) || T >= (1ll << 31))
+    return KDKL_ERR_SHAPE;
+  if (!(tau > 0.f) || chunk < 0) return KDKL_ERR_ARG;
+  memset(eff, 0, sizeof(*eff));
+  if (opt) {
+    if (opt->struct_size != (int32_t)sizeof(kdkl_options)) return KDKL_ERR_ARG;
+    *eff = *opt;
+  }
+  if (eff->teacher_mode < 0 || eff->teacher_mode > 1) return KDKL_ERR_ARG;
+  if (eff->teacher_mode == 1 && tau != 1.0f) return KDKL_ERR_ARG;
+  if (eff->dhidden_dtype < 0 || eff->dhidden_dtype > 1) return KDKL_ERR_ARG;
+  if (((uintptr_t)hidden & 15) || ((uintptr_t)weight & 15) || ((uintptr_t)ws & 15)) return KDKL_ERR_ALIGN;
+  *L = ws_layout(T, H, V, K, chunk);
+  if (ws_bytes < L->total) return KDKL_ERR_WORKSPACE;
+  DeviceInfo di;
+  int rc = device_info(&di);
+  if (rc) return rc;
+  if (di.cc_major != 10) return KDKL_ERR_ARCH;
+  return KDKL_OK;
+}
+
+template <typename Tp>
+static Tp* at(void* ws, size_t off) { return reinterpret_cast<Tp*>(reinterpret_cast<uint8_t*>(ws) + off); }
+
+static int next_pow2(int x) { int p = 2; while (p < x) p <<= 1; return p; }
+
+}  // namespace kdkl
+
+using namespace kdkl;
+
+extern "C" {
+
+const char* kdkl_last_error(void) { return g_err; }
+int64_t kdkl_last_launch_count(void) { return g_launches; }
+
+size_t kdkl_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options*) {
+  if (T < 1 || H < 1 || V < 1 || K < 1) return 0;
+  return ws_layout(T, H, V, K, chunk).total;
+}
+
+int kdkl_forward(const void* hidden, const void* weight, const int32_t* topk_idx, const float* topk_val,
+                 const float* teacher_lse, const uint8_t* loss_mask, int64_t T, int64_t H, int64_t V, int32_t K,
+                 int64_t chunk, float tau, const kdkl_options* opt, void* ws, size_t ws_bytes, float* loss_out,
+                 float* loss_per_token, float* gathered_logits, int32_t* gathered_idx, void* cuda_stream) {
+  g_launches = 0;
+  if (!topk_idx || !topk_val || !loss_out) return KDKL_ERR_NULL;
+  kdkl_options o;
+  WsLayout L;
+  int rc = check_common(hidden, weight, T, H, V, K, chunk, tau, opt, ws, ws_bytes, &o, &L);
+  if (rc) return rc;
+  DeviceInfo di;
+  if ((rc = device_info(&di))) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  WsHeader* hdr = at<WsHeader>(ws, L.hdr);
+  const float inv_tau = 1.0f / tau;
+
+  header_reset_kernel<<<1, 32, 0, st>>>(hdr);
+  KDKL_LAUNCHED("header_reset_kernel");
+
+  const int Kpad = next_pow2(K);
+  const size_t prep_smem = (size_t)PREP_WARPS * Kpad * (4 + 4 + 2);
+  prep_kernel<<<(unsigned)((T + PREP_WARPS - 1) / PREP_WARPS), PREP_WARPS * 32, prep_smem, st>>>(
+      topk_idx, topk_val, teacher_lse, loss_mask, T, (int)V, K, Kpad, inv_tau, o.teacher_mode,
+      at<int>(ws, L.idx_sorted), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<int>(ws, L.nvalid),
+      at<float>(ws, L.M), at<float>(ws, L.Hent), hdr);
+  KDKL_LAUNCHED("prep_kernel");
+
+  CUtensorMap tmW;
+  if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, BN))) return rc;
+
+  for (long long s0 = 0; s0 < T; s0 += L.C) {
+    const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
+    CUtensorMap tmA;
+    const __nv_bfloat16* hA = reinterpret_cast<const __nv_bfloat16*>(hidden) + s0 * H;
+    if ((rc = make_tmap_bf16(&tmA, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, BK, BM))) return rc;
+    GemmParams p;
+    memset(&p, 0, sizeof(p));
+    p.M = (int)rows; p.N = (int)V; p.K = (int)H;
+    p.m_tiles = (int)((rows + BM - 1) / BM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1;
+    p.status = &hdr->status; p.go = nullptr;
+    p.scale_log2 = kLog2e * inv_tau; p.Ktop = K;
+    p.idx_sorted = at<int>(ws, L.idx_sorted) + s0 * K;
+    p.nvalid = at<int>(ws, L.nvalid) + s0;
+    p.part_m = at<float>(ws, L.part_m); p.part_s = at<float>(ws, L.part_s); p.part_stride = L.Cpad;
+    p.zg = at<float>(ws, L.zg) + s0 * K;
+    p.colread = at<int>(ws, L.colread) + s0 * K;
+    if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, p, di.sm_count, st))) return rc;
+
+    combine_kernel<<<(unsigned)((rows + 31) / 32), 256, 0, st>>>(
+        at<float>(ws, L.part_m), at<float>(ws, L.part_s), L.Cpad, (int)L.n_tiles_v, (int)rows, s0, K, inv_tau,
+        at<int>(ws, L.nvalid), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<float>(ws, L.zg),
+        at<int>(ws, L.colread), at<float>(ws, L.M), at<float>(ws, L.Hent), loss_mask, at<float>(ws, L.lz2),
+        at<float>(ws, L.logZ), at<float>(ws, L.loss_tok), loss_per_token, gathered_logits, gathered_idx, hdr);
+    KDKL_LAUNCHED("combine_kernel");
+  }
+  loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, tau, H, V, K,
+                                         loss_out, hdr);
+  KDKL_LAUNCHED("loss_reduce_kernel");
+  return KDKL_OK;
+}
+
+int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_mask, int64_t T, int64_t H,
+                  int64_t V, int32_t K, int64_t chunk, float tau, const kdkl_options* opt, float grad_loss, void* ws,
+                  size_t ws_bytes, void* dhidden, float* dweight, void* cuda_stream) {
+  g_launches = 0;
+  if (!dhidden || !dweight) return KDKL_ERR_NULL;
+  kdkl_options o;
+  WsLayout L;
+  int rc = check_common(hidden, weight, T, H, V, K, chunk, tau, opt, ws, ws_bytes, &o, &L);
+  if (rc) return rc;
+  if (((uintptr_t)dhidden & 15) || ((uintptr_t)dweight & 15)) return KDKL_ERR_ALIGN;
+  DeviceInfo di;
+  if ((rc = device_info(&di))) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  WsHeader* hdr = at<WsHeader>(ws, L.hdr);
+  const int* go = &hdr->go;
+  const float inv_tau = 1.0f / tau;
+
+  bwd_coef_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(at<float>(ws, L.M), loss_mask, T, H, V, K, grad_loss,
+                                                               inv_tau, at<float>(ws, L.coefA),
+                                                               at<float>(ws, L.coefB), hdr);
+  KDKL_LAUNCHED("bwd_coef_kernel");
+
+  __nv_bfloat16* G = at<__nv_bfloat16>(ws, L.G);
+  // W as the K-major B operand of the recompute GEMM, and as the MN-major B operand of dH = G W
+  CUtensorMap tmW, tmWmn;
+  if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, BN))) return rc;
+  if ((rc = make_tmap_bf16(&tmWmn, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, 64, BK))) return rc;
+
+  long long ci = 0;
+  for (long long s0 = 0; s0 < T; s0 += L.C, ++ci) {
+    const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
+    const __nv_bfloat16* hA = reinterpret_cast<const __nv_bfloat16*>(hidden) + s0 * H;
+    CUtensorMap tmA, tmG, tmGmn, tmhmn;
+    if ((rc = make_tmap_bf16(&tmA, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, BK, BM))) return rc;
+
+    // B1: recompute logits, G = coefA * q - coefB * p
+    GemmParams p;
+    memset(&p, 0, sizeof(p));
+    p.M = (int)rows; p.N = (int)V; p.K = (int)H;
+    p.m_tiles = (int)((rows + BM - 1) / BM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1;
+    p.status = &hdr->status; p.go = go;
+    p.scale_log2 = kLog2e * inv_tau; p.Ktop = K;
+    p.idx_sorted = at<int>(ws, L.idx_sorted) + s0 * K;
+    p.nvalid = at<int>(ws, L.nvalid) + s0;
+    p.p_sorted = at<float>(ws, L.p_sorted) + s0 * K;
+    p.lz2 = at<float>(ws, L.lz2) + s0;
+    p.coefA = at<float>(ws, L.coefA) + s0;
+    p.coefB = at<float>(ws, L.coefB) + s0;
+    p.G = G; p.ldg = L.Vpad;
+    if ((rc = launch_gemm<EPI_DLOGITS, false, false>(tmA, tmW, p, di.sm_count, st))) return rc;
+
+    // B2: dH[chunk] = G W   (M = rows, N = H, K = V)
+    if ((rc = make_tmap_bf16(&tmG, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, BK, BM))) return rc;
+    GemmParams p2;
+    memset(&p2, 0, sizeof(p2));
+    p2.M = (int)rows; p2.N = (int)H; p2.K = (int)V;
+    p2.m_tiles = (int)((rows + BM - 1) / BM); p2.n_tiles = (int)((H + BN - 1) / BN); p2.m_inner = 0;
+    p2.status = &hdr->status; p2.go = go;
+    p2.ldc = H; p2.accumulate = 0;
+    if (o.dhidden_dtype == 0) {
+      p2.C = reinterpret_cast<__nv_bfloat16*>(dhidden) + s0 * H;
+      if ((rc = launch_gemm<EPI_STORE_BF16, false, true>(tmG, tmWmn, p2, di.sm_count, st))) return rc;
+    } else {
+      p2.C = reinterpret_cast<float*>(dhidden) + s0 * H;
+      if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, p2, di.sm_count, st))) return rc;
+    }
+
+    // B3: dW (+)= G^T h   (M = V, N = H, K = rows)
+    // both operands MN-major: G is [t, v] with v (= M) contiguous, h is [t, h] with h (= N) contiguous
+    if ((rc = make_tmap_bf16(&tmGmn, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, 64, BK))) return rc;
+    if ((rc = make_tmap_bf16(&tmhmn, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, 64, BK))) return rc;
+    GemmParams p3;
+    memset(&p3, 0, sizeof(p3));
+    p3.M = (int)V; p3.N = (int)H; p3.K = (int)rows;
+    p3.m_tiles = (int)((V + BM - 1) / BM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0;
+    p3.status = &hdr->status; p3.go = go;
+    p3.C = dweight; p3.ldc = H;
+    p3.accumulate = (ci > 0 || o.accumulate_dweight) ? 1 : 0;
+    if ((rc = launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, p3, di.sm_count, st))) return rc;
+  }
+  return KDKL_OK;
+}
+
+int kdkl_status(const void* ws, void* cuda_stream, int32_t* code, int64_t* detail) {
+  if (!ws || !code) return KDKL_ERR_NULL;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  WsHeader h;
+  KDKL_CUDA(cudaMemcpyAsync(&h, ws, sizeof(h), cudaMemcpyDeviceToHost, st));
+  KDKL_CUDA(cudaStreamSynchronize(st));
+  *code = h.status;
+  if (detail) { detail[0] = h.where; detail[1] = h.n_tokens; detail[2] = h.n_bad_idx; }
+  return KDKL_OK;
+}
+
+int kdkl_saved_state(void* ws, int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options*,
+                     const float** logZ, const float** mass) {
+  if (!ws) return KDKL_ERR_NULL;
+  if (T < 1 || H < 1 || V < 1 || K < 1) return KDKL_ERR_SHAPE;
+  WsLayout L = ws_layout(T, H, V, K, chunk);
+  if (logZ) *logZ = at<float>(ws, L.logZ);
+  if (mass) *mass = at<float>(ws, L.M);
+  return KDKL_OK;
+}
+
+// ------------------------------------------------------------------ host-buffer entry point
+struct ArenaLayout { size_t hidden, weight, idx, val, lse, mask, loss, dh, dw, ws, total; };
+static ArenaLayout arena_layout(long long T, long long H, long long V, int K, long long chunk, int dh_fp32) {
+  ArenaLayout A;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = up(o + bytes, 256); return at; };
+  A.hidden = take((size_t)T * H * 2);
+  A.weight = take((size_t)V * H * 2);
+  A.idx = take((size_t)T * K * 4);
+  A.val = take((size_t)T * K * 4);
+  A.lse = take((size_t)T * 4);
+  A.mask = take((size_t)T);
+  A.loss = take(256);
+  A.dh = take((size_t)T * H * (dh_fp32 ? 4 : 2));
+  A.dw = take((size_t)V * H * 4);
+  A.ws = take(ws_layout(T, H, V, K, chunk).total);
+  A.total = o;
+  return A;
+}
+
+size_t kdkl_host_arena_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options* opt) {
+  if (T < 1 || H < 1 || V < 1 || K < 1) return 0;
+  return arena_layout(T, H, V, K, chunk, opt ? opt->dhidden_dtype : 0).total;
+}
+
+int kdkl_forward_backward_host(const void* hidden, const void* weight, const int32_t* topk_idx, const float* topk_val,
+                               const float* teacher_lse, const uint8_t* loss_mask, int64_t T, int64_t H, int64_t V,
+                               int32_t K, int64_t chunk, float tau, const kdkl_options* opt, float grad_loss,
+                               void* arena, size_t arena_bytes, float* loss_out, void* dhidden_out,
+                               float* dweight_out, void* cuda_stream) {
+  if (!hidden || !weight || !topk_idx || !topk_val || !arena || !loss_out) return KDKL_ERR_NULL;
+  if (T < 1 || H < 1 || V < 1 || K < 1) return KDKL_ERR_SHAPE;
+  if ((uintptr_t)arena & 255) return KDKL_ERR_ALIGN;
+  const int dh32 = opt ? opt->dhidden_dtype : 0;
+  ArenaLayout A = arena_layout(T, H, V, K, chunk, dh32);
+  if (arena_bytes < A.total) return KDKL_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  uint8_t* d = reinterpret_cast<uint8_t*>(arena);
+  KDKL_CUDA(cudaMemcpyAsync(d + A.hidden, hidden, (size_t)T * H * 2, cudaMemcpyHostToDevice, st));
+  KDKL_CUDA(cudaMemcpyAsync(d + A.weight, weight, (size_t)V * H * 2, cudaMemcpyHostToDevice, st));
+  KDKL_CUDA(cudaMemcpyAsync(d + A.idx, topk_idx, (size_t)T * K * 4, cudaMemcpyHostToDevice, st));
+  KDKL_CUDA(cudaMemcpyAsync(d + A.val, topk_val, (size_t)T * K * 4, cudaMemcpyHostToDevice, st));
+  if (teacher_lse) KDKL_CUDA(cudaMemcpyAsync(d + A.lse, teacher_lse, (size_t)T * 4, cudaMemcpyHostToDevice, st));
+  if (loss_mask) KDKL_CUDA(cudaMemcpyAsync(d + A.mask, loss_mask, (size_t)T, cudaMemcpyHostToDevice, st));
+  const size_t ws_bytes = ws_layout(T, H, V, K, chunk).total;
+  int rc = kdkl_forward(d + A.hidden, d + A.weight, reinterpret_cast<int32_t*>(d + A.idx),
+                        reinterpret_cast<float*>(d + A.val), teacher_lse ? reinterpret_cast<float*>(d + A.lse) : nullptr,
+                        loss_mask ? d + A.mask : nullptr, T, H, V, K, chunk, tau, opt, d + A.ws, ws_bytes,
+                        reinterpret_cast<float*>(d + A.loss), nullptr, nullptr, nullptr, cuda_stream);
+  if (rc) return rc;
+  const int64_t fl = g_launches;
+  rc = kdkl_backward(d + A.hidden, d + A.weight, loss_mask ? d + A.mask : nullptr, T, H, V, K, chunk, tau, opt,
+                     grad_loss, d + A.ws, ws_bytes, d + A.dh, reinterpret_cast<float*>(d + A.dw), cuda_stream);
+  if (rc) return rc;
+  g_launches += fl;
+  KDKL_CUDA(cudaMemcpyAsync(loss_out, d + A.loss, 4, cudaMemcpyDeviceToHost, st));
+  if (dhidden_out)
+    KDKL_CUDA(cudaMemcpyAsync(dhidden_out, d + A.dh, (size_t)T * H * (dh32 ? 4 : 2), cudaMemcpyDeviceToHost, st));
+  if (dweight_out) KDKL_CUDA(cudaMemcpyAsync(dweight_out, d + A.dw, (size_t)V * H * 4, cudaMemcpyDeviceToHost, st));
+  KDKL_CUDA(cudaStreamSynchronize(st));
+  return KDKL_OK;
+}
+
+// ------------------------------------------------------------------ bare GEMM
+int kdkl_gemm_bf16(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K, int32_t a_mn, int32_t b_mn,
+                   int32_t* status, void* cuda_stream) {
+  g_launches = 0;
+  if (!A || !B || !C) return KDKL_ERR_NULL;
+  if (M < 1 || N < 1 || K < 1 || (M % 8) || (N % 8) || (K % 8)) return KDKL_ERR_SHAPE;
+  if (((uintptr_t)A & 15) || ((uintptr_t)B & 15) || ((uintptr_t)C & 15)) return KDKL_ERR_ALIGN;
+  DeviceInfo di;
+  int rc = device_info(&di);
+  if (rc) return rc;
+  if (di.cc_major != 10) return KDKL_ERR_ARCH;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  CUtensorMap ta, tb;
+  if (a_mn) rc = make_tmap_bf16(&ta, A, (uint64_t)M, (uint64_t)K, (uint64_t)M * 2, 64, BK);
+  else      rc = make_tmap_bf16(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)K * 2, BK, BM);
+  if (rc) return rc;
+  if (b_mn) rc = make_tmap_bf16(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)N * 2, 64, BK);
+  else      rc = make_tmap_bf16(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)K * 2, BK, BN);
+  if (rc) return rc;
+  GemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.M = (int)M; p.N = (int)N; p.K = (int)K;
+  p.m_tiles = (int)((M + BM - 1) / BM); p.n_tiles = (int)((N + BN - 1) / BN); p.m_inner = 1;
+  p.status = status; p.C = C; p.ldc = N; p.accumulate = 0;
+  if (a_mn && b_mn) return launch_gemm<EPI_STORE_F32, true, true>(ta, tb, p, di.sm_count, st);
+  if (a_mn) return launch_gemm<EPI_STORE_F32, true, false>(ta, tb, p, di.sm_count, st);
+  if (b_mn) return launch_gemm<EPI_STORE_F32, false, true>(ta, tb, p, di.sm_count, st);
+  return launch_gemm<EPI_STORE_F32, false, false>(ta, tb, p, di.sm_count, st);
+}
+
+}  // extern "C"
