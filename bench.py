@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the fused chunked KL loss (forward + backward over the LM head) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl reference]
+
+A step is one kdkl_forward + kdkl_backward over one batch of synthetic input (the paper's
+loss-only benchmark shape). Prints ONE JSON line: tokens/s for the whole job, with the
+roofline of the dominant kernel (timed live with CUDA events between kernels), an
+end-to-end number through the host-buffer entry point, the clocks seen during the timed
+region and the fp64 CPU oracle timed on this machine's host cores on a bounded sample.
+
+With N > 1 (launched by torch.distributed.run) every rank runs its own batch of T tokens:
+token batches are independent, so there is no data-path collective ("weak" scaling);
+torch.distributed is used for the barrier and the max over ranks of the device time.
+
+--impl reference times the CPU oracle (the reference arm for this build: the paper ships no
+code to run) on rank 0 and prints the same line with "impl": "reference".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "KL fwd+bwd tokens/s & % of bf16 tensor peak; peak HBM GB vs sequence length"
+FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.1):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {}
+        for n in dir(nv):
+            if n.startswith("nvmlClocksThrottleReason") and isinstance(getattr(nv, n), int):
+                names[getattr(nv, n)] = n[len("nvmlClocksThrottleReason"):]
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if bit and (r & bit) == bit and name not in ("None", "All"):
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join(timeout=2)
+
+    def summary(self):
+        s = sorted(self.samples)
+        med = s[len(s) // 2] if s else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def oracle_data(cfg, n_rows: int, dev_tensors=None):
+    """The first n_rows tokens of the workload as float64 numpy arrays (prepared once, outside any timing)."""
+    import torch
+    from paper_2608_03796_b200 import inputs as I
+    if dev_tensors is None:
+        device = "cuda" if torch.cuda.is_available() else "cpu"
+        d = I.make_inputs(cfg, device=device, rows=torch.arange(n_rows, dtype=torch.int64))
+    else:
+        d = {k: (v if (v is None or k == "weight") else v[:n_rows]) for k, v in dev_tensors.items()}
+    out = {"hidden": d["hidden"].cpu().double().numpy(), "weight": d["weight"].cpu().double().numpy(),
+           "topk_idx": d["topk_idx"].cpu().numpy(), "topk_val": d["topk_val"].cpu().numpy(),
+           "mask": None if d["mask"] is None else d["mask"].cpu().numpy()}
+    return out
+
+
+def oracle_sample(cfg, od):
+    """Time the fp64 oracle (forward + gradients) on the prepared sample. Returns (tokens/s, threads, seconds)."""
+    from oracle.kdkl_oracle import kdkl_oracle
+    n_rows = od["hidden"].shape[0]
+    t0 = time.perf_counter()
+    kdkl_oracle(od["hidden"], od["weight"], od["topk_idx"], od["topk_val"], tau=cfg.tau, mask=od["mask"],
+                want_grads=True)
+    dt = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    return n_rows / dt, threads, dt
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_rows = args.ref_rows or 128
+    vals = []
+    od = oracle_data(cfg, n_rows)
+    for i in range(args.warmup + args.steps):
+        tps, threads, dt = oracle_sample(cfg, od)
+        if i >= args.warmup:
+            vals.append((tps, dt))
+    tps = sum(v[0] for v in vals) / len(vals)
+    ms = 1e3 * sum(v[1] for v in vals) / len(vals)
+    sample = f"{n_rows} tokens of {cfg.name} per step, forward + gradients, dense fp64"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tps, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(cfg), "sample": sample},
+        "cpu_baseline": {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tps, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_name(cfg):
+    return (f"{cfg.name}: T={cfg.T} H={cfg.H} V={cfg.V} K={cfg.K} chunk={cfg.chunk} tau={cfg.tau} "
+            f"bf16 hidden/weight, top-K teacher ({cfg.idx_dist} indices)")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--impl", default="kdkl", choices=["kdkl", "reference"])
+    ap.add_argument("--ref-rows", type=int, default=0,
+                    help="tokens in the CPU-oracle sample (0: 768 for the cpu_baseline leg, 128 per reference step)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2608_03796_b200 import inputs as I
+    cfg = I.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2608_03796_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    import __graft_entry__ as entry
+    if rank == 0:
+        entry.build()
+    if world > 1:
+        dist.barrier()
+    B.lib()
+    peaks = load_peaks()
+
+    # every rank: its own batch (seed offset by rank), generated on the device
+    import dataclasses
+    rcfg = dataclasses.replace(cfg, seed=cfg.seed + rank)
+    d = I.make_inputs(rcfg, device=dev)
+    T, H, V, K = cfg.T, cfg.H, cfg.V, cfg.K
+    torch.cuda.synchronize()
+    torch.cuda.reset_peak_memory_stats()
+    base_mem = torch.cuda.memory_allocated()
+    op = B.FusedChunkedKL(T, H, V, K, chunk=cfg.chunk, temperature=cfg.tau, device=dev)
+
+    def step():
+        op.forward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], loss_mask=d["mask"])
+        op.backward(d["hidden"], d["weight"], loss_mask=d["mask"])
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    code, detail = op.status()
+    if code != 0:
+        raise SystemExit(f"device status {code} {detail}")
+    launches_per_step = op.launches
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with ClockSampler(local_rank) as clk:
+        ev0.record()
+        for _ in range(args.steps):
+            step()
+        ev1.record()
+        barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    tt = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    ms_total = float(tt.item())
+    ms_step = ms_total / args.steps
+    loss_val = float(op.loss.item())
+    peak_mem = torch.cuda.max_memory_allocated()
+    ws_bytes = op.workspace.numel()
+
+    # per-kernel times, live, with an event between kernels (a separate short run)
+    stage_acc = {}
+    n_prof = 3
+    for _ in range(n_prof):
+        st = B.kdkl_profile_stages(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], op.workspace, op.loss,
+                                   op.dhidden, op.dweight, loss_mask=d["mask"], chunk=cfg.chunk, temperature=cfg.tau)
+        for k, (ms, n) in st.items():
+            a = stage_acc.setdefault(k, [0.0, 0])
+            a[0] += ms
+            a[1] += n
+    stages = {k: {"ms_per_step": v[0] / n_prof, "launches_per_step": v[1] // n_prof,
+                  "ms_per_launch": (v[0] / v[1] if v[1] else 0.0)} for k, v in stage_acc.items()}
+    gemm_stages = ["fwd_gemm_lse", "bwd_gemm_dlogits", "dhidden_gemm", "dweight_gemm"]
+    dom = max(gemm_stages, key=lambda k: stages[k]["ms_per_step"])
+    C = min(cfg.chunk, T)
+    flops_per_launch = 2.0 * C * H * V             # each of the four GEMMs: 2 * chunk * H * V per launch
+    dom_tflops = flops_per_launch / (stages[dom]["ms_per_launch"] * 1e-3) / 1e12
+    long_step = ms_total > 1000.0
+    peak_key = "bf16_tflops_sustained" if long_step else "bf16_tflops"
+    peak = float(peaks.get(peak_key, FALLBACK_PEAKS[peak_key]))
+    for k in gemm_stages:
+        stages[k]["tflops"] = flops_per_launch / (stages[k]["ms_per_launch"] * 1e-3) / 1e12
+
+    # end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
+    e2e = None
+    if not args.no_e2e:
+        opt = None
+        arena = torch.empty(B.kdkl_host_arena_bytes(T, H, V, K, cfg.chunk), dtype=torch.uint8, device=dev)
+        hh = {k: (v.cpu().pin_memory() if v is not None else None) for k, v in d.items()}
+        loss_h = torch.zeros(1, dtype=torch.float32).pin_memory()
+        dh_h = torch.empty(T, H, dtype=torch.bfloat16).pin_memory()
+        dw_h = torch.empty(V, H, dtype=torch.float32).pin_memory()
+
+        def e2e_step():
+            B.kdkl_forward_backward_host(hh["hidden"], hh["weight"], hh["topk_idx"], hh["topk_val"], arena, loss_h,
+                                         dh_h, dw_h, loss_mask=hh["mask"], chunk=cfg.chunk, temperature=cfg.tau,
+                                         opt=opt)
+        e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / args.e2e_steps
+        et = torch.tensor([e_ms], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(et, op=dist.ReduceOp.MAX)
+        e_ms = float(et.item())
+        h2d = sum(v.numel() * v.element_size() for v in hh.values() if v is not None)
+        d2h = 4 + dh_h.numel() * 2 + dw_h.numel() * 4
+        assert abs(float(loss_h.item()) - loss_val) <= 1e-5 * abs(loss_val)
+        e2e = {"value": world * T / (e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
+        del arena
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline and world == 1:
+        tps, threads, dt = oracle_sample(cfg, oracle_data(cfg, args.ref_rows or 768, d))
+        cpu_baseline = {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                        "sample": f"{args.ref_rows or 768} tokens of {cfg.name}, forward + gradients, dense fp64, {dt:.1f} s"}
+
+    tokens_per_s = world * T / (ms_step * 1e-3)
+    step_tflops = cfg.flops / (ms_step * 1e-3) / 1e12
+    line = {
+        "metric": METRIC, "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": workload_name(cfg), "l2": "inputs larger than L2 (weight 1 GiB, dW 2 GiB per step)",
+                   "per_rank_tokens": T, "parallelism": f"independent batches x{world}"},
+        "tflops_per_gpu": step_tflops,
+        "frac_of_bf16_burst_peak": step_tflops / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"])),
+        "frac_of_bf16_sustained_peak": step_tflops / float(peaks.get("bf16_tflops_sustained",
+                                                                     FALLBACK_PEAKS["bf16_tflops_sustained"])),
+        "peaks": peaks.get("_source"),
+        "peak_mem_gb": peak_mem / 1e9, "workspace_gb": ws_bytes / 1e9, "input_mem_gb": base_mem / 1e9,
+        "loss": loss_val,
+        "clocks": clk.summary(),
+        "gpu_launches": launches_per_step * args.steps,
+        "e2e": e2e,
+        "roofline": {"bound": "tensor", "kernel": dom, "achieved": dom_tflops, "peak": peak, "unit": "TFLOP/s",
+                     "frac": dom_tflops / peak, "peak_kind": f"{peak_key} ({peaks.get('_source')})",
+                     "traffic": None, "ms_per_launch": stages[dom]["ms_per_launch"],
+                     "flops_per_launch": flops_per_launch},
+        "stages": stages,
+        "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

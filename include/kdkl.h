@@ -125,6 +125,18 @@ int kdkl_forward_backward_host(const void* hidden_bf16, const void* weight_bf16,
                                size_t arena_bytes, float* loss_out, void* dhidden_out, float* dweight_out,
                                void* cuda_stream);
 
+/* Forward + backward on DEVICE buffers with a CUDA event between every kernel; synchronises and
+ * returns, per stage, the summed device time in ms and the number of launches. Stages:
+ * 0 teacher prep, 1 forward GEMM + online log-sum-exp + gather, 2 partial combine, 3 loss reduce,
+ * 4 backward coefficients, 5 recompute GEMM + dlogits, 6 dhidden GEMM, 7 dweight GEMM.
+ * stage_ms and stage_launches are HOST arrays of 8. Arguments as kdkl_forward / kdkl_backward. */
+int kdkl_profile_stages(const void* hidden_bf16, const void* weight_bf16, const int32_t* topk_idx,
+                        const float* topk_val, const float* teacher_lse, const uint8_t* loss_mask,
+                        int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, float temperature,
+                        const kdkl_options* opt, float grad_loss, void* workspace, size_t workspace_bytes,
+                        float* loss_out, void* dhidden, float* dweight, void* cuda_stream,
+                        float* stage_ms, int32_t* stage_launches);
+
 /* The tensor-core mainloop on its own: C[M,N] (fp32, row-major) = A * B^T with bf16 operands.
  * a_mn = 0: A is [M, K] row-major; 1: A is stored [K, M]. b_mn likewise for B ([N, K] or [K, N]).
  * M, N, K multiples of 8. status: device int32[2] the caller zeroed, receives {KDKL_ERR_TIMEOUT, site}

@@ -97,7 +97,7 @@ def kdkl_oracle(hidden, weight, topk_idx, topk_val, tau=1.0, mask=None, teacher_
     logZ = np.zeros(T)
     zg = np.full((T, K), np.nan)
     dH = np.zeros((T, H)) if want_grads else None
-    dW = np.zeros((V, H)) if want_grads else None
+    dW = None
     g = np.where(msk, float(grad_loss) / N, 0.0) if N > 0 else np.zeros(T)
 
     step = T if not row_block else int(row_block)
@@ -139,12 +139,13 @@ def kdkl_oracle(hidden, weight, topk_idx, topk_val, tau=1.0, mask=None, teacher_
             # Eq. "grad": dL/dz_v = M q_v - p_v, times g/tau (chain rule through s = z/tau)
             dz = (g[r0:r1, None] / tau) * (M[r0:r1, None] * np.exp(logq) - p)
             dH[r0:r1] = dz @ W                            # Algorithm 1: dh = G W
-            dW += dz.T @ h[r0:r1]                         # Algorithm 1: dW += G^T h
+            dWb = dz.T @ h[r0:r1]                         # Algorithm 1: dW += G^T h
+            dW = dWb if dW is None else dW + dWb
 
     loss = float(loss_tok.sum() / N) if N > 0 else 0.0
     out = {"loss": loss, "loss_tok": loss_tok, "logZ": logZ, "M": M, "gathered_logits": zg,
            "gathered_idx": np.asarray(topk_idx).astype(np.int32).copy(), "n_bad_idx": n_bad, "N": N}
     if want_grads:
         out["dH"] = dH
-        out["dW"] = dW
+        out["dW"] = dW if dW is not None else np.zeros((V, H))
     return out

@@ -24,7 +24,7 @@ ERRORS = {
 
 EXPORTS = [
     "kdkl_workspace_bytes", "kdkl_forward", "kdkl_backward", "kdkl_status", "kdkl_saved_state",
-    "kdkl_host_arena_bytes", "kdkl_forward_backward_host", "kdkl_gemm_bf16", "kdkl_last_error",
+    "kdkl_host_arena_bytes", "kdkl_forward_backward_host", "kdkl_profile_stages", "kdkl_gemm_bf16", "kdkl_last_error",
     "kdkl_last_launch_count",
 ]
 
@@ -68,6 +68,9 @@ def lib() -> ctypes.CDLL:
     L.kdkl_forward_backward_host.restype = ctypes.c_int
     L.kdkl_forward_backward_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, f32, vp, sz,
                                              vp, vp, vp, vp]
+    L.kdkl_profile_stages.restype = ctypes.c_int
+    L.kdkl_profile_stages.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, f32, vp, sz,
+                                      vp, vp, vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
     L.kdkl_gemm_bf16.restype = ctypes.c_int
     L.kdkl_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, vp, vp]
     L.kdkl_last_error.restype = ctypes.c_char_p
@@ -160,6 +163,25 @@ def kdkl_forward_backward_host(hidden, weight, topk_idx, topk_val, arena, loss_o
                                             _opt_ptr(opt), grad_loss, _ptr(arena),
                                             arena.numel() * arena.element_size(), _ptr(loss_out), _ptr(dhidden_out),
                                             _ptr(dweight_out), _stream()))
+
+
+STAGES = ["prep", "fwd_gemm_lse", "combine", "loss_reduce", "bwd_coef", "bwd_gemm_dlogits", "dhidden_gemm",
+          "dweight_gemm"]
+
+
+def kdkl_profile_stages(hidden, weight, topk_idx, topk_val, workspace, loss_out, dhidden, dweight, *,
+                        teacher_lse=None, loss_mask=None, chunk=0, temperature=1.0, opt=None, grad_loss=1.0):
+    """Forward + backward with an event between kernels: {stage: (ms, launches)}. Synchronises."""
+    T, H = hidden.shape
+    V = weight.shape[0]
+    K = topk_idx.shape[1]
+    ms = (ctypes.c_float * 8)()
+    nl = (ctypes.c_int32 * 8)()
+    _check(lib().kdkl_profile_stages(_ptr(hidden), _ptr(weight), _ptr(topk_idx), _ptr(topk_val), _ptr(teacher_lse),
+                                     _ptr(loss_mask), T, H, V, K, chunk, temperature, _opt_ptr(opt), grad_loss,
+                                     _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(loss_out),
+                                     _ptr(dhidden), _ptr(dweight), _stream(), ms, nl))
+    return {STAGES[i]: (float(ms[i]), int(nl[i])) for i in range(8)}
 
 
 def kdkl_gemm_bf16(A, B, C, M, N, K, a_mn=0, b_mn=0, status=None) -> None:

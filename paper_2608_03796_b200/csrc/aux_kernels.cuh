@@ -54,6 +54,7 @@ __global__ void header_reset_kernel(WsHeader* hdr) {
 // original slot of every entry) that the GEMM epilogues walk with a cursor.
 // Ignored tokens (mask = 0) get an empty row: their teacher entries are never read.
 constexpr int PREP_WARPS = 4;
+constexpr int kKeyUnusable = 0x7ffffffe, kKeyPad = 0x7fffffff;
 __global__ void __launch_bounds__(PREP_WARPS * 32)
 prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val,
             const float* __restrict__ teacher_lse, const uint8_t* __restrict__ mask, long long T, int V, int K,
@@ -80,8 +81,10 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
   // load, validate, scaled values
   float mx = -INFINITY;
   int bad = 0;
+  // keys: a usable index < kKeyUnusable (real slot without a usable index) < kKeyPad (sort padding),
+  // so after the sort positions [nvalid, K) hold exactly the real slots that were not gathered
   for (int k = lane; k < Kpad; k += 32) {
-    int key = 0x7fffffff;
+    int key = k < K ? kKeyUnusable : kKeyPad;
     float u = -INFINITY;
     if (k < K) {
       const int id = topk_idx[t * K + k];
@@ -106,7 +109,7 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
     lam = mx + logf(s);
   }
   __syncwarp();
-  for (int k = lane; k < Kpad; k += 32) pv[k] = keys[k] != 0x7fffffff ? expf(pv[k] - lam) : 0.f;
+  for (int k = lane; k < Kpad; k += 32) pv[k] = keys[k] < kKeyUnusable ? expf(pv[k] - lam) : 0.f;
   __syncwarp();
   // bitonic sort by key, (p, slot) carried along
   for (int size = 2; size <= Kpad; size <<= 1) {
@@ -131,7 +134,7 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
   for (int j = lane; j < Kpad; j += 32) {
     const int key = keys[j];
     float pj = 0.f;
-    if (key != 0x7fffffff) {
+    if (key < kKeyUnusable) {
       nv++;
       if (j == 0 || keys[j - 1] != key) {
         pj = pv[j];

@@ -8,6 +8,8 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <vector>
+
 #include "../../include/kdkl.h"
 #include "aux_kernels.cuh"
 #include "gemm_tcgen05.cuh"
@@ -32,6 +34,26 @@ static int cuda_fail(const char* what, cudaError_t e) {
     if (e__ != cudaSuccess) return cuda_fail(name, e__);  \
     ++g_launches;                                         \
   } while (0)
+
+// ------------------------------------------------------------------ per-stage event timing
+// Off unless kdkl_profile_stages() is running on this thread. When on, every launch site first
+// records an event tagged with its stage; the time between consecutive events is charged to the
+// earlier one's stage.
+enum { ST_PREP = 0, ST_F1, ST_COMBINE, ST_REDUCE, ST_COEF, ST_B1, ST_B2, ST_B3, ST_END, ST_COUNT = ST_END };
+struct StageTimer {
+  bool on = false;
+  std::vector<cudaEvent_t> ev;
+  std::vector<int> stage;
+};
+static thread_local StageTimer g_timer;
+static void stage_mark(int stage, cudaStream_t st) {
+  if (!g_timer.on) return;
+  cudaEvent_t e;
+  if (cudaEventCreate(&e) != cudaSuccess) return;
+  cudaEventRecord(e, st);
+  g_timer.ev.push_back(e);
+  g_timer.stage.push_back(stage);
+}
 
 // ------------------------------------------------------------------ tensor maps
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -198,6 +220,7 @@ int kdkl_forward(const void* hidden, const void* weight, const int32_t* topk_idx
   WsHeader* hdr = at<WsHeader>(ws, L.hdr);
   const float inv_tau = 1.0f / tau;
 
+  stage_mark(ST_PREP, st);
   header_reset_kernel<<<1, 32, 0, st>>>(hdr);
   KDKL_LAUNCHED("header_reset_kernel");
 
@@ -228,7 +251,9 @@ int kdkl_forward(const void* hidden, const void* weight, const int32_t* topk_idx
     p.part_m = at<float>(ws, L.part_m); p.part_s = at<float>(ws, L.part_s); p.part_stride = L.Cpad;
     p.zg = at<float>(ws, L.zg) + s0 * K;
     p.colread = at<int>(ws, L.colread) + s0 * K;
+    stage_mark(ST_F1, st);
     if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, p, di.sm_count, st))) return rc;
+    stage_mark(ST_COMBINE, st);
 
     combine_kernel<<<(unsigned)((rows + 31) / 32), 256, 0, st>>>(
         at<float>(ws, L.part_m), at<float>(ws, L.part_s), L.Cpad, (int)L.n_tiles_v, (int)rows, s0, K, inv_tau,
@@ -237,6 +262,7 @@ int kdkl_forward(const void* hidden, const void* weight, const int32_t* topk_idx
         at<float>(ws, L.logZ), at<float>(ws, L.loss_tok), loss_per_token, gathered_logits, gathered_idx, hdr);
     KDKL_LAUNCHED("combine_kernel");
   }
+  stage_mark(ST_REDUCE, st);
   loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, tau, H, V, K,
                                          loss_out, hdr);
   KDKL_LAUNCHED("loss_reduce_kernel");
@@ -260,6 +286,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
   const int* go = &hdr->go;
   const float inv_tau = 1.0f / tau;
 
+  stage_mark(ST_COEF, st);
   bwd_coef_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(at<float>(ws, L.M), loss_mask, T, H, V, K, grad_loss,
                                                                inv_tau, at<float>(ws, L.coefA),
                                                                at<float>(ws, L.coefB), hdr);
@@ -292,7 +319,9 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p.coefA = at<float>(ws, L.coefA) + s0;
     p.coefB = at<float>(ws, L.coefB) + s0;
     p.G = G; p.ldg = L.Vpad;
+    stage_mark(ST_B1, st);
     if ((rc = launch_gemm<EPI_DLOGITS, false, false>(tmA, tmW, p, di.sm_count, st))) return rc;
+    stage_mark(ST_B2, st);
 
     // B2: dH[chunk] = G W   (M = rows, N = H, K = V)
     if ((rc = make_tmap_bf16(&tmG, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, BK, BM))) return rc;
@@ -321,6 +350,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p3.status = &hdr->status; p3.go = go;
     p3.C = dweight; p3.ldc = H;
     p3.accumulate = (ci > 0 || o.accumulate_dweight) ? 1 : 0;
+    stage_mark(ST_B3, st);
     if ((rc = launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, p3, di.sm_count, st))) return rc;
   }
   return KDKL_OK;
@@ -408,6 +438,42 @@ int kdkl_forward_backward_host(const void* hidden, const void* weight, const int
   if (dweight_out) KDKL_CUDA(cudaMemcpyAsync(dweight_out, d + A.dw, (size_t)V * H * 4, cudaMemcpyDeviceToHost, st));
   KDKL_CUDA(cudaStreamSynchronize(st));
   return KDKL_OK;
+}
+
+// ------------------------------------------------------------------ per-stage profile
+int kdkl_profile_stages(const void* hidden, const void* weight, const int32_t* topk_idx, const float* topk_val,
+                        const float* teacher_lse, const uint8_t* loss_mask, int64_t T, int64_t H, int64_t V, int32_t K,
+                        int64_t chunk, float tau, const kdkl_options* opt, float grad_loss, void* ws, size_t ws_bytes,
+                        float* loss_out, void* dhidden, float* dweight, void* cuda_stream, float* stage_ms,
+                        int32_t* stage_launches) {
+  if (!stage_ms || !stage_launches) return KDKL_ERR_NULL;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  g_timer.on = true;
+  g_timer.ev.clear();
+  g_timer.stage.clear();
+  int rc = kdkl_forward(hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, T, H, V, K, chunk, tau, opt, ws,
+                        ws_bytes, loss_out, nullptr, nullptr, nullptr, cuda_stream);
+  const int64_t fl = g_launches;
+  if (rc == KDKL_OK)
+    rc = kdkl_backward(hidden, weight, loss_mask, T, H, V, K, chunk, tau, opt, grad_loss, ws, ws_bytes, dhidden,
+                       dweight, cuda_stream);
+  g_launches += fl;
+  stage_mark(ST_END, st);
+  g_timer.on = false;
+  cudaError_t e = cudaStreamSynchronize(st);
+  for (int i = 0; i < ST_COUNT; ++i) { stage_ms[i] = 0.f; stage_launches[i] = 0; }
+  for (size_t i = 0; e == cudaSuccess && i + 1 < g_timer.ev.size(); ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, g_timer.ev[i], g_timer.ev[i + 1]) == cudaSuccess) {
+      stage_ms[g_timer.stage[i]] += ms;
+      stage_launches[g_timer.stage[i]] += 1;
+    }
+  }
+  for (cudaEvent_t ev : g_timer.ev) cudaEventDestroy(ev);
+  g_timer.ev.clear();
+  g_timer.stage.clear();
+  if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
+  return rc;
 }
 
 // ------------------------------------------------------------------ bare GEMM
