@@ -144,6 +144,24 @@ int kdkl_profile_stages(const void* hidden_bf16, const void* weight_bf16, const 
 int kdkl_gemm_bf16(const void* A, const void* B, float* C, int64_t M, int64_t N, int64_t K,
                    int32_t a_mn, int32_t b_mn, int32_t* status, void* cuda_stream);
 
+/* (No counterpart in the paper: an addition for callers that cannot allocate device memory.)
+ * log Z[t] = logsumexp over the vocabulary of (W h_t) / temperature, the normaliser of Eq. "decomp",
+ * computed without any device allocation: the caller passes only inputs and the output, and the
+ * scratch for the per-vocab-tile partials is a fixed array inside the library (about 8 MiB, held by
+ * every GPU that loads the library until the process exits).
+ * Meant for code that may not call cudaMalloc: a plugin inside a server whose memory pool already owns
+ * the device, or a latency-critical callback that must stay out of the driver's allocator.
+ *   hidden_bf16 [T, H], weight_bf16 [V, H], logz_out [T] fp32: device pointers; H % 8 == 0;
+ *   V <= 262144 (larger V is rejected with KDKL_ERR_WORKSPACE and a message on stderr); any T >= 1
+ *   (processed 1024 tokens at a time). No cudaMalloc / cudaFree / allocating library call is made.
+ * The first call on each device also resolves the scratch array's device address and sets a kernel
+ * attribute; make that first call before any stream capture is open. All calls share the one scratch
+ * array and it keeps the previous call's contents (the parts that must start at zero are cleared on the
+ * stream at the start of each call): calls that overlap on the same GPU, on any streams, race.
+ * If a bounded wait inside the kernel expires, the affected outputs are NaN. */
+int kdkl_logz_noalloc(const void* hidden_bf16, const void* weight_bf16, int64_t T, int64_t H, int64_t V,
+                      float temperature, float* logz_out, void* cuda_stream);
+
 /* Text of the last KDKL_ERR_CUDA on this thread. */
 const char* kdkl_last_error(void);
 

@@ -25,7 +25,7 @@ ERRORS = {
 EXPORTS = [
     "kdkl_workspace_bytes", "kdkl_forward", "kdkl_backward", "kdkl_status", "kdkl_saved_state",
     "kdkl_host_arena_bytes", "kdkl_forward_backward_host", "kdkl_profile_stages", "kdkl_gemm_bf16", "kdkl_last_error",
-    "kdkl_last_launch_count",
+    "kdkl_last_launch_count", "kdkl_logz_noalloc",
 ]
 
 
@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
                                       vp, vp, vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
     L.kdkl_gemm_bf16.restype = ctypes.c_int
     L.kdkl_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, vp, vp]
+    L.kdkl_logz_noalloc.restype = ctypes.c_int
+    L.kdkl_logz_noalloc.argtypes = [vp, vp, i64, i64, i64, f32, vp, vp]
     L.kdkl_last_error.restype = ctypes.c_char_p
     L.kdkl_last_error.argtypes = []
     L.kdkl_last_launch_count.restype = ctypes.c_int64
@@ -186,6 +188,15 @@ def kdkl_profile_stages(hidden, weight, topk_idx, topk_val, workspace, loss_out,
 
 def kdkl_gemm_bf16(A, B, C, M, N, K, a_mn=0, b_mn=0, status=None) -> None:
     _check(lib().kdkl_gemm_bf16(_ptr(A), _ptr(B), _ptr(C), M, N, K, a_mn, b_mn, _ptr(status), _stream()))
+
+
+def kdkl_logz_noalloc(hidden, weight, logz_out, temperature=1.0) -> None:
+    """log Z per token with no device allocation by anyone: the scratch is a fixed array inside the
+    library (V <= 262144). For callers that may not call cudaMalloc (a plugin inside a server whose
+    pool owns the device, a latency-critical callback). Calls sharing a GPU must not overlap."""
+    T, H = hidden.shape
+    V = weight.shape[0]
+    _check(lib().kdkl_logz_noalloc(_ptr(hidden), _ptr(weight), T, H, V, temperature, _ptr(logz_out), _stream()))
 
 
 def kdkl_last_launch_count() -> int:
