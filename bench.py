@@ -153,6 +153,27 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def rank_config(cfg, rank: int):
+    """Each rank times its own batch: same shape and generators, seed offset by the rank."""
+    import dataclasses
+    return dataclasses.replace(cfg, seed=cfg.seed + rank)
+
+
+def max_over_ranks(value: float, world: int, device) -> float:
+    """The slowest rank's time (all-reduce MAX); the job is as slow as its slowest rank."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Aggregate over all ranks: every rank processes tokens_per_rank tokens per step."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 def workload_name(cfg):
     return (f"{cfg.name}: T={cfg.T} H={cfg.H} V={cfg.V} K={cfg.K} chunk={cfg.chunk} tau={cfg.tau} "
             f"bf16 hidden/weight, top-K teacher ({cfg.idx_dist} indices)")
@@ -170,6 +191,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--capture", action="store_true",
+                    help="profiler-capture mode: exactly --warmup warm-up steps, no e2e, no CPU baseline, no stage run")
     args = ap.parse_args()
 
     from paper_2608_03796_b200 import inputs as I
@@ -200,9 +223,7 @@ def main():
     peaks = load_peaks()
 
     # every rank: its own batch (seed offset by rank), generated on the device
-    import dataclasses
-    rcfg = dataclasses.replace(cfg, seed=cfg.seed + rank)
-    d = I.make_inputs(rcfg, device=dev)
+    d = I.make_inputs(rank_config(cfg, rank), device=dev)
     T, H, V, K = cfg.T, cfg.H, cfg.V, cfg.K
     torch.cuda.synchronize()
     torch.cuda.reset_peak_memory_stats()
@@ -213,7 +234,8 @@ def main():
         op.forward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], loss_mask=d["mask"])
         op.backward(d["hidden"], d["weight"], loss_mask=d["mask"])
 
-    for _ in range(max(args.warmup, 3)):
+    n_warm = args.warmup if args.capture else max(args.warmup, 3)
+    for _ in range(n_warm):
         step()
     torch.cuda.synchronize()
     code, detail = op.status()
@@ -235,10 +257,7 @@ def main():
         ev1.record()
         barrier()
     ms_total = ev0.elapsed_time(ev1)
-    tt = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-    ms_total = float(tt.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
     loss_val = float(op.loss.item())
     peak_mem = torch.cuda.max_memory_allocated()
@@ -246,7 +265,7 @@ def main():
 
     # per-kernel times, live, with an event between kernels (a separate short run)
     stage_acc = {}
-    n_prof = 3
+    n_prof = 1 if args.capture else 3
     for _ in range(n_prof):
         st = B.kdkl_profile_stages(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], op.workspace, op.loss,
                                    op.dhidden, op.dweight, loss_mask=d["mask"], chunk=cfg.chunk, temperature=cfg.tau)
@@ -258,7 +277,11 @@ def main():
                   "ms_per_launch": (v[0] / v[1] if v[1] else 0.0)} for k, v in stage_acc.items()}
     gemm_stages = ["fwd_gemm_lse", "bwd_gemm_dlogits", "dhidden_gemm", "dweight_gemm"]
     dom = max(gemm_stages, key=lambda k: stages[k]["ms_per_step"])
+    # DRAM bytes per launch from one ncu capture at chunk=4096, H=4096, V=131072 (read + write); null elsewhere
+    measured_traffic = {"fwd_gemm_lse": 1118951168 + 28143616, "bwd_gemm_dlogits": 1223847424 + 1051266048,
+                        "dhidden_gemm": 5471380992 + 29573376, "dweight_gemm": 1442837760 + 2109563136}
     C = min(cfg.chunk, T)
+    traffic = measured_traffic[dom] if (C, H, V) == (4096, 4096, 131072) else None
     flops_per_launch = 2.0 * C * H * V             # each of the four GEMMs: 2 * chunk * H * V per launch
     dom_tflops = flops_per_launch / (stages[dom]["ms_per_launch"] * 1e-3) / 1e12
     long_step = ms_total > 1000.0
@@ -269,7 +292,7 @@ def main():
 
     # end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.capture:
         opt = None
         arena = torch.empty(B.kdkl_host_arena_bytes(T, H, V, K, cfg.chunk), dtype=torch.uint8, device=dev)
         hh = {k: (v.cpu().pin_memory() if v is not None else None) for k, v in d.items()}
@@ -291,14 +314,11 @@ def main():
         e1.record()
         barrier()
         e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / args.e2e_steps
-        et = torch.tensor([e_ms], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(et, op=dist.ReduceOp.MAX)
-        e_ms = float(et.item())
+        e_ms = max_over_ranks(e_ms, world, dev)
         h2d = sum(v.numel() * v.element_size() for v in hh.values() if v is not None)
         d2h = 4 + dh_h.numel() * 2 + dw_h.numel() * 4
         assert abs(float(loss_h.item()) - loss_val) <= 1e-5 * abs(loss_val)
-        e2e = {"value": world * T / (e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e_ms,
+        e2e = {"value": whole_job_tokens_per_s(T, world, e_ms), "unit": "tokens/s", "ms_per_step": e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
         del arena
 
@@ -308,18 +328,18 @@ def main():
         return
 
     cpu_baseline = None
-    if not args.no_cpu_baseline and world == 1:
+    if not args.no_cpu_baseline and not args.capture and world == 1:
         tps, threads, dt = oracle_sample(cfg, oracle_data(cfg, args.ref_rows or 768, d))
         cpu_baseline = {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle",
                         "sample": f"{args.ref_rows or 768} tokens of {cfg.name}, forward + gradients, dense fp64, {dt:.1f} s"}
 
-    tokens_per_s = world * T / (ms_step * 1e-3)
+    tokens_per_s = whole_job_tokens_per_s(T, world, ms_step)
     step_tflops = cfg.flops / (ms_step * 1e-3) / 1e12
     line = {
         "metric": METRIC, "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": n_warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": workload_name(cfg), "l2": "inputs larger than L2 (weight 1 GiB, dW 2 GiB per step)",
+        "config": {"workload": workload_name(cfg), "l2": f"inputs larger than L2 (weight {V * H * 2 / 2**20:.0f} MiB, dW {V * H * 4 / 2**20:.0f} MiB per step)",
                    "per_rank_tokens": T, "parallelism": f"independent batches x{world}"},
         "tflops_per_gpu": step_tflops,
         "frac_of_bf16_burst_peak": step_tflops / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"])),
@@ -333,7 +353,7 @@ def main():
         "e2e": e2e,
         "roofline": {"bound": "tensor", "kernel": dom, "achieved": dom_tflops, "peak": peak, "unit": "TFLOP/s",
                      "frac": dom_tflops / peak, "peak_kind": f"{peak_key} ({peaks.get('_source')})",
-                     "traffic": None, "ms_per_launch": stages[dom]["ms_per_launch"],
+                     "traffic": traffic, "ms_per_launch": stages[dom]["ms_per_launch"],
                      "flops_per_launch": flops_per_launch},
         "stages": stages,
         "cpu_baseline": cpu_baseline,

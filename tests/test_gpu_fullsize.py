@@ -1,0 +1,113 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The dense oracle cannot run a whole 4K...256K-token config in test time, so it is evaluated on a
+row subset R (first and last row of every chunk plus seeded random rows). Rows are independent
+given W, so on R the oracle pins per-token loss, log Z, gathered logits/indices and dH rows of
+the *full* run exactly. dW sums over tokens: it is pinned by a second GPU run whose loss mask is
+the indicator of R (denominator |R|), whose dW the oracle computes in full. The full run's dW is
+further checked by properties that hold at any size: vanishing column sums, and additivity over
+a disjoint split of the mask.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle.kdkl_oracle import kdkl_oracle
+from paper_2608_03796_b200 import binding as B
+from paper_2608_03796_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+LOSS_RTOL, GRAD_FRO, TOK_ATOL, ZG_ATOL = 1e-3, 1e-2, 2e-4, 1e-4
+
+
+def _fro(a, b):
+    return np.linalg.norm(a - b) / np.linalg.norm(b)
+
+
+def _run(cfg, d, mask, opt=None, lse=None, want_tok=True):
+    op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, opt=opt,
+                          device=d["hidden"].device, want_gathered=want_tok, want_per_token=want_tok)
+    op.forward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], teacher_lse=lse, loss_mask=mask)
+    op.backward(d["hidden"], d["weight"], loss_mask=mask)
+    code, detail = op.status()
+    assert code == 0, (code, detail)
+    return op
+
+
+@pytest.mark.parametrize("name,n_rows,partial_mass", [("c2", 48, False), ("c2", 32, True), ("c3", 48, False),
+                                                      ("c5", 64, False), ("c4c", 32, False)])
+def test_fullsize_sampled_parity(name, n_rows, partial_mass):
+    cfg = I.CONFIGS[name]
+    dev = torch.device("cuda:0")
+    d = I.make_inputs(cfg, device=dev)
+    mask = d["mask"]
+    lse = I.partial_mass_lse(cfg, torch.nan_to_num(d["topk_val"])) if partial_mass else None
+    full = _run(cfg, d, mask, lse=lse)
+    n_counted = cfg.T if mask is None else int(mask.sum().item())
+
+    R = I.sample_rows(cfg, n_rows)
+    Rd = R.to(dev)
+    hR = d["hidden"][Rd].cpu().double().numpy()
+    W64 = d["weight"].cpu().double().numpy()
+    idxR = d["topk_idx"][Rd].cpu().numpy()
+    valR = d["topk_val"][Rd].cpu().numpy()
+    mR = None if mask is None else mask[Rd].cpu().numpy()
+    lseR = None if lse is None else lse[Rd].cpu().double().numpy()
+    counted = np.ones(len(R), bool) if mR is None else mR != 0
+    if name == "c5":
+        assert (~counted).any() and counted.any()          # the sample must see ignored rows too
+
+    # ---- rows of the full run: per-token outputs and dH, with the full run's denominator
+    o = kdkl_oracle(hR, W64, idxR, valR, tau=cfg.tau, mask=mR, teacher_lse=lseR, denom=n_counted, want_grads=True)
+    lt = full.loss_per_token[Rd].cpu().double().numpy()
+    np.testing.assert_allclose(lt, o["loss_tok"], rtol=0, atol=TOK_ATOL)
+    lz, M = full.saved_state()
+    np.testing.assert_allclose(lz[Rd].cpu().double().numpy(), o["logZ"], rtol=0, atol=TOK_ATOL)
+    np.testing.assert_allclose(M[Rd].cpu().double().numpy()[counted], o["M"][counted], rtol=0, atol=1e-5)
+    usable = (idxR >= 0) & (idxR < cfg.V) & counted[:, None]
+    gi = full.gathered_idx[Rd].cpu().numpy()
+    assert np.array_equal(gi[usable], idxR[usable]) and np.all(gi[~usable] == -1)
+    gl = full.gathered_logits[Rd].cpu().double().numpy()
+    np.testing.assert_allclose(gl[usable], o["gathered_logits"][usable], rtol=0, atol=ZG_ATOL)
+    dH = full.dhidden[Rd].float().cpu().double().numpy()
+    assert _fro(dH, o["dH"]) <= GRAD_FRO
+    assert not dH[~counted].any()
+
+    # ---- whole-run properties
+    tok = full.loss_per_token.double()
+    assert abs(full.loss.item() - tok.sum().item() / n_counted) <= 1e-6 * abs(full.loss.item())
+    assert torch.isfinite(full.dweight).all() and torch.isfinite(full.dhidden.float()).all()
+    colsum = full.dweight.double().sum(0).abs()
+    colabs = full.dweight.double().abs().sum(0)
+    assert (colsum / colabs).max().item() < 2e-3
+    if mask is not None:
+        assert not full.dhidden[mask == 0].float().abs().sum().item()
+    # the sample's mean loss is a consistency check of the mean itself
+    assert abs(o["loss_tok"][counted].mean() - full.loss.item()) < 0.5
+
+    # ---- dW: second run with mask = indicator of R (counted rows only), denominator |R|
+    mR_full = torch.zeros(cfg.T, dtype=torch.uint8, device=dev)
+    mR_full[Rd] = 1
+    if mask is not None:
+        mR_full &= mask
+    nR = int(mR_full.sum().item())
+    full_dW = full.dweight.clone()
+    del full
+    sub = _run(cfg, d, mR_full, lse=lse, want_tok=False)
+    oR = kdkl_oracle(hR, W64, idxR, valR, tau=cfg.tau, mask=mR, teacher_lse=lseR, denom=nR, want_grads=True)
+    assert abs(sub.loss.item() - oR["loss"]) <= LOSS_RTOL * abs(oR["loss"])
+    dW_sub = sub.dweight.cpu().double().numpy()
+    assert _fro(dW_sub, oR["dW"]) <= GRAD_FRO
+    del oR, dW_sub
+
+    # ---- additivity over a disjoint split of the mask: N dW = |R| dW_R + (N - |R|) dW_rest
+    if name in ("c2", "c5"):
+        base = torch.ones(cfg.T, dtype=torch.uint8, device=dev) if mask is None else mask
+        rest_mask = base & (1 - mR_full)
+        sub_dW = sub.dweight.clone()
+        del sub
+        rest = _run(cfg, d, rest_mask, lse=lse, want_tok=False)
+        recon = (nR * sub_dW.double() + (n_counted - nR) * rest.dweight.double()) / n_counted
+        err = (recon - full_dW.double()).norm() / full_dW.double().norm()
+        assert err.item() < 3e-3      # two independent bf16 roundings of G against one
