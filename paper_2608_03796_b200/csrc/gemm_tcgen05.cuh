@@ -13,6 +13,7 @@
 // and the shared-memory descriptors.
 //
 // Epilogues (the fused parts of the loss):
+// Output tiles leave through swizzled shared-memory boxes and TMA store / reduce-add.
 //   EPI_STORE_F32   plain fp32 store or += (dWeight accumulation, Algorithm 1 "dW += G^T h")
 //   EPI_STORE_BF16  bf16 store (dHidden, Algorithm 1 "dh = G W")
 //   EPI_LSE         forward: per (row, vocab tile) online max / sum-exp of z/tau and gather of
@@ -34,7 +35,9 @@ constexpr int B_STAGE_BYTES = BN * BK * 2;   // 32 KiB
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int GEMM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
-constexpr int GEMM_SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int STAGING_WARP_BYTES = 2 * 4096;   // per epilogue warp: two 32-row x 128-byte output boxes
+constexpr int STAGING_BYTES = 4 * STAGING_WARP_BYTES;
+constexpr int GEMM_SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
 enum { EPI_STORE_F32 = 0, EPI_STORE_BF16 = 1, EPI_LSE = 2, EPI_DLOGITS = 3 };
 
@@ -44,10 +47,8 @@ struct GemmParams {
   int m_inner;               // 1: consecutive tile ids walk M first (B panel shared), 0: N first
   int* status;               // device status word pair {code, where}
   const int* go;             // optional: kernel returns at once when *go == 0
-  // EPI_STORE_*
-  void* C;                   // fp32 or bf16 [M, ldc]
-  long long ldc;
-  int accumulate;            // fp32 only: 1 -> C += D
+  // EPI_STORE_F32: 1 -> output += D (TMA reduce-add), 0 -> output = D. Outputs go through tmC.
+  int accumulate;
   // EPI_LSE / EPI_DLOGITS: all row-indexed pointers are already offset to this chunk's row 0
   float scale_log2;          // log2(e) / tau
   int Ktop;                  // teacher slots per row
@@ -62,8 +63,6 @@ struct GemmParams {
   const float* coefA;        // [rows] g_t * M_t / tau
   const float* coefB;        // [rows] g_t / tau
   const float* p_sorted;     // [rows, Ktop]
-  __nv_bfloat16* G;          // [rows, ldg]
-  long long ldg;
 };
 
 __device__ __forceinline__ int lower_bound_i32(const int* a, int n, int key) {
@@ -97,13 +96,14 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 template <int EPI, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const GemmParams p) {
+                    const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
-  // barriers and bookkeeping live after the stage ring
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * STAGE_BYTES);
-  const uint32_t bar0 = smem_base + STAGES * STAGE_BYTES;
+  // after the stage ring: the epilogue's output staging boxes, then barriers and bookkeeping
+  const uint32_t staging0 = smem_base + STAGES * STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * STAGE_BYTES + STAGING_BYTES);
+  const uint32_t bar0 = staging0 + STAGING_BYTES;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
@@ -123,6 +123,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     mbar_fence_init();
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
+    if (EPI != EPI_LSE) tma_prefetch_desc(&tmC);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
@@ -219,7 +220,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int lg = warp & 3;                   // TMEM lane group this warp may read
     const int row_in_tile = lg * 32 + lane;
-    uint32_t lt = 0;
+    constexpr bool kBf16Out = (EPI == EPI_STORE_BF16 || EPI == EPI_DLOGITS);
+    uint32_t lt = 0, nbox = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
       int mt, nt;
@@ -251,56 +253,21 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint32_t taddr = tmem_base + (uint32_t(lg * 32) << 16) + acc * BN;
 
       float m_run = -INFINITY, s_run = 0.f;
+      const int box_row0 = m0 + lg * 32;       // first output row of this warp's boxes
+      const bool box_ok = box_row0 < p.M;      // warp-uniform
 #pragma unroll 1
       for (int w = 0; w < BN / 32; ++w) {
         const int col0 = n0 + w * 32;
-        if (col0 >= p.N) break;                // uniform: whole window past the edge
+        // uniform: whole window past the edge. bf16 outputs are staged as pairs of windows
+        // (64 columns = one 128-byte row), so a pair is always completed.
+        if (col0 >= p.N && (!kBf16Out || (w & 1) == 0)) break;
         uint32_t r[32];
         __syncwarp();
         tmem_ld32(taddr + w * 32, r);
         tmem_ld_wait();
         const bool full_w = col0 + 32 <= p.N;
 
-        if (EPI == EPI_STORE_F32) {
-          if (row_ok) {
-            float* dst = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col0;
-            if (full_w && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
-                                       __uint_as_float(r[j + 3]));
-                if (p.accumulate) {
-                  const float4 o = *reinterpret_cast<const float4*>(dst + j);
-                  v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-                }
-                *reinterpret_cast<float4*>(dst + j) = v;
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (col0 + j < p.N) dst[j] = __uint_as_float(r[j]) + (p.accumulate ? dst[j] : 0.f);
-            }
-          }
-        } else if (EPI == EPI_STORE_BF16) {
-          if (row_ok) {
-            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col0;
-            if (full_w && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                uint4 v;
-                v.x = pack_bf16x2(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-                v.y = pack_bf16x2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-                v.z = pack_bf16x2(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
-                v.w = pack_bf16x2(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
-                *reinterpret_cast<uint4*>(dst + j) = v;
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(r[j]));
-            }
-          }
-        } else if (EPI == EPI_LSE) {
+        if (EPI == EPI_LSE) {
           if (row_ok) {
             // gather the student logit at every teacher index that falls in this window
             while (next_idx < col0 + 32) {
@@ -325,39 +292,60 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             s_run = s_run * ex2_approx(m_run - m_new) + acc_s;
             m_run = m_new;
           }
-        } else {  // EPI_DLOGITS
-          if (row_ok) {
-            float g[32];
-            const bool live = (row_a != 0.f) || (row_b != 0.f);
+        } else {
+          // Output path: the warp's 32 rows x 128 bytes go to a swizzled shared-memory box (16-byte
+          // chunk c of row i sits at chunk c ^ (i & 7), the layout a 128-byte-swizzle tensor map
+          // expects) and leave with one TMA store / reduce-add; two boxes alternate.
+          const uint32_t sbox = staging0 + (warp - 2) * STAGING_WARP_BYTES + (nbox & 1u) * 4096u;
+          const uint32_t srow = sbox + lane * 128;
+          const bool first_half = !kBf16Out || (w & 1) == 0;
+          if (first_half) {
+            if (lane == 0) bulk_wait_read<1>();   // the store issued two boxes ago has read this box
+            __syncwarp();
+          }
+          if (EPI == EPI_STORE_F32) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const float q = ex2_approx(fmaf(__uint_as_float(r[j]), p.scale_log2, -row_lz2));
-              g[j] = live ? row_a * q : 0.f;
-            }
-            while (next_idx < col0 + 32) {
-              const int off = next_idx - col0;
-              const float bp = row_b * p.p_sorted[(long long)row * p.Ktop + cur];
+            for (int c = 0; c < 8; ++c)
+              st_shared_v4(srow + ((c ^ (lane & 7)) << 4), r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+          } else {
+            uint32_t v[16];
+            if (EPI == EPI_STORE_BF16) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) g[j] -= (off == j) ? bp : 0.f;
-              ++cur;
-              next_idx = cur < nv ? idxrow[cur] : 0x7fffffff;
-            }
-            __nv_bfloat16* dst = p.G + (long long)row * p.ldg + col0;
-            if (full_w) {
+              for (int j = 0; j < 16; ++j) v[j] = pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+            } else {  // EPI_DLOGITS
+              float g[32];
+              const bool live = (row_a != 0.f) || (row_b != 0.f);
 #pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                uint4 v;
-                v.x = pack_bf16x2(g[j], g[j + 1]);
-                v.y = pack_bf16x2(g[j + 2], g[j + 3]);
-                v.z = pack_bf16x2(g[j + 4], g[j + 5]);
-                v.w = pack_bf16x2(g[j + 6], g[j + 7]);
-                *reinterpret_cast<uint4*>(dst + j) = v;
+              for (int j = 0; j < 32; ++j) {
+                const float q = ex2_approx(fmaf(__uint_as_float(r[j]), p.scale_log2, -row_lz2));
+                g[j] = live ? row_a * q : 0.f;
               }
-            } else {
+              while (next_idx < col0 + 32) {
+                const int off = next_idx - col0;
+                const float bp = row_b * p.p_sorted[(long long)row * p.Ktop + cur];
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(g[j]);
+                for (int j = 0; j < 32; ++j) g[j] -= (off == j) ? bp : 0.f;
+                ++cur;
+                next_idx = cur < nv ? idxrow[cur] : 0x7fffffff;
+              }
+#pragma unroll
+              for (int j = 0; j < 16; ++j) v[j] = pack_bf16x2(g[2 * j], g[2 * j + 1]);
             }
+            const int cbase = (w & 1) * 4;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              st_shared_v4(srow + (((cbase + c) ^ (lane & 7)) << 4), v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+          }
+          if (!kBf16Out || (w & 1) == 1) {
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0 && box_ok) {
+              const int cx = kBf16Out ? col0 - 32 : col0;
+              if (EPI == EPI_STORE_F32 && p.accumulate) tma_reduce_add_2d(&tmC, sbox, cx, box_row0);
+              else tma_store_2d(&tmC, sbox, cx, box_row0);
+            }
+            if (lane == 0) bulk_commit();
+            ++nbox;
           }
         }
       }
@@ -373,6 +361,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       }
     }
+    if (EPI != EPI_LSE && lane == 0) bulk_wait_all();   // every output box has been written
   }
 
   // ---------------------------------------------------------------- teardown

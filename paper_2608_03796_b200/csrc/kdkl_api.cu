@@ -75,15 +75,15 @@ static EncodeTiledFn get_encode_fn() {
 // 2-D bf16 tensor, `inner` contiguous elements per row, `outer` rows of `pitch_bytes`;
 // boxes of box_inner x box_outer written to shared memory with the 128-byte swizzle;
 // out-of-bounds elements read as zero.
-static int make_tmap_bf16(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_bytes,
-                          uint32_t box_inner, uint32_t box_outer) {
+static int make_tmap(CUtensorMap* m, CUtensorMapDataType dtype, const void* base, uint64_t inner, uint64_t outer,
+                     uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_outer) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) { snprintf(g_err, sizeof(g_err), "cuTensorMapEncodeTiled entry point not found"); return KDKL_ERR_CUDA; }
   cuuint64_t dims[2] = {inner, outer};
   cuuint64_t strides[1] = {pitch_bytes};
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  CUresult r = fn(m, dtype, 2, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -93,6 +93,18 @@ static int make_tmap_bf16(CUtensorMap* m, const void* base, uint64_t inner, uint
     return KDKL_ERR_CUDA;
   }
   return KDKL_OK;
+}
+
+static int make_tmap_bf16(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_bytes,
+                          uint32_t box_inner, uint32_t box_outer) {
+  return make_tmap(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, base, inner, outer, pitch_bytes, box_inner, box_outer);
+}
+// Output maps: the epilogue stores boxes of 32 rows x 128 bytes (32 fp32 or 64 bf16 columns).
+static int make_tmap_out_f32(CUtensorMap* m, void* base, uint64_t cols, uint64_t rows, uint64_t ld_elems) {
+  return make_tmap(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, base, cols, rows, ld_elems * 4, 32, 32);
+}
+static int make_tmap_out_bf16(CUtensorMap* m, void* base, uint64_t cols, uint64_t rows, uint64_t ld_elems) {
+  return make_tmap(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, base, cols, rows, ld_elems * 2, 64, 32);
 }
 
 // ------------------------------------------------------------------ device / launch helpers
@@ -106,8 +118,8 @@ static int device_info(DeviceInfo* di) {
 }
 
 template <int EPI, bool A_MN, bool B_MN>
-static int launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, int sm_count,
-                       cudaStream_t st) {
+static int launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const GemmParams& p,
+                       int sm_count, cudaStream_t st) {
   auto kern = gemm_tcgen05_kernel<EPI, A_MN, B_MN>;
   static bool attr_set = false;   // per instantiation
   if (!attr_set) {
@@ -116,7 +128,7 @@ static int launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const GemmP
   }
   const int tiles = p.m_tiles * p.n_tiles;
   const int grid = tiles < sm_count ? tiles : sm_count;
-  kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ta, tb, p);
+  kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ta, tb, tc, p);
   KDKL_LAUNCHED("gemm_tcgen05_kernel");
   return KDKL_OK;
 }
@@ -252,7 +264,7 @@ int kdkl_forward(const void* hidden, const void* weight, const int32_t* topk_idx
     p.zg = at<float>(ws, L.zg) + s0 * K;
     p.colread = at<int>(ws, L.colread) + s0 * K;
     stage_mark(ST_F1, st);
-    if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, p, di.sm_count, st))) return rc;
+    if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA /*no output map*/, p, di.sm_count, st))) return rc;
     stage_mark(ST_COMBINE, st);
 
     combine_kernel<<<(unsigned)((rows + 31) / 32), 256, 0, st>>>(
@@ -298,6 +310,9 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
   if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, BN))) return rc;
   if ((rc = make_tmap_bf16(&tmWmn, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, 64, BK))) return rc;
 
+  CUtensorMap tmdW;
+  if ((rc = make_tmap_out_f32(&tmdW, dweight, (uint64_t)H, (uint64_t)V, (uint64_t)H))) return rc;
+
   long long ci = 0;
   for (long long s0 = 0; s0 < T; s0 += L.C, ++ci) {
     const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
@@ -318,9 +333,10 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p.lz2 = at<float>(ws, L.lz2) + s0;
     p.coefA = at<float>(ws, L.coefA) + s0;
     p.coefB = at<float>(ws, L.coefB) + s0;
-    p.G = G; p.ldg = L.Vpad;
+    CUtensorMap tmGout;
+    if ((rc = make_tmap_out_bf16(&tmGout, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad))) return rc;
     stage_mark(ST_B1, st);
-    if ((rc = launch_gemm<EPI_DLOGITS, false, false>(tmA, tmW, p, di.sm_count, st))) return rc;
+    if ((rc = launch_gemm<EPI_DLOGITS, false, false>(tmA, tmW, tmGout, p, di.sm_count, st))) return rc;
     stage_mark(ST_B2, st);
 
     // B2: dH[chunk] = G W   (M = rows, N = H, K = V)
@@ -330,13 +346,16 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p2.M = (int)rows; p2.N = (int)H; p2.K = (int)V;
     p2.m_tiles = (int)((rows + BM - 1) / BM); p2.n_tiles = (int)((H + BN - 1) / BN); p2.m_inner = 0;
     p2.status = &hdr->status; p2.go = go;
-    p2.ldc = H; p2.accumulate = 0;
+    p2.accumulate = 0;
+    CUtensorMap tmdH;
     if (o.dhidden_dtype == 0) {
-      p2.C = reinterpret_cast<__nv_bfloat16*>(dhidden) + s0 * H;
-      if ((rc = launch_gemm<EPI_STORE_BF16, false, true>(tmG, tmWmn, p2, di.sm_count, st))) return rc;
+      if ((rc = make_tmap_out_bf16(&tmdH, reinterpret_cast<__nv_bfloat16*>(dhidden) + s0 * H, (uint64_t)H,
+                                   (uint64_t)rows, (uint64_t)H))) return rc;
+      if ((rc = launch_gemm<EPI_STORE_BF16, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
     } else {
-      p2.C = reinterpret_cast<float*>(dhidden) + s0 * H;
-      if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, p2, di.sm_count, st))) return rc;
+      if ((rc = make_tmap_out_f32(&tmdH, reinterpret_cast<float*>(dhidden) + s0 * H, (uint64_t)H, (uint64_t)rows,
+                                  (uint64_t)H))) return rc;
+      if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
     }
 
     // B3: dW (+)= G^T h   (M = V, N = H, K = rows)
@@ -348,10 +367,9 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p3.M = (int)V; p3.N = (int)H; p3.K = (int)rows;
     p3.m_tiles = (int)((V + BM - 1) / BM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0;
     p3.status = &hdr->status; p3.go = go;
-    p3.C = dweight; p3.ldc = H;
     p3.accumulate = (ci > 0 || o.accumulate_dweight) ? 1 : 0;
     stage_mark(ST_B3, st);
-    if ((rc = launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, p3, di.sm_count, st))) return rc;
+    if ((rc = launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, tmdW, p3, di.sm_count, st))) return rc;
   }
   return KDKL_OK;
 }
@@ -499,11 +517,13 @@ int kdkl_gemm_bf16(const void* A, const void* B, float* C, int64_t M, int64_t N,
   memset(&p, 0, sizeof(p));
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
   p.m_tiles = (int)((M + BM - 1) / BM); p.n_tiles = (int)((N + BN - 1) / BN); p.m_inner = 1;
-  p.status = status; p.C = C; p.ldc = N; p.accumulate = 0;
-  if (a_mn && b_mn) return launch_gemm<EPI_STORE_F32, true, true>(ta, tb, p, di.sm_count, st);
-  if (a_mn) return launch_gemm<EPI_STORE_F32, true, false>(ta, tb, p, di.sm_count, st);
-  if (b_mn) return launch_gemm<EPI_STORE_F32, false, true>(ta, tb, p, di.sm_count, st);
-  return launch_gemm<EPI_STORE_F32, false, false>(ta, tb, p, di.sm_count, st);
+  p.status = status; p.accumulate = 0;
+  CUtensorMap tc;
+  if ((rc = make_tmap_out_f32(&tc, C, (uint64_t)N, (uint64_t)M, (uint64_t)N))) return rc;
+  if (a_mn && b_mn) return launch_gemm<EPI_STORE_F32, true, true>(ta, tb, tc, p, di.sm_count, st);
+  if (a_mn) return launch_gemm<EPI_STORE_F32, true, false>(ta, tb, tc, p, di.sm_count, st);
+  if (b_mn) return launch_gemm<EPI_STORE_F32, false, true>(ta, tb, tc, p, di.sm_count, st);
+  return launch_gemm<EPI_STORE_F32, false, false>(ta, tb, tc, p, di.sm_count, st);
 }
 
 }  // extern "C"

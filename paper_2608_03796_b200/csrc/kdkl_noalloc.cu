@@ -175,7 +175,7 @@ extern "C" int kdkl_logz_noalloc(const void* hidden_bf16, const void* weight_bf1
     p.part_stride = kPassRows;
     const int tiles = p.m_tiles * p.n_tiles;
     const int grid = tiles < pd->sm_count ? tiles : pd->sm_count;
-    gemm_tcgen05_kernel<EPI_LSE, false, false><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(tmA, tmW, p);
+    gemm_tcgen05_kernel<EPI_LSE, false, false><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(tmA, tmW, tmA /*no output map*/, p);
     logz_combine_kernel<<<(rows + 31) / 32, 256, 0, st>>>(p.part_m, p.part_s, n_tiles, rows, p.status, logz_out + s0);
     if (cudaGetLastError() != cudaSuccess) return KDKL_ERR_CUDA;
   }
