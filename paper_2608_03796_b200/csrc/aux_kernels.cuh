@@ -283,4 +283,28 @@ __global__ void bwd_coef_kernel(const float* __restrict__ Mv, const uint8_t* __r
   coefB[t] = g * inv_tau;
 }
 
+// ------------------------------------------------------------------------------------ split-K fix-up
+// out = part[0] + part[1] + ... in that fixed order (fp32), then one rounding to bf16 if asked.
+// part holds `splits` slabs `slab` elements apart; n4 = number of float4 groups to produce.
+__global__ void __launch_bounds__(256)
+splitk_fixup_kernel(const float* __restrict__ part, long long slab, int splits, long long n4,
+                    __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32, const int* go) {
+  if (go != nullptr && *go == 0) return;
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  float4 a = reinterpret_cast<const float4*>(part)[i];
+  for (int sidx = 1; sidx < splits; ++sidx) {
+    const float4 b = reinterpret_cast<const float4*>(part + (long long)sidx * slab)[i];
+    a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+  }
+  if (out_f32) reinterpret_cast<float4*>(out_f32)[i] = a;
+  if (out_bf16) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
+    uint2 v;
+    v.x = *reinterpret_cast<uint32_t*>(&lo);
+    v.y = *reinterpret_cast<uint32_t*>(&hi);
+    reinterpret_cast<uint2*>(out_bf16)[i] = v;
+  }
+}
+
 }  // namespace kdkl

@@ -45,6 +45,9 @@ struct GemmParams {
   int M, N, K;               // valid extents of this launch
   int m_tiles, n_tiles;
   int m_inner;               // 1: consecutive tile ids walk M first (B panel shared), 0: N first
+  int k_splits;              // >= 1: each tile's contraction is cut into this many work units, each
+                             // writing its own partial output (split s goes to output rows + s * split_rows)
+  int split_rows;
   int* status;               // device status word pair {code, where}
   const int* go;             // optional: kernel returns at once when *go == 0
   // EPI_STORE_F32: 1 -> output += D (TMA reduce-add), 0 -> output = D. Outputs go through tmC.
@@ -136,6 +139,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   const int num_tiles = p.m_tiles * p.n_tiles;
   const int kblocks = (p.K + BK - 1) / BK;
+  // work units: unit u = split * num_tiles + tile; a unit contracts k-blocks [kb0, kb1)
+  const int num_units = num_tiles * p.k_splits;
+  const int kb_per_split = (kblocks + p.k_splits - 1) / p.k_splits;
+  auto unit_decode = [&](int unit, int& tile, int& split, int& kb0, int& kb1) {
+    split = unit / num_tiles;
+    tile = unit - split * num_tiles;
+    kb0 = split * kb_per_split;
+    kb1 = kb0 + kb_per_split < kblocks ? kb0 + kb_per_split : kblocks;
+  };
 
   auto tile_coords = [&](int tile, int& mt, int& nt) {
     if (p.m_inner) { mt = tile % p.m_tiles; nt = tile / p.m_tiles; }
@@ -147,11 +159,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (lane == 0) {
       uint32_t it = 0, issued = 0, last_par = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        int mt, nt;
+      for (int unit = blockIdx.x; unit < num_units && ok; unit += gridDim.x) {
+        int tile, split, kb0, kb1, mt, nt;
+        unit_decode(unit, tile, split, kb0, kb1);
         tile_coords(tile, mt, nt);
         const int m0 = mt * BM, n0 = nt * BN;
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
@@ -190,13 +203,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint32_t idesc = make_idesc_bf16(BM, BN, A_MN ? 1u : 0u, B_MN ? 1u : 0u);
       uint32_t it = 0, lt = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+      for (int unit = blockIdx.x; unit < num_units && ok; unit += gridDim.x, ++lt) {
+        int tile, split, kb0, kb1;
+        unit_decode(unit, tile, split, kb0, kb1);
         const uint32_t acc = lt & 1u;
         const uint32_t aph = (lt >> 1) & 1u;
         if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + acc * BN;
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, 3)) { ok = false; break; }
@@ -209,7 +224,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                                      : make_smem_desc(sa + j * (UMMA_K * 2), 0, 1024);
             const uint64_t bd = B_MN ? make_smem_desc(sb + j * (UMMA_K * 128), BK * 128, 1024)
                                      : make_smem_desc(sb + j * (UMMA_K * 2), 0, 1024);
-            umma_bf16(tmem_d, ad, bd, idesc, (kb > 0 || j > 0) ? 1u : 0u);
+            umma_bf16(tmem_d, ad, bd, idesc, (kb > kb0 || j > 0) ? 1u : 0u);
           }
           umma_commit(empty_bar(s));           // frees the stage when these MMAs have read it
         }
@@ -223,8 +238,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     constexpr bool kBf16Out = (EPI == EPI_STORE_BF16 || EPI == EPI_DLOGITS);
     uint32_t lt = 0, nbox = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
-      int mt, nt;
+    for (int unit = blockIdx.x; unit < num_units && ok; unit += gridDim.x, ++lt) {
+      int tile, split, kb0, kb1, mt, nt;
+      unit_decode(unit, tile, split, kb0, kb1);
       tile_coords(tile, mt, nt);
       const int m0 = mt * BM, n0 = nt * BN;
       const int row = m0 + row_in_tile;
@@ -341,8 +357,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             __syncwarp();
             if (lane == 0 && box_ok) {
               const int cx = kBf16Out ? col0 - 32 : col0;
-              if (EPI == EPI_STORE_F32 && p.accumulate) tma_reduce_add_2d(&tmC, sbox, cx, box_row0);
-              else tma_store_2d(&tmC, sbox, cx, box_row0);
+              const int cy = box_row0 + split * p.split_rows;
+              if (EPI == EPI_STORE_F32 && p.accumulate) tma_reduce_add_2d(&tmC, sbox, cx, cy);
+              else tma_store_2d(&tmC, sbox, cx, cy);
             }
             if (lane == 0) bulk_commit();
             ++nbox;

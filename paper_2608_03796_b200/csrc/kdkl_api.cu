@@ -126,8 +126,8 @@ static int launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUten
     KDKL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES));
     attr_set = true;
   }
-  const int tiles = p.m_tiles * p.n_tiles;
-  const int grid = tiles < sm_count ? tiles : sm_count;
+  const int units = p.m_tiles * p.n_tiles * p.k_splits;
+  const int grid = units < sm_count ? units : sm_count;
   kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ta, tb, tc, p);
   KDKL_LAUNCHED("gemm_tcgen05_kernel");
   return KDKL_OK;
@@ -136,10 +136,28 @@ static int launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUten
 // ------------------------------------------------------------------ workspace
 static inline size_t up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// How many work units to cut each output tile's contraction into so that the units fill whole
+// waves of SMs: the smallest count (<= 4, each unit keeping >= 32 k-blocks) that reaches 95 %
+// wave efficiency, else the most efficient one. Sized for the 148 SMs of a B200.
+static int choose_k_splits(long long tiles, long long kblocks) {
+  const long long sms = 148;
+  int best = 1;
+  double best_eff = 0.0;
+  for (int sp = 1; sp <= 4; ++sp) {
+    if (sp > 1 && kblocks / sp < 32) break;
+    const long long units = tiles * sp;
+    const double eff = (double)units / (double)(((units + sms - 1) / sms) * sms);
+    if (eff > best_eff + 1e-9) { best_eff = eff; best = sp; }
+    if (eff >= 0.95) break;
+  }
+  return best;
+}
+
 struct WsLayout {
   long long C, Cpad, Vpad, n_tiles_v;
+  int dh_splits;             // split-K factor of the dH GEMM at full chunks
   size_t hdr, idx_sorted, p_sorted, perm, zg, colread, nvalid, M, Hent, lz2, logZ, loss_tok, coefA, coefB;
-  size_t part_m, part_s, G, total;
+  size_t part_m, part_s, G, dh_part, total;
 };
 
 static WsLayout ws_layout(long long T, long long H, long long V, int K, long long chunk) {
@@ -168,6 +186,8 @@ static WsLayout ws_layout(long long T, long long H, long long V, int K, long lon
   L.part_m = take((size_t)L.n_tiles_v * L.Cpad * 4);
   L.part_s = take((size_t)L.n_tiles_v * L.Cpad * 4);
   L.G = take((size_t)L.Cpad * L.Vpad * 2);
+  L.dh_splits = choose_k_splits(((L.C + BM - 1) / BM) * ((H + BN - 1) / BN), (V + BK - 1) / BK);
+  L.dh_part = take(L.dh_splits > 1 ? (size_t)L.dh_splits * L.Cpad * H * 4 : 0);
   L.total = o;
   return L;
 }
@@ -255,7 +275,7 @@ int kdkl_forward(const void* hidden, const void* weight, const int32_t* topk_idx
     GemmParams p;
     memset(&p, 0, sizeof(p));
     p.M = (int)rows; p.N = (int)V; p.K = (int)H;
-    p.m_tiles = (int)((rows + BM - 1) / BM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1;
+    p.m_tiles = (int)((rows + BM - 1) / BM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1; p.k_splits = 1;
     p.status = &hdr->status; p.go = nullptr;
     p.scale_log2 = kLog2e * inv_tau; p.Ktop = K;
     p.idx_sorted = at<int>(ws, L.idx_sorted) + s0 * K;
@@ -324,7 +344,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     GemmParams p;
     memset(&p, 0, sizeof(p));
     p.M = (int)rows; p.N = (int)V; p.K = (int)H;
-    p.m_tiles = (int)((rows + BM - 1) / BM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1;
+    p.m_tiles = (int)((rows + BM - 1) / BM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1; p.k_splits = 1;
     p.status = &hdr->status; p.go = go;
     p.scale_log2 = kLog2e * inv_tau; p.Ktop = K;
     p.idx_sorted = at<int>(ws, L.idx_sorted) + s0 * K;
@@ -347,8 +367,23 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p2.m_tiles = (int)((rows + BM - 1) / BM); p2.n_tiles = (int)((H + BN - 1) / BN); p2.m_inner = 0;
     p2.status = &hdr->status; p2.go = go;
     p2.accumulate = 0;
+    // a short last chunk may want a different split; never more than the workspace was sized for
+    int sp = choose_k_splits((long long)p2.m_tiles * p2.n_tiles, (V + BK - 1) / BK);
+    if (sp > L.dh_splits) sp = L.dh_splits;
+    p2.k_splits = sp;
     CUtensorMap tmdH;
-    if (o.dhidden_dtype == 0) {
+    if (sp > 1) {
+      // partial sums of each split go to fp32 slabs [split][Cpad, H]; a fixed-order fix-up adds them
+      float* part = at<float>(ws, L.dh_part);
+      p2.split_rows = (int)L.Cpad;
+      if ((rc = make_tmap_out_f32(&tmdH, part, (uint64_t)H, (uint64_t)sp * L.Cpad, (uint64_t)H))) return rc;
+      if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
+      const long long n4 = rows * H / 4;
+      splitk_fixup_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(
+          part, (long long)L.Cpad * H, sp, n4, o.dhidden_dtype == 0 ? reinterpret_cast<__nv_bfloat16*>(dhidden) + s0 * H : nullptr,
+          o.dhidden_dtype == 1 ? reinterpret_cast<float*>(dhidden) + s0 * H : nullptr, go);
+      KDKL_LAUNCHED("splitk_fixup_kernel");
+    } else if (o.dhidden_dtype == 0) {
       if ((rc = make_tmap_out_bf16(&tmdH, reinterpret_cast<__nv_bfloat16*>(dhidden) + s0 * H, (uint64_t)H,
                                    (uint64_t)rows, (uint64_t)H))) return rc;
       if ((rc = launch_gemm<EPI_STORE_BF16, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
@@ -365,7 +400,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     GemmParams p3;
     memset(&p3, 0, sizeof(p3));
     p3.M = (int)V; p3.N = (int)H; p3.K = (int)rows;
-    p3.m_tiles = (int)((V + BM - 1) / BM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0;
+    p3.m_tiles = (int)((V + BM - 1) / BM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0; p3.k_splits = 1;
     p3.status = &hdr->status; p3.go = go;
     p3.accumulate = (ci > 0 || o.accumulate_dweight) ? 1 : 0;
     stage_mark(ST_B3, st);
@@ -516,7 +551,7 @@ int kdkl_gemm_bf16(const void* A, const void* B, float* C, int64_t M, int64_t N,
   GemmParams p;
   memset(&p, 0, sizeof(p));
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
-  p.m_tiles = (int)((M + BM - 1) / BM); p.n_tiles = (int)((N + BN - 1) / BN); p.m_inner = 1;
+  p.m_tiles = (int)((M + BM - 1) / BM); p.n_tiles = (int)((N + BN - 1) / BN); p.m_inner = 1; p.k_splits = 1;
   p.status = status; p.accumulate = 0;
   CUtensorMap tc;
   if ((rc = make_tmap_out_f32(&tc, C, (uint64_t)N, (uint64_t)M, (uint64_t)N))) return rc;

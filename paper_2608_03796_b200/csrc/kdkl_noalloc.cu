@@ -164,7 +164,7 @@ extern "C" int kdkl_logz_noalloc(const void* hidden_bf16, const void* weight_bf1
     GemmParams p;
     memset(&p, 0, sizeof(p));
     p.M = rows; p.N = (int)V; p.K = (int)H;
-    p.m_tiles = (rows + BM - 1) / BM; p.n_tiles = n_tiles; p.m_inner = 1;
+    p.m_tiles = (rows + BM - 1) / BM; p.n_tiles = n_tiles; p.m_inner = 1; p.k_splits = 1;
     p.status = reinterpret_cast<int*>(sc + kOffStatus);
     p.scale_log2 = 1.4426950408889634f / temperature;
     p.Ktop = 1;
