@@ -551,7 +551,8 @@ int kdkl_gemm_bf16(const void* A, const void* B, float* C, int64_t M, int64_t N,
   GemmParams p;
   memset(&p, 0, sizeof(p));
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
-  p.m_tiles = (int)((M + BM - 1) / BM); p.n_tiles = (int)((N + BN - 1) / BN); p.m_inner = 1; p.k_splits = 1;
+  p.m_tiles = (int)((M + BM - 1) / BM); p.n_tiles = (int)((N + BN - 1) / BN); p.k_splits = 1;
+  p.m_inner = p.m_tiles <= p.n_tiles ? 1 : 0;   // walk the shorter dimension first: the other operand streams once
   p.status = status; p.accumulate = 0;
   CUtensorMap tc;
   if ((rc = make_tmap_out_f32(&tc, C, (uint64_t)N, (uint64_t)M, (uint64_t)N))) return rc;

@@ -1,0 +1,178 @@
+"""Sequence-length sweep of the fused chunked KL loss: iteration rate and peak memory versus T.
+
+    python -m paper_2608_03796_b200.sweep --out profiles/sweep_sequence_length.md
+
+Mirrors the paper's loss-only benchmark (appendix "Toy Loss-Kernel Benchmark Configuration"): every
+setting runs in a fresh process so that an out-of-memory failure cannot contaminate later
+measurements; timing is the mean forward + backward time after warm-up; memory is the peak
+allocated CUDA memory (inputs, outputs and workspace are all torch allocations).
+
+Two methods:
+  fused  the library (kdkl_forward + kdkl_backward)
+  dense  a plain torch comparator that materialises the [T, V] logits, a dense log-softmax and the
+         scattered dense teacher (section "Full Dense KL Computation"). It exists only to show what the
+         fused path saves; it is expected to run out of memory at long T, which is recorded as such.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _cfg(name: str):
+    from paper_2608_03796_b200 import inputs as I
+    if name in I.CONFIGS:
+        return I.CONFIGS[name]
+    if name.startswith("T"):                       # the 4K shape at another length, e.g. T8192
+        return dataclasses.replace(I.CONFIGS["c2"], name=name, T=int(name[1:]))
+    raise KeyError(name)
+
+
+def worker(method: str, name: str, steps: int) -> dict:
+    import torch
+    from paper_2608_03796_b200 import binding as B
+    from paper_2608_03796_b200 import inputs as I
+
+    cfg = _cfg(name)
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    d = I.make_inputs(cfg, device=dev)
+    torch.cuda.synchronize()
+    torch.cuda.reset_peak_memory_stats()
+    out = {"method": method, "workload": name, "T": cfg.T, "H": cfg.H, "V": cfg.V, "K": cfg.K, "chunk": cfg.chunk,
+           "input_gb": torch.cuda.memory_allocated() / 1e9}
+    if method == "fused":
+        op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev)
+
+        def step():
+            op.forward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], loss_mask=d["mask"])
+            op.backward(d["hidden"], d["weight"], loss_mask=d["mask"])
+            return op.loss
+        out["workspace_gb"] = op.workspace.numel() / 1e9
+    else:
+        h = d["hidden"].clone().requires_grad_(True)
+        W = d["weight"].clone().requires_grad_(True)
+        counted = torch.ones(cfg.T, dtype=torch.bool, device=dev) if d["mask"] is None else d["mask"] != 0
+        idx = d["topk_idx"].long().clamp_(min=0)
+        val = torch.nan_to_num(d["topk_val"])
+
+        def step():
+            h.grad = None
+            W.grad = None
+            z = (h @ W.T).float() / cfg.tau
+            logq = torch.log_softmax(z, dim=-1)
+            pk = torch.softmax(val / cfg.tau, dim=-1) * counted[:, None]
+            p = torch.zeros_like(logq).scatter_add_(1, idx, pk)
+            per_tok = torch.nn.functional.kl_div(logq, p, reduction="none").sum(-1)
+            loss = per_tok.sum() / counted.sum()
+            loss.backward()
+            return loss.detach()
+    try:
+        for _ in range(2):
+            loss = step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            loss = step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        out.update(ms_per_iter=ms, it_per_s=1e3 / ms, tokens_per_s=cfg.T / (ms * 1e-3),
+                   tflops=cfg.flops / (ms * 1e-3) / 1e12, loss=float(loss.item()),
+                   peak_gb=torch.cuda.max_memory_allocated() / 1e9)
+        if method == "fused":
+            code, _ = op.status()
+            out["status"] = code
+    except torch.OutOfMemoryError:
+        out.update(oom=True, peak_gb=torch.cuda.max_memory_allocated() / 1e9)
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--worker", default=None)
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--steps", type=int, default=0)
+    ap.add_argument("--fused", default="c2,T8192,T16384,c3,c4a,c4b,c4c,c5")
+    ap.add_argument("--dense", default="c2,T8192,T16384,c3")
+    ap.add_argument("--out", default="")
+    args = ap.parse_args()
+    if ROOT not in sys.path:
+        sys.path.insert(0, ROOT)
+    if args.worker:
+        cfg = _cfg(args.workload)
+        steps = args.steps or (10 if cfg.T <= 32768 else 3)
+        print("SWEEP " + json.dumps(worker(args.worker, args.workload, steps)), flush=True)
+        return
+
+    rows = []
+    for method, names in (("fused", args.fused), ("dense", args.dense)):
+        for name in [n for n in names.split(",") if n]:
+            t0 = time.time()
+            r = subprocess.run([sys.executable, "-m", "paper_2608_03796_b200.sweep", "--worker", method,
+                                "--workload", name], cwd=ROOT, capture_output=True, text=True)
+            rec = None
+            for line in r.stdout.splitlines():
+                if line.startswith("SWEEP "):
+                    rec = json.loads(line[6:])
+            if rec is None:
+                rec = {"method": method, "workload": name, "failed": (r.stderr or r.stdout)[-300:]}
+            rec["wall_s"] = round(time.time() - t0, 1)
+            rows.append(rec)
+            print(json.dumps(rec), flush=True)
+
+    if args.out:
+        peaks = {}
+        pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        if os.path.exists(pk):
+            peaks = json.load(open(pk))
+        burst = float(peaks.get("bf16_tflops", 1590.0))
+        sust = float(peaks.get("bf16_tflops_sustained", 1400.0))
+        lines = ["# Sequence-length sweep: iteration rate and peak memory (one B200, fresh process per setting)", "",
+                 "Command: `python -m paper_2608_03796_b200.sweep --out " + args.out + "`", "",
+                 f"Peaks used: bf16 burst {burst} / sustained {sust} TFLOP/s "
+                 f"({'measured' if peaks else 'fallback'}). FLOPs counted as 8*T*H*V per iteration.", "",
+                 "| method | workload | T | ms/iter | it/s | tokens/s | TFLOP/s | % burst | % sustained | peak GB | workspace GB |",
+                 "|---|---|---|---|---|---|---|---|---|---|---|"]
+        for r in rows:
+            if "ms_per_iter" in r:
+                lines.append(f"| {r['method']} | {r['workload']} | {r['T']} | {r['ms_per_iter']:.2f} | {r['it_per_s']:.3f} | "
+                             f"{r['tokens_per_s']:.0f} | {r['tflops']:.0f} | {100 * r['tflops'] / burst:.1f} | "
+                             f"{100 * r['tflops'] / sust:.1f} | {r['peak_gb']:.2f} | {r.get('workspace_gb', 0):.2f} |")
+            elif r.get("oom"):
+                lines.append(f"| {r['method']} | {r['workload']} | {r['T']} | out of memory | | | | | | > {r['peak_gb']:.1f} | |")
+            else:
+                lines.append(f"| {r['method']} | {r['workload']} | | failed: {r.get('failed', '')[:80]} | | | | | | | |")
+        # least-squares line through the fused peaks of the H=4096 / V=131072 family
+        pts = [(r["T"], r["peak_gb"]) for r in rows if r["method"] == "fused" and "ms_per_iter" in r
+               and r["H"] == 4096 and r["V"] == 131072 and r["T"] >= 32768]
+        if len(pts) >= 3:
+            n = len(pts)
+            sx = sum(p[0] for p in pts); sy = sum(p[1] for p in pts)
+            sxx = sum(p[0] * p[0] for p in pts); sxy = sum(p[0] * p[1] for p in pts)
+            b = (n * sxy - sx * sy) / (n * sxx - sx * sx)
+            a = (sy - b * sx) / n
+            res = max(abs(a + b * t - y) / y for t, y in pts)
+            lines += ["", f"Fused peak memory, T >= 32768: peak = {a:.3f} GB + {b * 1e6:.2f} KB/token x T "
+                          f"(largest relative residual {100 * res:.2f} %): linear in T."]
+        dense = [(r["T"], r["peak_gb"]) for r in rows if r["method"] == "dense" and "ms_per_iter" in r]
+        if len(dense) >= 2:
+            (t0_, y0), (t1_, y1) = dense[0], dense[-1]
+            slope = (y1 - y0) / (t1_ - t0_)
+            lines += ["", f"Dense comparator: {slope * 1e6:.0f} KB/token between T={t0_} and T={t1_} "
+                          f"(about {slope * 1e9 / rows[0]['V']:.1f} bytes per logit); extrapolated to T=32768: "
+                          f"{y0 + slope * (32768 - t0_):.0f} GB."]
+        with open(os.path.join(ROOT, args.out), "w") as f:
+            f.write("\n".join(lines) + "\n")
+
+
+if __name__ == "__main__":
+    main()
