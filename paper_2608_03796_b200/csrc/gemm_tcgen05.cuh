@@ -63,6 +63,7 @@ struct GemmParams {
   float* zg;                 // [rows, Ktop] gathered logits, sorted order
   int* colread;              // [rows, Ktop] column actually read, sorted order
   const float* lz2;          // [rows] log2-domain log-normaliser
+  int neg_a;                 // 1 when the upstream gradient is negative (coefA <= 0 for every row)
   const float* coefA;        // [rows] g_t * M_t / tau
   const float* coefB;        // [rows] g_t / tau
   const float* p_sorted;     // [rows, Ktop]
@@ -251,14 +252,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       // per-row state that does not need the accumulator: fetched before the wait
       int cur = 0, nv = 0, next_idx = 0x7fffffff;
       const int* idxrow = nullptr;
-      float row_a = 0.f, row_b = 0.f, row_lz2 = 0.f;
+      float row_b = 0.f, row_off = -INFINITY;
       if (EPI == EPI_LSE || EPI == EPI_DLOGITS) {
         if (row_ok) {
           idxrow = p.idx_sorted + (long long)row * p.Ktop;
           nv = p.nvalid[row];
           cur = lower_bound_i32(idxrow, nv, n0);
           next_idx = cur < nv ? idxrow[cur] : 0x7fffffff;
-          if (EPI == EPI_DLOGITS) { row_a = p.coefA[row]; row_b = p.coefB[row]; row_lz2 = p.lz2[row]; }
+          if (EPI == EPI_DLOGITS) {
+            const float a = p.coefA[row];
+            row_b = p.coefB[row];
+            row_off = a != 0.f ? log2f(fabsf(a)) - p.lz2[row] : -INFINITY;   // sign: see neg_a
+          }
         }
       }
 
@@ -293,18 +298,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               ++cur;
               next_idx = cur < nv ? idxrow[cur] : 0x7fffffff;
             }
-            // online max / sum-exp in the log2 domain
-            float t[32];
+            // online max / sum-exp in the log2 domain: max on the raw logits (the scale is positive),
+            // then one FFMA + ex2 + add per element
             float wmax = -INFINITY;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              t[j] = (full_w || col0 + j < p.N) ? __uint_as_float(r[j]) * p.scale_log2 : -INFINITY;
-              wmax = fmaxf(wmax, t[j]);
+              if (!full_w && col0 + j >= p.N) r[j] = 0xff800000u;   // -inf: columns past the vocabulary
+              wmax = fmaxf(wmax, __uint_as_float(r[j]));
             }
-            const float m_new = fmaxf(m_run, wmax);
+            const float m_new = fmaxf(m_run, wmax * p.scale_log2);
             float acc_s = 0.f;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) acc_s += ex2_approx(t[j] - m_new);
+            for (int j = 0; j < 32; ++j) acc_s += ex2_approx(fmaf(__uint_as_float(r[j]), p.scale_log2, -m_new));
             s_run = s_run * ex2_approx(m_run - m_new) + acc_s;
             m_run = m_new;
           }
@@ -329,12 +334,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
               for (int j = 0; j < 16; ++j) v[j] = pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
             } else {  // EPI_DLOGITS
+              // a_t * 2^(s - lz2) = 2^(s + (log2 a_t - lz2)): the row coefficient rides in the exponent
+              // (a_t = 0 for ignored tokens gives -inf, hence exact zeros)
               float g[32];
-              const bool live = (row_a != 0.f) || (row_b != 0.f);
 #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const float q = ex2_approx(fmaf(__uint_as_float(r[j]), p.scale_log2, -row_lz2));
-                g[j] = live ? row_a * q : 0.f;
+              for (int j = 0; j < 32; ++j) g[j] = ex2_approx(fmaf(__uint_as_float(r[j]), p.scale_log2, row_off));
+              if (p.neg_a) {                   // uniform: the whole call has a negative upstream gradient
+#pragma unroll
+                for (int j = 0; j < 32; ++j) g[j] = -g[j];
               }
               while (next_idx < col0 + 32) {
                 const int off = next_idx - col0;

@@ -353,6 +353,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p.lz2 = at<float>(ws, L.lz2) + s0;
     p.coefA = at<float>(ws, L.coefA) + s0;
     p.coefB = at<float>(ws, L.coefB) + s0;
+    p.neg_a = grad_loss < 0.f ? 1 : 0;
     CUtensorMap tmGout;
     if ((rc = make_tmap_out_bf16(&tmGout, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad))) return rc;
     stage_mark(ST_B1, st);

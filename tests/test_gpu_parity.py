@@ -167,6 +167,13 @@ def test_k1_and_large_k():
     _compare(_run(d, 33, 64, 2048, 600, 0, 0.9), _oracle(d, 0.9), d)
 
 
+def test_negative_upstream_gradient():
+    T, H, V, K = 130, 64, 1500, 6
+    d = _small_case(T, H, V, K, seed=21, mask_frac=0.1)
+    op = _run(d, T, H, V, K, 64, 1.2, grad_loss=-2.0)
+    _compare(op, _oracle(d, 1.2, grad_loss=-2.0), d)
+
+
 def test_all_tokens_ignored_gives_zero():
     d = _small_case(50, 64, 512, 4, seed=15)
     d["mask"] = torch.zeros(50, dtype=torch.uint8)
