@@ -278,8 +278,8 @@ def main():
     gemm_stages = ["fwd_gemm_lse", "bwd_gemm_dlogits", "dhidden_gemm", "dweight_gemm"]
     dom = max(gemm_stages, key=lambda k: stages[k]["ms_per_step"])
     # DRAM bytes per launch from one ncu capture at chunk=4096, H=4096, V=131072 (read + write); null elsewhere
-    measured_traffic = {"fwd_gemm_lse": 1118951168 + 28143616, "bwd_gemm_dlogits": 1223847424 + 1051266048,
-                        "dhidden_gemm": 5471380992 + 29573376, "dweight_gemm": 1442837760 + 2109563136}
+    measured_traffic = {"fwd_gemm_lse": 1118791680 + 25831168, "bwd_gemm_dlogits": 1249679104 + 1053059584,
+                        "dhidden_gemm": 5458027520 + 117394432, "dweight_gemm": 1551928576 + 2114988800}
     C = min(cfg.chunk, T)
     traffic = measured_traffic[dom] if (C, H, V) == (4096, 4096, 131072) else None
     flops_per_launch = 2.0 * C * H * V             # each of the four GEMMs: 2 * chunk * H * V per launch

@@ -7,7 +7,7 @@
 //               a time); two TMEM accumulator stages let tile i's epilogue overlap tile
 //               i+1's MMAs
 //
-// One CTA per SM (grid = min(tiles, SM count)), tiles of 128 x 256, k-blocks of 64.
+// One CTA per SM; tiles of 128 x 256 per CTA (256 x 256 per CTA pair, see GemmCfg), k-blocks of 64.
 // Either operand may be K-major (its rows are contiguous along K) or MN-major (stored
 // [K, M] / [K, N], contiguous along M / N); the difference is confined to the TMA boxes
 // and the shared-memory descriptors.
@@ -28,16 +28,28 @@
 
 namespace kdkl {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int BM = 128, BN = 256, BK = 64;   // per-CTA accumulator: 128 TMEM lanes x 256 fp32 columns
 constexpr int UMMA_K = 16;
-constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KiB
-constexpr int B_STAGE_BYTES = BN * BK * 2;   // 32 KiB
-constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int GEMM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
 constexpr int STAGING_WARP_BYTES = 2 * 4096;   // per epilogue warp: two 32-row x 128-byte output boxes
 constexpr int STAGING_BYTES = 4 * STAGING_WARP_BYTES;
-constexpr int GEMM_SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+// NCTA = 1: one CTA per 128 x 256 tile. NCTA = 2: a pair of CTAs (cluster of two, cta_group::2)
+// shares one 256 x 256 tile: each CTA stages its 128 rows of A and its 128 rows of B, the leader
+// issues one MMA for both, and each CTA keeps the 128 x 256 half of D in its own TMEM. A pair
+// moves a third less operand data per flop through shared memory and L2, and the smaller stage
+// buys a deeper ring.
+template <int NCTA>
+struct GemmCfg {
+  static constexpr int TILE_M = BM * NCTA;
+  static constexpr int B_ROWS = BN / NCTA;               // rows of B each CTA stages
+  static constexpr int A_STAGE_BYTES = BM * BK * 2;      // 16 KiB
+  static constexpr int B_STAGE_BYTES = B_ROWS * BK * 2;  // 32 / 16 KiB
+  static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+  static constexpr int STAGES = NCTA == 2 ? 6 : 4;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
 
 enum { EPI_STORE_F32 = 0, EPI_STORE_BF16 = 1, EPI_LSE = 2, EPI_DLOGITS = 3 };
 
@@ -97,10 +109,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int EPI, bool A_MN, bool B_MN>
+template <int EPI, bool A_MN, bool B_MN, int NCTA>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
+  using Cfg = GemmCfg<NCTA>;
+  constexpr int STAGES = Cfg::STAGES, STAGE_BYTES = Cfg::STAGE_BYTES, A_STAGE_BYTES = Cfg::A_STAGE_BYTES;
+  constexpr int TILE_M = Cfg::TILE_M, B_ROWS = Cfg::B_ROWS;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -120,9 +135,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   if (p.go != nullptr && *p.go == 0) return;   // uniform across the grid
 
+  // pair bookkeeping: the leader (cluster rank 0) owns the barriers that gate the MMAs
+  const uint32_t cta_rank = NCTA == 2 ? cluster_ctarank() : 0u;
+  const bool leader = cta_rank == 0u;
+  const int worker = blockIdx.x / NCTA, num_workers = gridDim.x / NCTA;
+  auto leader_bar = [&](uint32_t bar) { return NCTA == 2 ? map_to_cta(bar, 0u) : bar; };
+
   if (threadIdx.x == 0) {
+    // full (used in the leader): one arrival, the leader's producer announcing the bytes of both CTAs'
+    // loads; tempty (leader): one arrival per epilogue warp of the pair
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4 * NCTA); }
     *abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmA);
@@ -130,11 +153,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (EPI != EPI_LSE) tma_prefetch_desc(&tmC);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
-    tmem_relinquish();
+    if (NCTA == 2) { tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS); tmem_relinquish_pair(); }
+    else           { tmem_alloc(smem_u32(tmem_slot), TMEM_COLS); tmem_relinquish(); }
   }
   tc_fence_before();
   __syncthreads();
+  if (NCTA == 2) cluster_sync_all();   // the peer's barriers exist before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -160,30 +184,39 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (lane == 0) {
       uint32_t it = 0, issued = 0, last_par = 0;
       bool ok = true;
-      for (int unit = blockIdx.x; unit < num_units && ok; unit += gridDim.x) {
+      // a load lands in this CTA's stage and signals the full barrier of the pair's leader
+      auto load = [&](uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+        if (NCTA == 2) tma_load_2d_pair(dst, tm, x, y, bar); else tma_load_2d(dst, tm, x, y, bar);
+      };
+      for (int unit = worker; unit < num_units && ok; unit += num_workers) {
         int tile, split, kb0, kb1, mt, nt;
         unit_decode(unit, tile, split, kb0, kb1);
         tile_coords(tile, mt, nt);
-        const int m0 = mt * BM, n0 = nt * BN;
+        const int m0 = mt * TILE_M + (int)cta_rank * BM;      // this CTA's rows of A
+        const int n0 = nt * BN + (int)cta_rank * B_ROWS;      // this CTA's rows of B
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
           const uint32_t sa = smem_base + s * STAGE_BYTES;
           const uint32_t sb = sa + A_STAGE_BYTES;
-          mbar_arrive_expect_tx(full_bar(s), STAGE_BYTES);
+          const uint32_t fb = leader_bar(full_bar(s));
+          // The peer's bytes may land before this announcement: the phase still cannot complete
+          // before the leader's single arrival, and the peer reuses a stage only after the MMAs
+          // that consumed it have been committed.
+          if (leader) mbar_arrive_expect_tx(full_bar(s), NCTA * STAGE_BYTES);
           const int k0 = kb * BK;
           if (!A_MN) {
-            tma_load_2d(sa, &tmA, k0, m0, full_bar(s));
+            load(sa, &tmA, k0, m0, fb);
           } else {
 #pragma unroll
-            for (int i = 0; i < BM / 64; ++i) tma_load_2d(sa + i * (BK * 128), &tmA, m0 + 64 * i, k0, full_bar(s));
+            for (int i = 0; i < BM / 64; ++i) load(sa + i * (BK * 128), &tmA, m0 + 64 * i, k0, fb);
           }
           if (!B_MN) {
-            tma_load_2d(sb, &tmB, k0, n0, full_bar(s));
+            load(sb, &tmB, k0, n0, fb);
           } else {
 #pragma unroll
-            for (int i = 0; i < BN / 64; ++i) tma_load_2d(sb + i * (BK * 128), &tmB, n0 + 64 * i, k0, full_bar(s));
+            for (int i = 0; i < B_ROWS / 64; ++i) load(sb + i * (BK * 128), &tmB, n0 + 64 * i, k0, fb);
           }
           issued |= 1u << s;
           last_par = (last_par & ~(1u << s)) | (ph << s);
@@ -191,20 +224,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
       if (!ok) {
         // aborted: give the copies still in flight a bounded time to land before the CTA exits
-        for (int s = 0; s < STAGES; ++s) {
-          if (!((issued >> s) & 1u)) continue;
-          const uint64_t t0 = globaltimer_ns();
-          while (!mbar_try_wait(full_bar(s), (last_par >> s) & 1u) && globaltimer_ns() - t0 < 2000000ull) {}
+        if (NCTA == 1) {
+          for (int s = 0; s < STAGES; ++s) {
+            if (!((issued >> s) & 1u)) continue;
+            const uint64_t t0 = globaltimer_ns();
+            while (!mbar_try_wait(full_bar(s), (last_par >> s) & 1u) && globaltimer_ns() - t0 < 2000000ull) {}
+          }
+        } else {
+          const uint64_t t0 = globaltimer_ns();   // the barrier may be the peer's: a bounded pause instead
+          while (globaltimer_ns() - t0 < 2000000ull) {}
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc_bf16(BM, BN, A_MN ? 1u : 0u, B_MN ? 1u : 0u);
+    // ------------------------------------------------------------ MMA issuer (the leader's, for the pair)
+    if (lane == 0 && leader) {
+      const uint32_t idesc = make_idesc_bf16(TILE_M, BN, A_MN ? 1u : 0u, B_MN ? 1u : 0u);
+      auto mma = [&](uint32_t d, uint64_t ad, uint64_t bd, uint32_t accf) {
+        if (NCTA == 2) umma_bf16_pair(d, ad, bd, idesc, accf); else umma_bf16(d, ad, bd, idesc, accf);
+      };
+      auto commit = [&](uint32_t bar) { if (NCTA == 2) umma_commit_pair(bar); else umma_commit(bar); };
       uint32_t it = 0, lt = 0;
       bool ok = true;
-      for (int unit = blockIdx.x; unit < num_units && ok; unit += gridDim.x, ++lt) {
+      for (int unit = worker; unit < num_units && ok; unit += num_workers, ++lt) {
         int tile, split, kb0, kb1;
         unit_decode(unit, tile, split, kb0, kb1);
         const uint32_t acc = lt & 1u;
@@ -225,11 +267,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                                      : make_smem_desc(sa + j * (UMMA_K * 2), 0, 1024);
             const uint64_t bd = B_MN ? make_smem_desc(sb + j * (UMMA_K * 128), BK * 128, 1024)
                                      : make_smem_desc(sb + j * (UMMA_K * 2), 0, 1024);
-            umma_bf16(tmem_d, ad, bd, idesc, (kb > kb0 || j > 0) ? 1u : 0u);
+            mma(tmem_d, ad, bd, (kb > kb0 || j > 0) ? 1u : 0u);
           }
-          umma_commit(empty_bar(s));           // frees the stage when these MMAs have read it
+          commit(empty_bar(s));                // frees the stage (in both CTAs) when these MMAs have read it
         }
-        if (ok) umma_commit(tfull_bar(acc));   // accumulator complete
+        if (ok) commit(tfull_bar(acc));        // accumulator complete (signalled in both CTAs)
       }
     }
   } else {
@@ -239,11 +281,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     constexpr bool kBf16Out = (EPI == EPI_STORE_BF16 || EPI == EPI_DLOGITS);
     uint32_t lt = 0, nbox = 0;
     bool ok = true;
-    for (int unit = blockIdx.x; unit < num_units && ok; unit += gridDim.x, ++lt) {
+    for (int unit = worker; unit < num_units && ok; unit += num_workers, ++lt) {
       int tile, split, kb0, kb1, mt, nt;
       unit_decode(unit, tile, split, kb0, kb1);
       tile_coords(tile, mt, nt);
-      const int m0 = mt * BM, n0 = nt * BN;
+      const int m0 = mt * TILE_M + (int)cta_rank * BM, n0 = nt * BN;   // this CTA's 128 x 256 part of D
       const int row = m0 + row_in_tile;
       const bool row_ok = row < p.M;
       const uint32_t acc = lt & 1u;
@@ -376,7 +418,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       // accumulator stage is free again
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (lane == 0) {
+        if (NCTA == 2) mbar_arrive_cluster(leader_bar(tempty_bar(acc))); else mbar_arrive(tempty_bar(acc));
+      }
 
       if (EPI == EPI_LSE) {
         if (row_ok) {
@@ -392,8 +436,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   __syncwarp();
   tc_fence_before();
   __syncthreads();
+  if (NCTA == 2) cluster_sync_all();   // neither CTA leaves while the other may still reach its barriers
   tc_fence_after();
-  if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+  if (warp == 1) {
+    if (NCTA == 2) tmem_dealloc_pair(tmem_base, TMEM_COLS); else tmem_dealloc(tmem_base, TMEM_COLS);
+  }
 }
 
 }  // namespace kdkl

@@ -108,6 +108,13 @@ static int make_tmap_out_bf16(CUtensorMap* m, void* base, uint64_t cols, uint64_
 }
 
 // ------------------------------------------------------------------ device / launch helpers
+// All GEMMs of the loss run as CTA pairs (256 x 256 tile per pair, see GemmCfg).
+#ifndef KDKL_NCTA
+#define KDKL_NCTA 2
+#endif
+constexpr int kNCTA = KDKL_NCTA;
+constexpr int kTileM = GemmCfg<kNCTA>::TILE_M;
+constexpr int kBRows = GemmCfg<kNCTA>::B_ROWS;
 struct DeviceInfo { int sm_count; int cc_major; bool ok; };
 static int device_info(DeviceInfo* di) {
   int dev = 0;
@@ -120,15 +127,33 @@ static int device_info(DeviceInfo* di) {
 template <int EPI, bool A_MN, bool B_MN>
 static int launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const GemmParams& p,
                        int sm_count, cudaStream_t st) {
-  auto kern = gemm_tcgen05_kernel<EPI, A_MN, B_MN>;
+  auto kern = gemm_tcgen05_kernel<EPI, A_MN, B_MN, kNCTA>;
+  constexpr int smem = GemmCfg<kNCTA>::SMEM_BYTES;
   static bool attr_set = false;   // per instantiation
   if (!attr_set) {
-    KDKL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES));
+    KDKL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_set = true;
   }
+  // persistent: one worker (a CTA, or a pair of CTAs on neighbouring SMs) per SM (pair), each walking
+  // the work units with a stride of the worker count
   const int units = p.m_tiles * p.n_tiles * p.k_splits;
-  const int grid = units < sm_count ? units : sm_count;
-  kern<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ta, tb, tc, p);
+  const int max_workers = sm_count / kNCTA;
+  const int workers = units < max_workers ? units : max_workers;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)(workers * kNCTA), 1, 1);
+  cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kNCTA;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ta, tb, tc, p);
+  if (e != cudaSuccess) return cuda_fail("gemm_tcgen05_kernel launch", e);
   KDKL_LAUNCHED("gemm_tcgen05_kernel");
   return KDKL_OK;
 }
@@ -140,7 +165,7 @@ static inline size_t up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // waves of SMs: the smallest count (<= 4, each unit keeping >= 32 k-blocks) that reaches 95 %
 // wave efficiency, else the most efficient one. Sized for the 148 SMs of a B200.
 static int choose_k_splits(long long tiles, long long kblocks) {
-  const long long sms = 148;
+  const long long sms = 148 / kNCTA;
   int best = 1;
   double best_eff = 0.0;
   for (int sp = 1; sp <= 4; ++sp) {
@@ -186,7 +211,7 @@ static WsLayout ws_layout(long long T, long long H, long long V, int K, long lon
   L.part_m = take((size_t)L.n_tiles_v * L.Cpad * 4);
   L.part_s = take((size_t)L.n_tiles_v * L.Cpad * 4);
   L.G = take((size_t)L.Cpad * L.Vpad * 2);
-  L.dh_splits = choose_k_splits(((L.C + BM - 1) / BM) * ((H + BN - 1) / BN), (V + BK - 1) / BK);
+  L.dh_splits = choose_k_splits(((L.C + kTileM - 1) / kTileM) * ((H + BN - 1) / BN), (V + BK - 1) / BK);
   L.dh_part = take(L.dh_splits > 1 ? (size_t)L.dh_splits * L.Cpad * H * 4 : 0);
   L.total = o;
   return L;
@@ -265,7 +290,7 @@ int kdkl_forward(const void* hidden, const void* weight, const int32_t* topk_idx
   KDKL_LAUNCHED("prep_kernel");
 
   CUtensorMap tmW;
-  if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, BN))) return rc;
+  if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, kBRows))) return rc;
 
   for (long long s0 = 0; s0 < T; s0 += L.C) {
     const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
@@ -275,7 +300,7 @@ int kdkl_forward(const void* hidden, const void* weight, const int32_t* topk_idx
     GemmParams p;
     memset(&p, 0, sizeof(p));
     p.M = (int)rows; p.N = (int)V; p.K = (int)H;
-    p.m_tiles = (int)((rows + BM - 1) / BM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1; p.k_splits = 1;
+    p.m_tiles = (int)((rows + kTileM - 1) / kTileM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1; p.k_splits = 1;
     p.status = &hdr->status; p.go = nullptr;
     p.scale_log2 = kLog2e * inv_tau; p.Ktop = K;
     p.idx_sorted = at<int>(ws, L.idx_sorted) + s0 * K;
@@ -327,7 +352,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
   __nv_bfloat16* G = at<__nv_bfloat16>(ws, L.G);
   // W as the K-major B operand of the recompute GEMM, and as the MN-major B operand of dH = G W
   CUtensorMap tmW, tmWmn;
-  if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, BN))) return rc;
+  if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, kBRows))) return rc;
   if ((rc = make_tmap_bf16(&tmWmn, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, 64, BK))) return rc;
 
   CUtensorMap tmdW;
@@ -344,7 +369,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     GemmParams p;
     memset(&p, 0, sizeof(p));
     p.M = (int)rows; p.N = (int)V; p.K = (int)H;
-    p.m_tiles = (int)((rows + BM - 1) / BM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1; p.k_splits = 1;
+    p.m_tiles = (int)((rows + kTileM - 1) / kTileM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1; p.k_splits = 1;
     p.status = &hdr->status; p.go = go;
     p.scale_log2 = kLog2e * inv_tau; p.Ktop = K;
     p.idx_sorted = at<int>(ws, L.idx_sorted) + s0 * K;
@@ -365,7 +390,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     GemmParams p2;
     memset(&p2, 0, sizeof(p2));
     p2.M = (int)rows; p2.N = (int)H; p2.K = (int)V;
-    p2.m_tiles = (int)((rows + BM - 1) / BM); p2.n_tiles = (int)((H + BN - 1) / BN); p2.m_inner = 0;
+    p2.m_tiles = (int)((rows + kTileM - 1) / kTileM); p2.n_tiles = (int)((H + BN - 1) / BN); p2.m_inner = 0;
     p2.status = &hdr->status; p2.go = go;
     p2.accumulate = 0;
     // a short last chunk may want a different split; never more than the workspace was sized for
@@ -401,7 +426,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     GemmParams p3;
     memset(&p3, 0, sizeof(p3));
     p3.M = (int)V; p3.N = (int)H; p3.K = (int)rows;
-    p3.m_tiles = (int)((V + BM - 1) / BM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0; p3.k_splits = 1;
+    p3.m_tiles = (int)((V + kTileM - 1) / kTileM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0; p3.k_splits = 1;
     p3.status = &hdr->status; p3.go = go;
     p3.accumulate = (ci > 0 || o.accumulate_dweight) ? 1 : 0;
     stage_mark(ST_B3, st);
@@ -547,12 +572,12 @@ int kdkl_gemm_bf16(const void* A, const void* B, float* C, int64_t M, int64_t N,
   else      rc = make_tmap_bf16(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)K * 2, BK, BM);
   if (rc) return rc;
   if (b_mn) rc = make_tmap_bf16(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)N * 2, 64, BK);
-  else      rc = make_tmap_bf16(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)K * 2, BK, BN);
+  else      rc = make_tmap_bf16(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)K * 2, BK, kBRows);
   if (rc) return rc;
   GemmParams p;
   memset(&p, 0, sizeof(p));
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
-  p.m_tiles = (int)((M + BM - 1) / BM); p.n_tiles = (int)((N + BN - 1) / BN); p.k_splits = 1;
+  p.m_tiles = (int)((M + kTileM - 1) / kTileM); p.n_tiles = (int)((N + BN - 1) / BN); p.k_splits = 1;
   p.m_inner = p.m_tiles <= p.n_tiles ? 1 : 0;   // walk the shorter dimension first: the other operand streams once
   p.status = status; p.accumulate = 0;
   CUtensorMap tc;

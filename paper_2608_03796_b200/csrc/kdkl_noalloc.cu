@@ -117,8 +117,8 @@ int setup_device(int dev, PerDevice** out) {
     void* ptr = nullptr;
     if (e == cudaSuccess) e = cudaGetSymbolAddress(&ptr, g_scratch);
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(gemm_tcgen05_kernel<EPI_LSE, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               GEMM_SMEM_BYTES);
+      e = cudaFuncSetAttribute(gemm_tcgen05_kernel<EPI_LSE, false, false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               GemmCfg<1>::SMEM_BYTES);
     if (e != cudaSuccess) {
       snprintf(g_text, sizeof(g_text), "set-up on device %d failed: %s", dev, cudaGetErrorString(e));
       return KDKL_ERR_CUDA;
@@ -175,7 +175,7 @@ extern "C" int kdkl_logz_noalloc(const void* hidden_bf16, const void* weight_bf1
     p.part_stride = kPassRows;
     const int tiles = p.m_tiles * p.n_tiles;
     const int grid = tiles < pd->sm_count ? tiles : pd->sm_count;
-    gemm_tcgen05_kernel<EPI_LSE, false, false><<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(tmA, tmW, tmA /*no output map*/, p);
+    gemm_tcgen05_kernel<EPI_LSE, false, false, 1><<<grid, GEMM_THREADS, GemmCfg<1>::SMEM_BYTES, st>>>(tmA, tmW, tmA /*no output map*/, p);
     logz_combine_kernel<<<(rows + 31) / 32, 256, 0, st>>>(p.part_m, p.part_s, n_tiles, rows, p.status, logz_out + s0);
     if (cudaGetLastError() != cudaSuccess) return KDKL_ERR_CUDA;
   }
