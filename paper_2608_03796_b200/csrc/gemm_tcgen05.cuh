@@ -38,8 +38,7 @@ constexpr int STAGING_BYTES = 4 * STAGING_WARP_BYTES;
 // NCTA = 1: one CTA per 128 x 256 tile. NCTA = 2: a pair of CTAs (cluster of two, cta_group::2)
 // shares one 256 x 256 tile: each CTA stages its 128 rows of A and its 128 rows of B, the leader
 // issues one MMA for both, and each CTA keeps the 128 x 256 half of D in its own TMEM. A pair
-// moves a third less operand data per flop through shared memory and L2, and the smaller stage
-// buys a deeper ring.
+// moves a third less operand data per flop through shared memory and L2.
 template <int NCTA>
 struct GemmCfg {
   static constexpr int TILE_M = BM * NCTA;
@@ -47,7 +46,7 @@ struct GemmCfg {
   static constexpr int A_STAGE_BYTES = BM * BK * 2;      // 16 KiB
   static constexpr int B_STAGE_BYTES = B_ROWS * BK * 2;  // 32 / 16 KiB
   static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-  static constexpr int STAGES = NCTA == 2 ? 6 : 4;
+  static constexpr int STAGES = 4;   // measured: 3 starves the tensor pipe, 5 and 6 are no faster than 4
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
