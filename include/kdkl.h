@@ -100,6 +100,33 @@ int kdkl_backward(const void* hidden_bf16, const void* weight_bf16, const uint8_
                   const kdkl_options* opt, float grad_loss, void* workspace, size_t workspace_bytes,
                   void* dhidden, float* dweight, void* cuda_stream);
 
+/* Vocabulary-sharded use (the paper's tensor-parallel variant: section "Full Chunked KL Computation", last
+ * sentences, and Algorithm 1's "distributed max", "reduce sigma", "reduce dh across shards").
+ * Rank r holds the weight rows [vocab_offset, vocab_offset + V_local) of a vocabulary of V_total entries;
+ * hidden states, the teacher record (GLOBAL indices) and the mask are replicated. Per step and rank:
+ *   1. kdkl_forward_shard: the local sweep. Writes shard_stats [2, T] fp32 (device): row 0 the local
+ *      log2-domain normaliser log2 sum_{v local} 2^(z_v log2e / tau), row 1 the local cross term
+ *      sum_{k local} p_k z_k / tau. M and the teacher entropy use all usable entries on every rank.
+ *      gathered_logits / gathered_idx (optional) are filled for the local entries only (global index).
+ *   2. the caller gathers the shard_stats of all ranks into all_stats [n_shards, 2, T] (for instance an
+ *      NCCL all-gather); this library performs no communication.
+ *   3. kdkl_forward_finish: log Z = logsumexp over shards, C = sum over shards, loss as in kdkl_forward;
+ *      identical on every rank. Stores the global log Z in the workspace for backward.
+ *   4. kdkl_backward with weight_local, V = V_local and the same workspace: dweight is the local slice
+ *      [V_local, H] (complete, no communication); dhidden is this shard's partial sum over its vocabulary
+ *      rows, to be summed over ranks by the caller (use dhidden_dtype = 1 for an fp32 reduction).
+ * V_total < 2^30. Other arguments and errors as kdkl_forward. */
+int kdkl_forward_shard(const void* hidden_bf16, const void* weight_local_bf16, const int32_t* topk_idx,
+                       const float* topk_val, const float* teacher_lse, const uint8_t* loss_mask,
+                       int64_t T, int64_t H, int64_t V_local, int64_t vocab_offset, int64_t V_total, int32_t K,
+                       int64_t chunk, float temperature, const kdkl_options* opt, void* workspace,
+                       size_t workspace_bytes, float* shard_stats, float* gathered_logits,
+                       int32_t* gathered_idx, void* cuda_stream);
+int kdkl_forward_finish(const float* all_stats, int32_t n_shards, const uint8_t* loss_mask, int64_t T, int64_t H,
+                        int64_t V_local, int32_t K, int64_t chunk, float temperature, const kdkl_options* opt,
+                        void* workspace, size_t workspace_bytes, float* loss_out, float* loss_per_token,
+                        void* cuda_stream);
+
 /* Synchronises the stream and reads the device status of the last forward/backward on this
  * workspace: *code = KDKL_OK or a device-detected KDKL_ERR_*; detail[0] = site/row of the error,
  * detail[1] = number of counted tokens, detail[2] = number of ignored (>= V) teacher indices.

@@ -25,7 +25,7 @@ ERRORS = {
 EXPORTS = [
     "kdkl_workspace_bytes", "kdkl_forward", "kdkl_backward", "kdkl_status", "kdkl_saved_state",
     "kdkl_host_arena_bytes", "kdkl_forward_backward_host", "kdkl_profile_stages", "kdkl_gemm_bf16", "kdkl_last_error",
-    "kdkl_last_launch_count", "kdkl_logz_noalloc",
+    "kdkl_last_launch_count", "kdkl_logz_noalloc", "kdkl_forward_shard", "kdkl_forward_finish",
 ]
 
 
@@ -57,6 +57,11 @@ def lib() -> ctypes.CDLL:
     L.kdkl_workspace_bytes.argtypes = [i64, i64, i64, i32, i64, vp]
     L.kdkl_forward.restype = ctypes.c_int
     L.kdkl_forward.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, vp, sz, vp, vp, vp, vp, vp]
+    L.kdkl_forward_shard.restype = ctypes.c_int
+    L.kdkl_forward_shard.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i32, i64, f32, vp, vp, sz,
+                                     vp, vp, vp, vp]
+    L.kdkl_forward_finish.restype = ctypes.c_int
+    L.kdkl_forward_finish.argtypes = [vp, i32, vp, i64, i64, i64, i32, i64, f32, vp, vp, sz, vp, vp, vp]
     L.kdkl_backward.restype = ctypes.c_int
     L.kdkl_backward.argtypes = [vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, f32, vp, sz, vp, vp, vp]
     L.kdkl_status.restype = ctypes.c_int
@@ -127,6 +132,28 @@ def kdkl_backward(hidden, weight, K, workspace, dhidden, dweight, *, loss_mask=N
     _check(lib().kdkl_backward(_ptr(hidden), _ptr(weight), _ptr(loss_mask), T, H, V, K, chunk, temperature,
                                _opt_ptr(opt), grad_loss, _ptr(workspace),
                                workspace.numel() * workspace.element_size(), _ptr(dhidden), _ptr(dweight), _stream()))
+
+
+def kdkl_forward_shard(hidden, weight_local, topk_idx, topk_val, workspace, shard_stats, *, vocab_offset, V_total,
+                       teacher_lse=None, loss_mask=None, chunk=0, temperature=1.0, opt=None, gathered_logits=None,
+                       gathered_idx=None) -> None:
+    """The local sweep of one vocabulary shard; fills shard_stats [2, T] (see include/kdkl.h)."""
+    T, H = hidden.shape
+    V_local = weight_local.shape[0]
+    K = topk_idx.shape[1]
+    _check(lib().kdkl_forward_shard(_ptr(hidden), _ptr(weight_local), _ptr(topk_idx), _ptr(topk_val),
+                                    _ptr(teacher_lse), _ptr(loss_mask), T, H, V_local, vocab_offset, V_total, K, chunk,
+                                    temperature, _opt_ptr(opt), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _ptr(shard_stats),
+                                    _ptr(gathered_logits), _ptr(gathered_idx), _stream()))
+
+
+def kdkl_forward_finish(all_stats, n_shards, T, H, V_local, K, workspace, loss_out, *, loss_mask=None, chunk=0,
+                        temperature=1.0, opt=None, loss_per_token=None) -> None:
+    """Completes the sharded forward from the gathered statistics [n_shards, 2, T]."""
+    _check(lib().kdkl_forward_finish(_ptr(all_stats), n_shards, _ptr(loss_mask), T, H, V_local, K, chunk, temperature,
+                                     _opt_ptr(opt), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                     _ptr(loss_out), _ptr(loss_per_token), _stream()))
 
 
 def kdkl_status(workspace):
@@ -240,3 +267,68 @@ class FusedChunkedKL:
 
     def saved_state(self):
         return kdkl_saved_state(self.workspace, self.T, self.H, self.V, self.K, self.chunk, self.opt)
+
+
+class ShardedFusedChunkedKL:
+    """One rank of the vocabulary-sharded loss (the paper's tensor-parallel variant).
+
+    The kernels do the local work; the two exchanges of Algorithm 1 are the caller's collectives:
+    an all-gather of the [2, T] shard statistics between the local sweep and the finish, and a sum of
+    the fp32 partial dhidden over ranks after backward. By default they go through torch.distributed
+    (NCCL); ``all_gather(out[n,2,T], local[2,T])`` and ``all_reduce_sum(tensor)`` can be injected.
+    """
+
+    def __init__(self, T, H, V_local, vocab_offset, V_total, K, n_shards, chunk=0, temperature=1.0, device="cuda",
+                 all_gather=None, all_reduce_sum=None, want_per_token=False):
+        self.T, self.H, self.V_local, self.K = T, H, V_local, K
+        self.vocab_offset, self.V_total, self.n_shards = vocab_offset, V_total, n_shards
+        self.chunk, self.temperature = chunk, temperature
+        self.opt = make_options(dhidden_dtype=1)            # fp32 partial dhidden: summed over ranks in fp32
+        self.workspace = torch.empty(kdkl_workspace_bytes(T, H, V_local, K, chunk, self.opt), dtype=torch.uint8,
+                                     device=device)
+        self.stats_local = torch.empty(2, T, dtype=torch.float32, device=device)
+        self.stats_all = torch.empty(n_shards, 2, T, dtype=torch.float32, device=device)
+        self.loss = torch.zeros(1, dtype=torch.float32, device=device)
+        self.loss_per_token = torch.empty(T, dtype=torch.float32, device=device) if want_per_token else None
+        self.dhidden = torch.empty(T, H, dtype=torch.float32, device=device)
+        self.dweight = torch.empty(V_local, H, dtype=torch.float32, device=device)
+        self._all_gather = all_gather or self._dist_all_gather
+        self._all_reduce_sum = all_reduce_sum or self._dist_all_reduce
+
+    @staticmethod
+    def _dist_all_gather(out, local):
+        import torch.distributed as dist
+        dist.all_gather_into_tensor(out.view(-1, out.shape[-1]), local)   # [R*2, T]: rank r's rows at 2r, 2r+1
+
+    @staticmethod
+    def _dist_all_reduce(t):
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+
+    def forward_local(self, hidden, weight_local, topk_idx, topk_val, teacher_lse=None, loss_mask=None):
+        kdkl_forward_shard(hidden, weight_local, topk_idx, topk_val, self.workspace, self.stats_local,
+                           vocab_offset=self.vocab_offset, V_total=self.V_total, teacher_lse=teacher_lse,
+                           loss_mask=loss_mask, chunk=self.chunk, temperature=self.temperature, opt=self.opt)
+
+    def forward_finish(self, loss_mask=None):
+        kdkl_forward_finish(self.stats_all, self.n_shards, self.T, self.H, self.V_local, self.K, self.workspace,
+                            self.loss, loss_mask=loss_mask, chunk=self.chunk, temperature=self.temperature,
+                            opt=self.opt, loss_per_token=self.loss_per_token)
+        return self.loss
+
+    def forward(self, hidden, weight_local, topk_idx, topk_val, teacher_lse=None, loss_mask=None):
+        self.forward_local(hidden, weight_local, topk_idx, topk_val, teacher_lse, loss_mask)
+        self._all_gather(self.stats_all, self.stats_local)          # Algorithm 1: distributed max / reduce sigma
+        return self.forward_finish(loss_mask)
+
+    def backward_local(self, hidden, weight_local, loss_mask=None, grad_loss=1.0):
+        kdkl_backward(hidden, weight_local, self.K, self.workspace, self.dhidden, self.dweight, loss_mask=loss_mask,
+                      chunk=self.chunk, temperature=self.temperature, opt=self.opt, grad_loss=grad_loss)
+
+    def backward(self, hidden, weight_local, loss_mask=None, grad_loss=1.0):
+        self.backward_local(hidden, weight_local, loss_mask, grad_loss)
+        self._all_reduce_sum(self.dhidden)                          # Algorithm 1: reduce dh across shards
+        return self.dhidden, self.dweight
+
+    def status(self):
+        return kdkl_status(self.workspace)

@@ -53,12 +53,15 @@ __global__ void header_reset_kernel(WsHeader* hdr) {
 // and an index-sorted copy of the row (idx ascending, p merged over duplicate indices, the
 // original slot of every entry) that the GEMM epilogues walk with a cursor.
 // Ignored tokens (mask = 0) get an empty row: their teacher entries are never read.
+// Vocabulary shards: this rank owns rows [v0, v0 + V) of a vocabulary of V_total entries. Every
+// usable teacher entry (index < V_total) counts towards p, M and Hent on every rank; only the
+// entries inside the local window are gathered here, under their local index.
 constexpr int PREP_WARPS = 4;
 constexpr int kKeyUnusable = 0x7ffffffe, kKeyPad = 0x7fffffff;
 __global__ void __launch_bounds__(PREP_WARPS * 32)
 prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val,
-            const float* __restrict__ teacher_lse, const uint8_t* __restrict__ mask, long long T, int V, int K,
-            int Kpad, float inv_tau, int teacher_mode, int* __restrict__ idx_sorted, float* __restrict__ p_sorted,
+            const float* __restrict__ teacher_lse, const uint8_t* __restrict__ mask, long long T, int V, int v0,
+            int V_total, int K, int Kpad, float inv_tau, int teacher_mode, int* __restrict__ idx_sorted, float* __restrict__ p_sorted,
             uint16_t* __restrict__ perm, int* __restrict__ nvalid, float* __restrict__ Mout,
             float* __restrict__ Hent, WsHeader* hdr) {
   extern __shared__ uint8_t prep_smem[];
@@ -81,15 +84,18 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
   // load, validate, scaled values
   float mx = -INFINITY;
   int bad = 0;
-  // keys: a usable index < kKeyUnusable (real slot without a usable index) < kKeyPad (sort padding),
-  // so after the sort positions [nvalid, K) hold exactly the real slots that were not gathered
+  // keys: the global index < kKeyUnusable (real slot without a usable index) < kKeyPad (sort padding).
+  // Every rank sorts the same keys, so M and Hent below are summed in the same order everywhere and
+  // come out bitwise identical on all shards.
   for (int k = lane; k < Kpad; k += 32) {
     int key = k < K ? kKeyUnusable : kKeyPad;
     float u = -INFINITY;
     if (k < K) {
       const int id = topk_idx[t * K + k];
-      if (id >= 0 && id < V) { key = id; u = topk_val[t * K + k] * inv_tau; }
-      else if (id >= V) bad++;
+      if (id >= 0 && id < V_total) {
+        key = id;
+        u = topk_val[t * K + k] * inv_tau;
+      } else if (id >= V_total) bad++;
     }
     keys[k] = key; pv[k] = u; slot[k] = (uint16_t)k;
     mx = fmaxf(mx, u);
@@ -128,25 +134,41 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
       __syncwarp();
     }
   }
-  // merge duplicate indices into the head of each run (scatter-add semantics)
+  // merge duplicate indices into the head of each run (scatter-add semantics). Shared memory is only
+  // read from here on, so lanes may run ahead of each other.
+  auto merged_p = [&](int j) -> float {
+    const int key = keys[j];
+    if (key >= kKeyUnusable || (j > 0 && keys[j - 1] == key)) return 0.f;
+    float pj = pv[j];
+    for (int q = j + 1; q < Kpad && keys[q] == key; ++q) pj += pv[q];
+    return pj;
+  };
+  // M, Hent, and the number of entries below / inside this rank's vocabulary window [v0, v0 + V)
   float msum = 0.f, hsum = 0.f;
-  int nv = 0;
+  int lo = 0, hi = 0;
   for (int j = lane; j < Kpad; j += 32) {
     const int key = keys[j];
-    float pj = 0.f;
     if (key < kKeyUnusable) {
-      nv++;
-      if (j == 0 || keys[j - 1] != key) {
-        pj = pv[j];
-        for (int q = j + 1; q < Kpad && keys[q] == key; ++q) pj += pv[q];
-        msum += pj;
-        if (pj > 0.f) hsum += pj * logf(pj);
-      }
+      if (key < v0) lo++;
+      if (key < v0 + V) hi++;
+      const float pj = merged_p(j);
+      msum += pj;
+      if (pj > 0.f) hsum += pj * logf(pj);
     }
-    if (j < K) { out_idx[j] = key; out_p[j] = pj; out_perm[j] = slot[j]; }
   }
   msum = warp_sum(msum); hsum = warp_sum(hsum);
-  nv = (int)warp_sum((float)nv);
+  lo = (int)warp_sum((float)lo); hi = (int)warp_sum((float)hi);
+  // write out with the local window rotated to the front: positions [0, hi - lo) hold this rank's
+  // entries under their local index, ascending; the rest follows (never gathered here)
+  const int nv = hi - lo;
+  for (int j = lane; j < K; j += 32) {
+    const int key = keys[j];
+    const bool local = j >= lo && j < hi;
+    const int pos = local ? j - lo : (j < lo ? nv + j : j);
+    out_idx[pos] = local ? key - v0 : key;
+    out_p[pos] = merged_p(j);
+    out_perm[pos] = slot[j];
+  }
   if (lane == 0) { nvalid[t] = nv; Mout[t] = msum; Hent[t] = hsum; }
 }
 
@@ -163,7 +185,7 @@ combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_
                const int* __restrict__ colread, const float* __restrict__ Mv, const float* __restrict__ Hent,
                const uint8_t* __restrict__ mask, float* __restrict__ lz2, float* __restrict__ logZ_nat,
                float* __restrict__ loss_tok, float* __restrict__ loss_tok_user, float* __restrict__ g_logits,
-               int* __restrict__ g_idx, WsHeader* hdr) {
+               int* __restrict__ g_idx, int v0, float* __restrict__ shard_stats, long long T_total, WsHeader* hdr) {
   __shared__ float sm_m[8][32], sm_s[8][32];
   __shared__ float sm_lz[32];
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
@@ -208,13 +230,18 @@ combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_
         const float z = zg[t * K + j];
         c += p_sorted[t * K + j] * z;
         if (g_logits) g_logits[t * K + sl] = z;
-        if (g_idx) g_idx[t * K + sl] = colread[t * K + j];
+        if (g_idx) g_idx[t * K + sl] = colread[t * K + j] + v0;
       } else {
         if (g_logits) g_logits[t * K + sl] = __int_as_float(0x7fc00000);
         if (g_idx) g_idx[t * K + sl] = -1;
       }
     }
     c = warp_sum(c) * inv_tau;
+    if (shard_stats != nullptr) {
+      // a vocabulary shard: hand the local log-normaliser and cross term to the cross-shard reduction
+      if (tx == 0) { shard_stats[t] = sm_lz[ty * 4 + i]; shard_stats[T_total + t] = c; }
+      continue;
+    }
     if (tx == 0) {
       const bool counted = mask == nullptr || mask[t] != 0;
       const float lz = sm_lz[ty * 4 + i] * kLn2;
@@ -227,6 +254,37 @@ combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_
       if (loss_tok_user) loss_tok_user[t] = L;
     }
   }
+}
+
+// ------------------------------------------------------------------------------------ shard finish
+// After the shards' statistics have been gathered ([R][2][T]: log2-domain local normaliser, local cross
+// term): log Z = logsumexp over shards, C = sum over shards (fixed order), L = Hent - C + M log Z.
+// Writes the global normaliser over the local one so that backward rebuilds the global softmax.
+__global__ void shard_finish_kernel(const float* __restrict__ all_stats, int R, long long T,
+                                    const float* __restrict__ Mv, const float* __restrict__ Hent,
+                                    const uint8_t* __restrict__ mask, float* __restrict__ lz2,
+                                    float* __restrict__ logZ_nat, float* __restrict__ loss_tok,
+                                    float* __restrict__ loss_tok_user, WsHeader* hdr) {
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= T) return;
+  float m = -INFINITY;
+  for (int r = 0; r < R; ++r) m = fmaxf(m, all_stats[(long long)r * 2 * T + t]);
+  float s = 0.f, c = 0.f;
+  for (int r = 0; r < R; ++r) {
+    s += exp2f(all_stats[(long long)r * 2 * T + t] - m);
+    c += all_stats[(long long)r * 2 * T + T + t];
+  }
+  const float l2 = m + log2f(s);
+  lz2[t] = l2;
+  logZ_nat[t] = l2 * kLn2;
+  const bool counted = mask == nullptr || mask[t] != 0;
+  float L = 0.f;
+  if (counted) {
+    L = Hent[t] - c + Mv[t] * l2 * kLn2;
+    if (!isfinite(L)) { atomicCAS(&hdr->status, 0, -11); atomicCAS(&hdr->where, 0, (int)t); }
+  }
+  loss_tok[t] = L;
+  if (loss_tok_user) loss_tok_user[t] = L;
 }
 
 // ------------------------------------------------------------------------------------ loss reduce

@@ -261,12 +261,16 @@ size_t kdkl_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t 
   return ws_layout(T, H, V, K, chunk).total;
 }
 
-int kdkl_forward(const void* hidden, const void* weight, const int32_t* topk_idx, const float* topk_val,
-                 const float* teacher_lse, const uint8_t* loss_mask, int64_t T, int64_t H, int64_t V, int32_t K,
-                 int64_t chunk, float tau, const kdkl_options* opt, void* ws, size_t ws_bytes, float* loss_out,
-                 float* loss_per_token, float* gathered_logits, int32_t* gathered_idx, void* cuda_stream) {
+// Forward over the vocabulary rows [v0, v0 + V) this caller holds. Unsharded: v0 = 0, V_total = V,
+// shard_stats = NULL and the loss is finished here. Sharded: the per-token local normaliser and cross
+// term go to shard_stats [2, T] and kdkl_forward_finish completes the loss after the gather.
+static int forward_impl(const void* hidden, const void* weight, const int32_t* topk_idx, const float* topk_val,
+                        const float* teacher_lse, const uint8_t* loss_mask, int64_t T, int64_t H, int64_t V,
+                        int64_t v0, int64_t V_total, int32_t K, int64_t chunk, float tau, const kdkl_options* opt,
+                        void* ws, size_t ws_bytes, float* shard_stats, float* loss_out, float* loss_per_token,
+                        float* gathered_logits, int32_t* gathered_idx, void* cuda_stream) {
   g_launches = 0;
-  if (!topk_idx || !topk_val || !loss_out) return KDKL_ERR_NULL;
+  if (!topk_idx || !topk_val || (!loss_out && !shard_stats)) return KDKL_ERR_NULL;
   kdkl_options o;
   WsLayout L;
   int rc = check_common(hidden, weight, T, H, V, K, chunk, tau, opt, ws, ws_bytes, &o, &L);
@@ -284,7 +288,7 @@ int kdkl_forward(const void* hidden, const void* weight, const int32_t* topk_idx
   const int Kpad = next_pow2(K);
   const size_t prep_smem = (size_t)PREP_WARPS * Kpad * (4 + 4 + 2);
   prep_kernel<<<(unsigned)((T + PREP_WARPS - 1) / PREP_WARPS), PREP_WARPS * 32, prep_smem, st>>>(
-      topk_idx, topk_val, teacher_lse, loss_mask, T, (int)V, K, Kpad, inv_tau, o.teacher_mode,
+      topk_idx, topk_val, teacher_lse, loss_mask, T, (int)V, (int)v0, (int)V_total, K, Kpad, inv_tau, o.teacher_mode,
       at<int>(ws, L.idx_sorted), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<int>(ws, L.nvalid),
       at<float>(ws, L.M), at<float>(ws, L.Hent), hdr);
   KDKL_LAUNCHED("prep_kernel");
@@ -316,11 +320,58 @@ int kdkl_forward(const void* hidden, const void* weight, const int32_t* topk_idx
         at<float>(ws, L.part_m), at<float>(ws, L.part_s), L.Cpad, (int)L.n_tiles_v, (int)rows, s0, K, inv_tau,
         at<int>(ws, L.nvalid), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<float>(ws, L.zg),
         at<int>(ws, L.colread), at<float>(ws, L.M), at<float>(ws, L.Hent), loss_mask, at<float>(ws, L.lz2),
-        at<float>(ws, L.logZ), at<float>(ws, L.loss_tok), loss_per_token, gathered_logits, gathered_idx, hdr);
+        at<float>(ws, L.logZ), at<float>(ws, L.loss_tok), loss_per_token, gathered_logits, gathered_idx, (int)v0,
+        shard_stats, T, hdr);
     KDKL_LAUNCHED("combine_kernel");
   }
+  if (shard_stats != nullptr) return KDKL_OK;   // the loss is completed by kdkl_forward_finish
   stage_mark(ST_REDUCE, st);
   loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, tau, H, V, K,
+                                         loss_out, hdr);
+  KDKL_LAUNCHED("loss_reduce_kernel");
+  return KDKL_OK;
+}
+
+int kdkl_forward(const void* hidden, const void* weight, const int32_t* topk_idx, const float* topk_val,
+                 const float* teacher_lse, const uint8_t* loss_mask, int64_t T, int64_t H, int64_t V, int32_t K,
+                 int64_t chunk, float tau, const kdkl_options* opt, void* ws, size_t ws_bytes, float* loss_out,
+                 float* loss_per_token, float* gathered_logits, int32_t* gathered_idx, void* cuda_stream) {
+  if (!loss_out) return KDKL_ERR_NULL;
+  return forward_impl(hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, T, H, V, 0, V, K, chunk, tau, opt, ws,
+                      ws_bytes, nullptr, loss_out, loss_per_token, gathered_logits, gathered_idx, cuda_stream);
+}
+
+int kdkl_forward_shard(const void* hidden, const void* weight_local, const int32_t* topk_idx, const float* topk_val,
+                       const float* teacher_lse, const uint8_t* loss_mask, int64_t T, int64_t H, int64_t V_local,
+                       int64_t vocab_offset, int64_t V_total, int32_t K, int64_t chunk, float tau,
+                       const kdkl_options* opt, void* ws, size_t ws_bytes, float* shard_stats, float* gathered_logits,
+                       int32_t* gathered_idx, void* cuda_stream) {
+  if (!shard_stats) return KDKL_ERR_NULL;
+  if (vocab_offset < 0 || V_local < 1 || vocab_offset + V_local > V_total || V_total >= (1ll << 30)) return KDKL_ERR_SHAPE;
+  return forward_impl(hidden, weight_local, topk_idx, topk_val, teacher_lse, loss_mask, T, H, V_local, vocab_offset,
+                      V_total, K, chunk, tau, opt, ws, ws_bytes, shard_stats, nullptr, nullptr, gathered_logits,
+                      gathered_idx, cuda_stream);
+}
+
+int kdkl_forward_finish(const float* all_stats, int32_t n_shards, const uint8_t* loss_mask, int64_t T, int64_t H,
+                        int64_t V_local, int32_t K, int64_t chunk, float tau, const kdkl_options* opt, void* ws,
+                        size_t ws_bytes, float* loss_out, float* loss_per_token, void* cuda_stream) {
+  g_launches = 0;
+  if (!all_stats || !loss_out || !ws) return KDKL_ERR_NULL;
+  if (n_shards < 1 || T < 1 || H < 1 || V_local < 1 || K < 1) return KDKL_ERR_SHAPE;
+  kdkl_options o;
+  memset(&o, 0, sizeof(o));
+  if (opt) { if (opt->struct_size != (int32_t)sizeof(kdkl_options)) return KDKL_ERR_ARG; o = *opt; }
+  WsLayout L = ws_layout(T, H, V_local, K, chunk);
+  if (ws_bytes < L.total) return KDKL_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  WsHeader* hdr = at<WsHeader>(ws, L.hdr);
+  shard_finish_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(all_stats, n_shards, T, at<float>(ws, L.M),
+                                                                   at<float>(ws, L.Hent), loss_mask,
+                                                                   at<float>(ws, L.lz2), at<float>(ws, L.logZ),
+                                                                   at<float>(ws, L.loss_tok), loss_per_token, hdr);
+  KDKL_LAUNCHED("shard_finish_kernel");
+  loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, tau, H, V_local, K,
                                          loss_out, hdr);
   KDKL_LAUNCHED("loss_reduce_kernel");
   return KDKL_OK;
