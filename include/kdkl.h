@@ -189,6 +189,12 @@ int kdkl_gemm_bf16(const void* A, const void* B, float* C, int64_t M, int64_t N,
 int kdkl_logz_noalloc(const void* hidden_bf16, const void* weight_bf16, int64_t T, int64_t H, int64_t V,
                       float temperature, float* logz_out, void* cuda_stream);
 
+/* Exercises the bounded wait every kernel of this library uses on its mbarriers: one thread waits on
+ * a barrier that nothing completes, gives up after limit_ns (1 .. 1e9) and the kernel returns normally.
+ * status: device int32[2], zeroed by the caller; afterwards {KDKL_ERR_TIMEOUT, 99}. The context stays
+ * usable. (No counterpart in the paper: failure handling of this implementation.) */
+int kdkl_wait_selftest(int32_t* status, int64_t limit_ns, void* cuda_stream);
+
 /* Text of the last KDKL_ERR_CUDA on this thread. */
 const char* kdkl_last_error(void);
 

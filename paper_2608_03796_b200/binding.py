@@ -26,6 +26,7 @@ EXPORTS = [
     "kdkl_workspace_bytes", "kdkl_forward", "kdkl_backward", "kdkl_status", "kdkl_saved_state",
     "kdkl_host_arena_bytes", "kdkl_forward_backward_host", "kdkl_profile_stages", "kdkl_gemm_bf16", "kdkl_last_error",
     "kdkl_last_launch_count", "kdkl_logz_noalloc", "kdkl_forward_shard", "kdkl_forward_finish",
+    "kdkl_wait_selftest",
 ]
 
 
@@ -80,6 +81,8 @@ def lib() -> ctypes.CDLL:
     L.kdkl_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, vp, vp]
     L.kdkl_logz_noalloc.restype = ctypes.c_int
     L.kdkl_logz_noalloc.argtypes = [vp, vp, i64, i64, i64, f32, vp, vp]
+    L.kdkl_wait_selftest.restype = ctypes.c_int
+    L.kdkl_wait_selftest.argtypes = [vp, i64, vp]
     L.kdkl_last_error.restype = ctypes.c_char_p
     L.kdkl_last_error.argtypes = []
     L.kdkl_last_launch_count.restype = ctypes.c_int64
@@ -224,6 +227,11 @@ def kdkl_logz_noalloc(hidden, weight, logz_out, temperature=1.0) -> None:
     T, H = hidden.shape
     V = weight.shape[0]
     _check(lib().kdkl_logz_noalloc(_ptr(hidden), _ptr(weight), T, H, V, temperature, _ptr(logz_out), _stream()))
+
+
+def kdkl_wait_selftest(status, limit_ns: int) -> None:
+    """A wait nobody satisfies must expire into status = {KDKL_ERR_TIMEOUT, 99} (see include/kdkl.h)."""
+    _check(lib().kdkl_wait_selftest(_ptr(status), limit_ns, _stream()))
 
 
 def kdkl_last_launch_count() -> int:

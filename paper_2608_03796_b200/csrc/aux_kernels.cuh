@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "sm100_prims.cuh"
+
 namespace kdkl {
 
 constexpr int KDKL_MAGIC = 0x4b444b4c;  // "KDKL"
@@ -362,6 +364,21 @@ splitk_fixup_kernel(const float* __restrict__ part, long long slab, int splits, 
     v.x = *reinterpret_cast<uint32_t*>(&lo);
     v.y = *reinterpret_cast<uint32_t*>(&hi);
     reinterpret_cast<uint2*>(out_bf16)[i] = v;
+  }
+}
+
+// ------------------------------------------------------------------------------------ wait self-test
+// One thread waits on an mbarrier that nothing will ever complete, with a short limit. The wait must
+// give up, record KDKL_ERR_TIMEOUT and the site in status[0..1], and the kernel must return normally.
+__global__ void wait_expiry_kernel(int* status, unsigned long long limit_ns, int site) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    mbar_fence_init();
+    const bool ok = mbar_wait(smem_u32(&bar), 0u, &abort_flag, status, site, limit_ns);
+    if (ok) atomicExch(status + 1, -1);   // would mean the barrier completed by itself
   }
 }
 

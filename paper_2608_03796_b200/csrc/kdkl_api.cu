@@ -129,11 +129,9 @@ static int launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUten
                        int sm_count, cudaStream_t st) {
   auto kern = gemm_tcgen05_kernel<EPI, A_MN, B_MN, kNCTA>;
   constexpr int smem = GemmCfg<kNCTA>::SMEM_BYTES;
-  static bool attr_set = false;   // per instantiation
-  if (!attr_set) {
-    KDKL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    attr_set = true;
-  }
+  // set on every launch: the attribute belongs to the current device's copy of the kernel, and a
+  // process may drive several devices
+  KDKL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
   // persistent: one worker (a CTA, or a pair of CTAs on neighbouring SMs) per SM (pair), each walking
   // the work units with a stride of the worker count
   const int units = p.m_tiles * p.n_tiles * p.k_splits;
@@ -604,6 +602,16 @@ int kdkl_profile_stages(const void* hidden, const void* weight, const int32_t* t
   g_timer.stage.clear();
   if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
   return rc;
+}
+
+// ------------------------------------------------------------------ bounded-wait self-test
+int kdkl_wait_selftest(int32_t* status, int64_t limit_ns, void* cuda_stream) {
+  if (!status) return KDKL_ERR_NULL;
+  if (limit_ns < 1 || limit_ns > 1000000000ll) return KDKL_ERR_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  wait_expiry_kernel<<<1, 32, 0, st>>>(status, (unsigned long long)limit_ns, 99);
+  KDKL_LAUNCHED("wait_expiry_kernel");
+  return KDKL_OK;
 }
 
 // ------------------------------------------------------------------ bare GEMM

@@ -50,7 +50,7 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;
 // Bounded wait. Returns false when the CTA has aborted (flag set by any role) or the
 // limit expired (then it sets the flag itself and records `where` in the status word).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status_word, int where) {
+                                          int* status_word, int where, uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = globaltimer_ns();
   uint32_t spins = 0;
@@ -58,7 +58,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      if (globaltimer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         if (status_word != nullptr) {
           atomicCAS(status_word, 0, -8);       // KDKL_ERR_TIMEOUT
