@@ -28,6 +28,9 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 def _cfg(name: str):
     from paper_2608_03796_b200 import inputs as I
+    if "@" in name:                                # a config at another chunk size, e.g. c3@8192
+        base, chunk = name.split("@")
+        return dataclasses.replace(_cfg(base), name=name, chunk=int(chunk))
     if name in I.CONFIGS:
         return I.CONFIGS[name]
     if name.startswith("T"):                       # the 4K shape at another length, e.g. T8192
@@ -154,7 +157,7 @@ def main():
         # least-squares line through the fused peaks of the H=4096 / V=131072 family
         pts = [(r["T"], r["peak_gb"]) for r in rows if r["method"] == "fused" and "ms_per_iter" in r
                and r["H"] == 4096 and r["V"] == 131072 and r["T"] >= 32768]
-        if len(pts) >= 3:
+        if len(pts) >= 3 and len({p[0] for p in pts}) >= 3:
             n = len(pts)
             sx = sum(p[0] for p in pts); sy = sum(p[1] for p in pts)
             sxx = sum(p[0] * p[0] for p in pts); sxy = sum(p[0] * p[1] for p in pts)
