@@ -263,6 +263,15 @@ def main():
     peak_mem = torch.cuda.max_memory_allocated()
     ws_bytes = op.workspace.numel()
 
+    # peak memory versus sequence length for this shape, from the allocation sizes alone (inputs + outputs +
+    # workspace; the measured sweep is in profiles/): the vocabulary-sized part does not grow with T
+    def allocation_gb(tokens):
+        mask_bytes = tokens if d["mask"] is not None else 0
+        fixed = V * H * 2 + V * H * 4 + 4
+        per_t = tokens * (H * 2 + K * 8 + H * 2) + mask_bytes
+        return (fixed + per_t + B.kdkl_workspace_bytes(tokens, H, V, K, cfg.chunk)) / 1e9
+    mem_model = {str(t): round(allocation_gb(t), 3) for t in (4096, 32768, 65536, 131072, 262144)}
+
     # per-kernel times, live, with an event between kernels (a separate short run)
     stage_acc = {}
     n_prof = 1 if args.capture else 3
@@ -347,6 +356,7 @@ def main():
                                                                      FALLBACK_PEAKS["bf16_tflops_sustained"])),
         "peaks": peaks.get("_source"),
         "peak_mem_gb": peak_mem / 1e9, "workspace_gb": ws_bytes / 1e9, "input_mem_gb": base_mem / 1e9,
+        "peak_mem_gb_vs_tokens": mem_model,
         "loss": loss_val,
         "clocks": clk.summary(),
         "gpu_launches": launches_per_step * args.steps,
