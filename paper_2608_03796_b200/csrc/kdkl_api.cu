@@ -380,11 +380,11 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
                   size_t ws_bytes, void* dhidden, float* dweight, void* cuda_stream) {
   g_launches = 0;
   if (!dhidden || !dweight) return KDKL_ERR_NULL;
+  if (((uintptr_t)dhidden & 15) || ((uintptr_t)dweight & 15)) return KDKL_ERR_ALIGN;
   kdkl_options o;
   WsLayout L;
   int rc = check_common(hidden, weight, T, H, V, K, chunk, tau, opt, ws, ws_bytes, &o, &L);
   if (rc) return rc;
-  if (((uintptr_t)dhidden & 15) || ((uintptr_t)dweight & 15)) return KDKL_ERR_ALIGN;
   DeviceInfo di;
   if ((rc = device_info(&di))) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);

@@ -41,3 +41,39 @@ def test_sizes_without_a_gpu():
 def test_options_struct_layout():
     o = binding.make_options(teacher_mode=1, denom_override=3.0)
     assert o.struct_size == 20 and o.teacher_mode == 1 and o.denom_override == 3.0
+
+
+def test_host_side_argument_checks_without_a_gpu():
+    """Argument errors are detected before any CUDA call, so they can be checked on a CPU-only box.
+    Pointers are fake but non-null and aligned: nothing dereferences them on these paths."""
+    entry.build()
+    L = binding.lib()
+    P, Q = 0x10000, 0x20000                       # 16-byte aligned dummies
+    T, H, V, K = 64, 64, 512, 4
+    ws = binding.kdkl_workspace_bytes(T, H, V, K)
+
+    def fwd(hidden=P, weight=P, idx=P, val=P, T=T, H=H, V=V, K=K, chunk=0, tau=1.0, opt=None, wsp=Q, wsb=ws, loss=P):
+        return L.kdkl_forward(hidden, weight, idx, val, None, None, T, H, V, K, chunk, tau, opt, wsp, wsb, loss,
+                              None, None, None, None)
+    assert fwd(hidden=None) == -1 and fwd(loss=None) == -1 and fwd(idx=None) == -1
+    assert fwd(T=0) == -2 and fwd(H=60) == -2 and fwd(K=0) == -2 and fwd(K=2000) == -2
+    assert fwd(tau=0.0) == -5 and fwd(tau=-1.0) == -5 and fwd(chunk=-1) == -5
+    assert fwd(hidden=P + 2) == -3 and fwd(wsp=Q + 8) == -3
+    assert fwd(wsb=ws - 1) == -4
+    bad_opt = binding.make_options()
+    bad_opt.struct_size = 7
+    assert fwd(opt=binding._opt_ptr(bad_opt)) == -5
+    assert fwd(opt=binding._opt_ptr(binding.make_options(teacher_mode=1)), tau=2.0) == -5
+    # backward: same checks plus its own outputs
+    def bwd(dh=P, dw=P, **kw):
+        a = dict(hidden=P, weight=P, T=T, H=H, V=V, K=K, chunk=0, tau=1.0, wsp=Q, wsb=ws)
+        a.update(kw)
+        return L.kdkl_backward(a["hidden"], a["weight"], None, a["T"], a["H"], a["V"], a["K"], a["chunk"], a["tau"],
+                               None, 1.0, a["wsp"], a["wsb"], dh, dw, None)
+    assert bwd(dh=None) == -1 and bwd(dw=None) == -1 and bwd(V=0) == -2 and bwd(wsb=16) == -4 and bwd(dw=P + 4) == -3
+    # sharded entry: window must lie inside the vocabulary
+    assert L.kdkl_forward_shard(P, P, P, P, None, None, T, H, 256, 300, V, K, 0, 1.0, None, Q, ws, P, None, None,
+                                None) == -2
+    assert L.kdkl_gemm_bf16(P, P, P, 64, 64, 60, 0, 0, None, None) == -2
+    assert L.kdkl_wait_selftest(P, 0, None) == -5
+    assert L.kdkl_logz_noalloc(P, P, 8, 64, 262144 + 256, 1.0, P, None) == -4
