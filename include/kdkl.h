@@ -189,6 +189,25 @@ int kdkl_gemm_bf16(const void* A, const void* B, float* C, int64_t M, int64_t N,
 int kdkl_logz_noalloc(const void* hidden_bf16, const void* weight_bf16, int64_t T, int64_t H, int64_t V,
                       float temperature, float* logz_out, void* cuda_stream);
 
+#define KDKL_ERR_OVERFLOW (-12) /* teacher top-K: more logits tied at the selection threshold than the list holds */
+
+/* The teacher cache record of the offline pipeline (paper, section "Offline Distillation with a Top-K
+ * Teacher": the K largest entries per position are cached; the retained mass M <= 1 is not renormalised,
+ * which needs the full normaliser). For teacher hidden states [T, H] and teacher head [V, H] (bf16):
+ *   topk_idx [T, K] int32, topk_val [T, K] fp32: the K largest logits z = W h per token, by value
+ *            descending, ties by the smaller index first (exact selection, not an approximation);
+ *   lse [T] fp32: log sum_v exp(z_v / temperature), the `teacher_lse` argument of kdkl_forward.
+ * Two tensor-core sweeps: the first gives the log-sum-exp and per-vocab-tile maxima, whose K-th largest
+ * is a threshold that every member of the top-K must reach; the second recomputes the logits and keeps
+ * those at or above it; a per-row sort finishes. K <= 256, K <= V <= 2^20, H % 8 == 0, and either
+ * V >= 256 K (at least K vocabulary tiles, so the threshold exists) or V <= 8192 (every logit is sorted).
+ * workspace: device, kdkl_teacher_topk_workspace_bytes(); its first words are a status block readable
+ * with kdkl_status (KDKL_ERR_OVERFLOW / KDKL_ERR_TIMEOUT). Enqueue-only. */
+size_t kdkl_teacher_topk_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K);
+int kdkl_teacher_topk(const void* hidden_bf16, const void* weight_bf16, int64_t T, int64_t H, int64_t V, int32_t K,
+                      float temperature, void* workspace, size_t workspace_bytes, int32_t* topk_idx,
+                      float* topk_val, float* lse, void* cuda_stream);
+
 /* Exercises the bounded wait every kernel of this library uses on its mbarriers: one thread waits on
  * a barrier that nothing completes, gives up after limit_ns (1 .. 1e9) and the kernel returns normally.
  * status: device int32[2], zeroed by the caller; afterwards {KDKL_ERR_TIMEOUT, 99}. The context stays

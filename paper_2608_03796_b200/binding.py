@@ -19,14 +19,14 @@ KDKL_OK = 0
 ERRORS = {
     -1: "KDKL_ERR_NULL", -2: "KDKL_ERR_SHAPE", -3: "KDKL_ERR_ALIGN", -4: "KDKL_ERR_WORKSPACE",
     -5: "KDKL_ERR_ARG", -6: "KDKL_ERR_ARCH", -7: "KDKL_ERR_CUDA", -8: "KDKL_ERR_TIMEOUT",
-    -9: "KDKL_ERR_STATE", -10: "KDKL_ERR_INDEX", -11: "KDKL_ERR_NONFINITE",
+    -9: "KDKL_ERR_STATE", -10: "KDKL_ERR_INDEX", -11: "KDKL_ERR_NONFINITE", -12: "KDKL_ERR_OVERFLOW",
 }
 
 EXPORTS = [
     "kdkl_workspace_bytes", "kdkl_forward", "kdkl_backward", "kdkl_status", "kdkl_saved_state",
     "kdkl_host_arena_bytes", "kdkl_forward_backward_host", "kdkl_profile_stages", "kdkl_gemm_bf16", "kdkl_last_error",
     "kdkl_last_launch_count", "kdkl_logz_noalloc", "kdkl_forward_shard", "kdkl_forward_finish",
-    "kdkl_wait_selftest",
+    "kdkl_wait_selftest", "kdkl_teacher_topk", "kdkl_teacher_topk_workspace_bytes",
 ]
 
 
@@ -81,6 +81,10 @@ def lib() -> ctypes.CDLL:
     L.kdkl_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, vp, vp]
     L.kdkl_logz_noalloc.restype = ctypes.c_int
     L.kdkl_logz_noalloc.argtypes = [vp, vp, i64, i64, i64, f32, vp, vp]
+    L.kdkl_teacher_topk_workspace_bytes.restype = sz
+    L.kdkl_teacher_topk_workspace_bytes.argtypes = [i64, i64, i64, i32]
+    L.kdkl_teacher_topk.restype = ctypes.c_int
+    L.kdkl_teacher_topk.argtypes = [vp, vp, i64, i64, i64, i32, f32, vp, sz, vp, vp, vp, vp]
     L.kdkl_wait_selftest.restype = ctypes.c_int
     L.kdkl_wait_selftest.argtypes = [vp, i64, vp]
     L.kdkl_last_error.restype = ctypes.c_char_p
@@ -227,6 +231,21 @@ def kdkl_logz_noalloc(hidden, weight, logz_out, temperature=1.0) -> None:
     T, H = hidden.shape
     V = weight.shape[0]
     _check(lib().kdkl_logz_noalloc(_ptr(hidden), _ptr(weight), T, H, V, temperature, _ptr(logz_out), _stream()))
+
+
+def kdkl_teacher_topk(hidden, weight, K, temperature=1.0, workspace=None):
+    """The teacher cache record: (topk_idx int32 [T,K], topk_val fp32 [T,K] descending, lse fp32 [T], workspace)."""
+    T, H = hidden.shape
+    V = weight.shape[0]
+    if workspace is None:
+        workspace = torch.empty(lib().kdkl_teacher_topk_workspace_bytes(T, H, V, K), dtype=torch.uint8,
+                                device=hidden.device)
+    idx = torch.empty(T, K, dtype=torch.int32, device=hidden.device)
+    val = torch.empty(T, K, dtype=torch.float32, device=hidden.device)
+    lse = torch.empty(T, dtype=torch.float32, device=hidden.device)
+    _check(lib().kdkl_teacher_topk(_ptr(hidden), _ptr(weight), T, H, V, K, temperature, _ptr(workspace),
+                                   workspace.numel(), _ptr(idx), _ptr(val), _ptr(lse), _stream()))
+    return idx, val, lse, workspace
 
 
 def kdkl_wait_selftest(status, limit_ns: int) -> None:

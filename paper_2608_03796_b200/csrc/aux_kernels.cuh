@@ -367,6 +367,83 @@ splitk_fixup_kernel(const float* __restrict__ part, long long slab, int splits, 
   }
 }
 
+// ------------------------------------------------------------------------------------ teacher top-K
+// Descending bitonic sort of n (power of two) keys in shared memory by one warp; `idx` (optional) is
+// carried along and breaks ties by the smaller index.
+__device__ __forceinline__ void warp_bitonic_desc(float* key, int* idx, int n, int lane) {
+  for (int size = 2; size <= n; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int i = lane; i < (n >> 1); i += 32) {
+        const int lo = 2 * i - (i & (stride - 1));
+        const int hi = lo + stride;
+        const bool down = (lo & size) == 0;          // this block sorts descending
+        const float a = key[lo], b = key[hi];
+        bool a_first = a > b;                        // a belongs before b in descending order
+        if (a == b && idx != nullptr) a_first = idx[lo] < idx[hi];
+        if (a_first != down) {
+          key[lo] = b; key[hi] = a;
+          if (idx != nullptr) { const int t = idx[lo]; idx[lo] = idx[hi]; idx[hi] = t; }
+        }
+      }
+      __syncwarp();
+    }
+  }
+}
+
+// Sweep 1 -> threshold. One warp (block) per row. From the per-vocab-tile partials of the log-sum-exp
+// sweep: the row's log-sum-exp, and the K-th largest tile maximum. At least K logits reach that value
+// (the K tile maxima themselves), so every member of the exact top-K does: it is a safe threshold.
+__global__ void __launch_bounds__(32)
+topk_threshold_kernel(const float* __restrict__ part_m, const float* __restrict__ part_s, long long part_stride,
+                      int n_tiles, int npad, int K, float* __restrict__ thr, int* __restrict__ cand_cnt,
+                      float* __restrict__ lse_out) {
+  extern __shared__ float tk_smem[];
+  const int row = blockIdx.x, lane = threadIdx.x;
+  float m = -INFINITY;
+  for (int i = lane; i < npad; i += 32) {
+    const float v = i < n_tiles ? part_m[(long long)i * part_stride + row] : -INFINITY;
+    tk_smem[i] = v;
+    m = fmaxf(m, v);
+  }
+  m = warp_max(m);
+  float s = 0.f;
+  for (int i = lane; i < n_tiles; i += 32) s += part_s[(long long)i * part_stride + row] * exp2f(tk_smem[i] - m);
+  s = warp_sum(s);
+  __syncwarp();
+  warp_bitonic_desc(tk_smem, nullptr, npad, lane);
+  if (lane == 0) {
+    thr[row] = n_tiles >= K ? tk_smem[K - 1] : -INFINITY;
+    cand_cnt[row] = 0;
+    lse_out[row] = (m + log2f(s)) * kLn2;
+  }
+}
+
+// Sweep 2 -> record. One warp (block) per row: sort the emitted candidates by (logit descending, index
+// ascending) and keep the first K. More candidates than the list holds is reported, not hidden.
+__global__ void __launch_bounds__(32)
+topk_select_kernel(const int* __restrict__ cand_cnt, const int* __restrict__ cand_idx,
+                   const float* __restrict__ cand_val, int cap, int cpad, int K, int* __restrict__ out_idx,
+                   float* __restrict__ out_val, long long row0, int* status) {
+  extern __shared__ float tk_smem[];
+  int* sidx = reinterpret_cast<int*>(tk_smem + cpad);
+  const int row = blockIdx.x, lane = threadIdx.x;
+  int n = cand_cnt[row];
+  if (n > cap) {
+    if (lane == 0) { atomicCAS(status, 0, -12); atomicCAS(status + 1, 0, (int)(row0 + row)); }
+    n = cap;
+  }
+  for (int i = lane; i < cpad; i += 32) {
+    tk_smem[i] = i < n ? cand_val[(long long)row * cap + i] : -INFINITY;
+    sidx[i] = i < n ? cand_idx[(long long)row * cap + i] : 0x7fffffff;
+  }
+  __syncwarp();
+  warp_bitonic_desc(tk_smem, sidx, cpad, lane);
+  for (int k = lane; k < K; k += 32) {
+    out_idx[(row0 + row) * K + k] = k < n ? sidx[k] : -1;
+    out_val[(row0 + row) * K + k] = k < n ? tk_smem[k] : -INFINITY;
+  }
+}
+
 // ------------------------------------------------------------------------------------ wait self-test
 // One thread waits on an mbarrier that nothing will ever complete, with a short limit. The wait must
 // give up, record KDKL_ERR_TIMEOUT and the site in status[0..1], and the kernel must return normally.

@@ -21,6 +21,7 @@
 //                   forward passes 1 and 2 in one sweep; Eq. "decomp")
 //   EPI_DLOGITS     backward: G = a_t * exp(z/tau - logZ) - b_t * p at the support, cast to
 //                   bf16 (Eq. "grad", Algorithm 1 backward)
+//   EPI_TOPK        teacher cache: emits the (column, logit) pairs above a per-row threshold
 #pragma once
 #include <cuda_bf16.h>
 
@@ -50,7 +51,7 @@ struct GemmCfg {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-enum { EPI_STORE_F32 = 0, EPI_STORE_BF16 = 1, EPI_LSE = 2, EPI_DLOGITS = 3 };
+enum { EPI_STORE_F32 = 0, EPI_STORE_BF16 = 1, EPI_LSE = 2, EPI_DLOGITS = 3, EPI_TOPK = 4 };
 
 struct GemmParams {
   int M, N, K;               // valid extents of this launch
@@ -78,6 +79,12 @@ struct GemmParams {
   const float* coefA;        // [rows] g_t * M_t / tau
   const float* coefB;        // [rows] g_t / tau
   const float* p_sorted;     // [rows, Ktop]
+  // EPI_TOPK: every logit with z * scale_log2 >= thr[row] is appended to the row's candidate list
+  const float* thr;          // [rows] threshold in the scaled (log2) domain
+  int* cand_cnt;             // [rows] running count (may exceed cand_cap: overflow is detected later)
+  int* cand_idx;             // [rows, cand_cap]
+  float* cand_val;           // [rows, cand_cap] raw logits
+  int cand_cap;
 };
 
 __device__ __forceinline__ int lower_bound_i32(const int* a, int n, int key) {
@@ -149,7 +156,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     mbar_fence_init();
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
-    if (EPI != EPI_LSE) tma_prefetch_desc(&tmC);
+    if (EPI != EPI_LSE && EPI != EPI_TOPK) tma_prefetch_desc(&tmC);
   }
   if (warp == 1) {
     if (NCTA == 2) { tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS); tmem_relinquish_pair(); }
@@ -293,7 +300,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       // per-row state that does not need the accumulator: fetched before the wait
       int cur = 0, nv = 0, next_idx = 0x7fffffff;
       const int* idxrow = nullptr;
-      float row_b = 0.f, row_off = -INFINITY;
+      float row_b = 0.f, row_off = -INFINITY, row_thr = INFINITY;
+      if (EPI == EPI_TOPK) { if (row_ok) row_thr = p.thr[row]; }
       if (EPI == EPI_LSE || EPI == EPI_DLOGITS) {
         if (row_ok) {
           idxrow = p.idx_sorted + (long long)row * p.Ktop;
@@ -353,6 +361,25 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int j = 0; j < 32; ++j) acc_s += ex2_approx(fmaf(__uint_as_float(r[j]), p.scale_log2, -m_new));
             s_run = s_run * ex2_approx(m_run - m_new) + acc_s;
             m_run = m_new;
+          }
+        } else if (EPI == EPI_TOPK) {
+          if (row_ok) {
+            // candidates of this window: a bit per column whose scaled logit reaches the row's threshold
+            uint32_t hits = 0u;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const bool in = (full_w || col0 + j < p.N) && (__uint_as_float(r[j]) * p.scale_log2 >= row_thr);
+              hits |= (in ? 1u : 0u) << j;
+            }
+            while (hits) {
+              const int j = __ffs(hits) - 1;
+              hits &= hits - 1u;
+              const int slot = atomicAdd(p.cand_cnt + row, 1);     // tiles of one row run on different SMs
+              if (slot < p.cand_cap) {
+                p.cand_idx[(long long)row * p.cand_cap + slot] = col0 + j;
+                p.cand_val[(long long)row * p.cand_cap + slot] = sel32(r, j);
+              }
+            }
           }
         } else {
           // Output path: the warp's 32 rows x 128 bytes go to a swizzled shared-memory box (16-byte
@@ -428,7 +455,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       }
     }
-    if (EPI != EPI_LSE && lane == 0) bulk_wait_all();   // every output box has been written
+    if (EPI != EPI_LSE && EPI != EPI_TOPK && lane == 0) bulk_wait_all();   // every output box has been written
   }
 
   // ---------------------------------------------------------------- teardown

@@ -604,6 +604,96 @@ int kdkl_profile_stages(const void* hidden, const void* weight, const int32_t* t
   return rc;
 }
 
+// ------------------------------------------------------------------ teacher top-K cache record
+constexpr long long kTopkTakeAllMaxV = 8192;
+struct TopkLayout { long long C, Cpad, n_tiles; int npad, cap, cpad; size_t hdr, zeros, part_m, part_s, thr, cnt, cidx, cval, total; };
+static int pow2_at_least(long long x) { int p = 32; while (p < x) p <<= 1; return p; }
+static TopkLayout topk_layout(long long T, long long V, int K) {
+  TopkLayout L;
+  L.C = T < 4096 ? T : 4096;
+  L.Cpad = (long long)up((size_t)L.C, 128);
+  L.n_tiles = (V + BN - 1) / BN;
+  L.npad = pow2_at_least(L.n_tiles);
+  // With at least K vocabulary tiles the threshold admits few more than K logits; with fewer tiles
+  // it says nothing, and every logit is a candidate (small vocabularies only: see kTopkTakeAllMaxV).
+  long long cap = 4ll * K > 256 ? 4ll * K : 256;
+  if (cap > 1024) cap = 1024;
+  if (L.n_tiles < K) cap = V;
+  if (cap > V) cap = V;
+  L.cap = (int)cap;
+  L.cpad = pow2_at_least(L.cap);
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = up(o + bytes, 256); return at; };
+  L.hdr = take(256);
+  L.zeros = take((size_t)L.Cpad * 4);
+  L.part_m = take((size_t)L.n_tiles * L.Cpad * 4);
+  L.part_s = take((size_t)L.n_tiles * L.Cpad * 4);
+  L.thr = take((size_t)L.Cpad * 4);
+  L.cnt = take((size_t)L.Cpad * 4);
+  L.cidx = take((size_t)L.Cpad * L.cap * 4);
+  L.cval = take((size_t)L.Cpad * L.cap * 4);
+  L.total = o;
+  return L;
+}
+
+size_t kdkl_teacher_topk_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K) {
+  if (T < 1 || H < 1 || V < 1 || K < 1) return 0;
+  return topk_layout(T, V, K).total;
+}
+
+int kdkl_teacher_topk(const void* hidden, const void* weight, int64_t T, int64_t H, int64_t V, int32_t K, float tau,
+                      void* ws, size_t ws_bytes, int32_t* topk_idx, float* topk_val, float* lse, void* cuda_stream) {
+  g_launches = 0;
+  if (!hidden || !weight || !ws || !topk_idx || !topk_val || !lse) return KDKL_ERR_NULL;
+  if (T < 1 || H < 1 || V < 1 || K < 1 || K > 256 || K > V || (H % 8) != 0 || V > (1ll << 20) || T >= (1ll << 31))
+    return KDKL_ERR_SHAPE;
+  if ((V + BN - 1) / BN < K && V > kTopkTakeAllMaxV) return KDKL_ERR_SHAPE;   // needs V >= 256 K or V <= 8192
+  if (!(tau > 0.f)) return KDKL_ERR_ARG;
+  if (((uintptr_t)hidden & 15) || ((uintptr_t)weight & 15) || ((uintptr_t)ws & 15)) return KDKL_ERR_ALIGN;
+  const TopkLayout L = topk_layout(T, V, K);
+  if (ws_bytes < L.total) return KDKL_ERR_WORKSPACE;
+  DeviceInfo di;
+  int rc = device_info(&di);
+  if (rc) return rc;
+  if (di.cc_major != 10) return KDKL_ERR_ARCH;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  int* status = at<int>(ws, L.hdr);
+  KDKL_CUDA(cudaMemsetAsync(at<uint8_t>(ws, L.hdr), 0, L.zeros + (size_t)L.Cpad * 4 - L.hdr, st));   // header + zero counts
+
+  CUtensorMap tmW;
+  if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, kBRows))) return rc;
+  for (long long s0 = 0; s0 < T; s0 += L.C) {
+    const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
+    CUtensorMap tmA;
+    const __nv_bfloat16* hA = reinterpret_cast<const __nv_bfloat16*>(hidden) + s0 * H;
+    if ((rc = make_tmap_bf16(&tmA, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, BK, BM))) return rc;
+    GemmParams p;
+    memset(&p, 0, sizeof(p));
+    p.M = (int)rows; p.N = (int)V; p.K = (int)H;
+    p.m_tiles = (int)((rows + kTileM - 1) / kTileM); p.n_tiles = (int)L.n_tiles; p.m_inner = 1; p.k_splits = 1;
+    p.status = status;
+    p.scale_log2 = kLog2e / tau; p.Ktop = 1;
+    p.nvalid = at<int>(ws, L.zeros); p.idx_sorted = at<int>(ws, L.zeros);     // no teacher entries to gather
+    p.part_m = at<float>(ws, L.part_m); p.part_s = at<float>(ws, L.part_s); p.part_stride = L.Cpad;
+    // sweep 1: per-tile maxima and sum-exp
+    if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA, p, di.sm_count, st))) return rc;
+    topk_threshold_kernel<<<(unsigned)rows, 32, (size_t)L.npad * 4, st>>>(
+        at<float>(ws, L.part_m), at<float>(ws, L.part_s), L.Cpad, (int)L.n_tiles, L.npad, K, at<float>(ws, L.thr),
+        at<int>(ws, L.cnt), lse + s0);
+    KDKL_LAUNCHED("topk_threshold_kernel");
+    // sweep 2: recompute, emit everything at or above the row's threshold
+    p.thr = at<float>(ws, L.thr); p.cand_cnt = at<int>(ws, L.cnt);
+    p.cand_idx = at<int>(ws, L.cidx); p.cand_val = at<float>(ws, L.cval); p.cand_cap = L.cap;
+    if ((rc = launch_gemm<EPI_TOPK, false, false>(tmA, tmW, tmA, p, di.sm_count, st))) return rc;
+    KDKL_CUDA(cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.cpad * 8));
+    topk_select_kernel<<<(unsigned)rows, 32, (size_t)L.cpad * 8, st>>>(
+        at<int>(ws, L.cnt), at<int>(ws, L.cidx), at<float>(ws, L.cval), L.cap, L.cpad, K, topk_idx, topk_val, s0,
+        status);
+    KDKL_LAUNCHED("topk_select_kernel");
+  }
+  return KDKL_OK;
+}
+
 // ------------------------------------------------------------------ bounded-wait self-test
 int kdkl_wait_selftest(int32_t* status, int64_t limit_ns, void* cuda_stream) {
   if (!status) return KDKL_ERR_NULL;

@@ -1,0 +1,93 @@
+"""GPU parity of the teacher top-K cache kernel against its dense fp64 oracle.
+
+The selection is decided by fp32 logits on the GPU and fp64 logits in the oracle, so two entries whose
+logits differ by less than the fp32 accumulation error may swap places or membership at the K-th
+boundary. What is unique is compared exactly (entries clearly above the boundary, sorted values,
+the log-sum-exp); the rest is checked for validity (every returned index is a genuine near-top entry).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle.kdkl_oracle import kdkl_oracle
+from oracle.teacher_oracle import teacher_topk_oracle
+from paper_2608_03796_b200 import binding as B
+
+pytestmark = pytest.mark.gpu
+EPS = 2e-4          # fp32 accumulation error bound on a logit of magnitude O(10)
+
+
+def _case(T, H, V, seed):
+    g = torch.Generator().manual_seed(seed)
+    h = torch.randn(T, H, generator=g).to(torch.bfloat16)
+    W = (torch.randn(V, H, generator=g) / H ** 0.5).to(torch.bfloat16)
+    return h, W
+
+
+def _check(h, W, K, tau):
+    dev = torch.device("cuda:0")
+    idx, val, lse, ws = B.kdkl_teacher_topk(h.to(dev), W.to(dev), K, temperature=tau)
+    code, _ = B.kdkl_status(ws)
+    assert code == 0
+    idx, val, lse = idx.cpu().numpy(), val.cpu().double().numpy(), lse.cpu().double().numpy()
+    o = teacher_topk_oracle(h.double().numpy(), W.double().numpy(), K, tau=tau)
+    np.testing.assert_allclose(lse, o["lse"], rtol=0, atol=2e-4)
+    T, V = o["z"].shape
+    assert idx.min() >= 0 and idx.max() < V
+    for t in range(T):
+        assert len(set(idx[t].tolist())) == K                             # K distinct entries
+        zt = o["z"][t]
+        np.testing.assert_allclose(val[t], zt[idx[t]], rtol=0, atol=EPS)   # values are the logits at those indices
+        assert np.all(np.diff(val[t]) <= 0)                                # sorted descending
+        kth = o["val"][t, -1]
+        assert np.all(zt[idx[t]] >= kth - EPS)                             # nothing below the boundary got in
+        sure = o["idx"][t][o["val"][t] > kth + EPS]                        # entries clearly above it must be there
+        assert set(sure.tolist()) <= set(idx[t].tolist())
+    exact = (idx == o["idx"]).mean()
+    assert exact > 0.98                                                    # position-exact except at near-ties
+    return idx, val, lse, o
+
+
+@pytest.mark.parametrize("T,H,V,K,tau", [(300, 264, 4120, 16, 1.0), (70, 64, 300, 100, 2.0), (5, 8, 9, 9, 1.0),
+                                         (1100, 128, 70000, 100, 1.0)])
+def test_teacher_topk_matches_oracle(T, H, V, K, tau):
+    h, W = _case(T, H, V, seed=T + V)
+    _check(h, W, K, tau)
+
+
+def test_ties_break_by_smaller_index_and_overflow_is_reported():
+    dev = torch.device("cuda:0")
+    T, H, V, K = 4, 64, 2048, 8
+    h, W = _case(T, H, V, seed=9)
+    W[100] = W[7]; W[1500] = W[7]                     # three identical vocabulary rows: exact ties
+    idx, val, lse, ws = B.kdkl_teacher_topk(h.to(dev), W.to(dev), 256, temperature=1.0)
+    assert B.kdkl_status(ws)[0] == 0
+    idx, val = idx.cpu().numpy(), val.cpu().numpy()
+    for t in range(T):
+        pos = {int(v): int(np.where(idx[t] == v)[0][0]) for v in (7, 100, 1500) if v in idx[t]}
+        if len(pos) == 3:
+            assert pos[7] < pos[100] < pos[1500] and val[t][pos[7]] == val[t][pos[1500]]
+    # a constant head: every logit ties, more candidates than the list can hold -> reported
+    Wc = torch.ones(4096, H).to(torch.bfloat16)       # 16 tiles >= K = 8: threshold path, list of 256
+    _, _, _, ws2 = B.kdkl_teacher_topk(h.to(dev), Wc.to(dev), 8, temperature=1.0)
+    assert B.kdkl_status(ws2)[0] == -12
+
+
+def test_cache_feeds_the_loss_with_exact_retained_mass():
+    """Teacher kernel -> cache record -> fused loss with teacher_lse: the paper's un-renormalised M < 1 path,
+    end to end on the GPU, against the oracles fed with their own (fp64) cache."""
+    dev = torch.device("cuda:0")
+    T, Ht, Hs, V, K, tau = 200, 96, 128, 3000, 20, 1.0
+    ht, Wt = _case(T, Ht, V, seed=41)
+    hs, Ws = _case(T, Hs, V, seed=42)
+    idx, val, lse, _ = B.kdkl_teacher_topk(ht.to(dev), Wt.to(dev), K, temperature=tau)
+    op = B.FusedChunkedKL(T, Hs, V, K, chunk=64, temperature=tau, device=dev)
+    op.forward(hs.to(dev), Ws.to(dev), idx, val, teacher_lse=lse)
+    op.backward(hs.to(dev), Ws.to(dev))
+    assert op.status()[0] == 0
+    ot = teacher_topk_oracle(ht.double().numpy(), Wt.double().numpy(), K, tau=tau)
+    o = kdkl_oracle(hs.double().numpy(), Ws.double().numpy(), ot["idx"], ot["val"], tau=tau, teacher_lse=ot["lse"])
+    assert o["M"].max() < 1.0
+    assert abs(op.loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
+    dW = op.dweight.cpu().double().numpy()
+    assert np.linalg.norm(dW - o["dW"]) / np.linalg.norm(o["dW"]) <= 1e-2
