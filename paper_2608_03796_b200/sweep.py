@@ -51,7 +51,15 @@ def worker(method: str, name: str, steps: int) -> dict:
     torch.cuda.reset_peak_memory_stats()
     out = {"method": method, "workload": name, "T": cfg.T, "H": cfg.H, "V": cfg.V, "K": cfg.K, "chunk": cfg.chunk,
            "input_gb": torch.cuda.memory_allocated() / 1e9}
-    if method == "fused":
+    if method == "teacher":
+        # the teacher cache kernel on the same shape: hidden / weight play the teacher's role
+        _, _, _, tws = B.kdkl_teacher_topk(d["hidden"], d["weight"], cfg.K, temperature=cfg.tau)
+        out["workspace_gb"] = tws.numel() / 1e9
+
+        def step():
+            B.kdkl_teacher_topk(d["hidden"], d["weight"], cfg.K, temperature=cfg.tau, workspace=tws)
+            return torch.zeros(1)
+    elif method == "fused":
         op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev)
 
         def step():
@@ -89,7 +97,8 @@ def worker(method: str, name: str, steps: int) -> dict:
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / steps
         out.update(ms_per_iter=ms, it_per_s=1e3 / ms, tokens_per_s=cfg.T / (ms * 1e-3),
-                   tflops=cfg.flops / (ms * 1e-3) / 1e12, loss=float(loss.item()),
+                   tflops=(0.5 if method == "teacher" else 1.0) * cfg.flops / (ms * 1e-3) / 1e12,   # teacher: 2 sweeps
+                   loss=float(loss.item()),
                    peak_gb=torch.cuda.max_memory_allocated() / 1e9)
         if method == "fused":
             code, _ = op.status()
