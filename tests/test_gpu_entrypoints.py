@@ -1,0 +1,55 @@
+"""The host-buffer end-to-end entry point and the per-stage profiling entry point against the plain calls."""
+import pytest
+import torch
+
+from paper_2608_03796_b200 import binding as B
+from paper_2608_03796_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+def _device_run(cfg, d, dev, opt=None):
+    g = {k: (v.to(dev) if v is not None else None) for k, v in d.items()}
+    op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev, opt=opt)
+    op.forward(g["hidden"], g["weight"], g["topk_idx"], g["topk_val"], loss_mask=g["mask"])
+    op.backward(g["hidden"], g["weight"], loss_mask=g["mask"])
+    assert op.status()[0] == 0
+    return g, op
+
+
+def test_host_buffer_call_equals_device_calls_bitwise():
+    cfg = I.CONFIGS["c1"]
+    d = I.make_inputs(cfg)
+    dev = torch.device("cuda:0")
+    _, op = _device_run(cfg, d, dev)
+    arena = torch.empty(B.kdkl_host_arena_bytes(cfg.T, cfg.H, cfg.V, cfg.K, cfg.chunk), dtype=torch.uint8, device=dev)
+    loss_h = torch.zeros(1).pin_memory()
+    dh_h = torch.empty(cfg.T, cfg.H, dtype=torch.bfloat16).pin_memory()
+    dw_h = torch.empty(cfg.V, cfg.H, dtype=torch.float32).pin_memory()
+    hh = {k: (v.pin_memory() if v is not None else None) for k, v in d.items()}
+    B.kdkl_forward_backward_host(hh["hidden"], hh["weight"], hh["topk_idx"], hh["topk_val"], arena, loss_h, dh_h, dw_h,
+                                 chunk=cfg.chunk, temperature=cfg.tau)
+    assert loss_h.item() == op.loss.item()
+    assert torch.equal(dh_h, op.dhidden.cpu()) and torch.equal(dw_h, op.dweight.cpu())
+    assert B.kdkl_last_launch_count() == op.launches
+    # too small an arena is refused before anything is copied
+    with pytest.raises(B.KdklError) as e:
+        B.kdkl_forward_backward_host(hh["hidden"], hh["weight"], hh["topk_idx"], hh["topk_val"], arena[:4096], loss_h,
+                                     dh_h, dw_h, chunk=cfg.chunk, temperature=cfg.tau)
+    assert e.value.code == -4
+
+
+def test_profile_stages_accounts_for_every_launch_and_changes_nothing():
+    cfg = I.CONFIGS["c1"]
+    d = I.make_inputs(cfg)
+    dev = torch.device("cuda:0")
+    g, op = _device_run(cfg, d, dev)
+    ref_loss, ref_dw = op.loss.clone(), op.dweight.clone()
+    st = B.kdkl_profile_stages(g["hidden"], g["weight"], g["topk_idx"], g["topk_val"], op.workspace, op.loss, op.dhidden,
+                               op.dweight, chunk=cfg.chunk, temperature=cfg.tau)
+    chunks = cfg.T // cfg.chunk
+    assert st["fwd_gemm_lse"][1] == chunks and st["bwd_gemm_dlogits"][1] == chunks
+    assert st["dhidden_gemm"][1] == chunks and st["dweight_gemm"][1] == chunks and st["combine"][1] == chunks
+    assert st["prep"][1] == 1 and st["loss_reduce"][1] == 1 and st["bwd_coef"][1] == 1
+    assert all(ms > 0 for ms, n in st.values())
+    assert torch.equal(op.loss, ref_loss) and torch.equal(op.dweight, ref_dw)
