@@ -111,3 +111,19 @@ def test_fullsize_sampled_parity(name, n_rows, partial_mass):
         recon = (nR * sub_dW.double() + (n_counted - nR) * rest.dweight.double()) / n_counted
         err = (recon - full_dW.double()).norm() / full_dW.double().norm()
         assert err.item() < 3e-3      # two independent bf16 roundings of G against one
+
+
+def test_fullsize_runs_are_bitwise_reproducible():
+    """No floating-point atomics on any result path: two runs of the benchmark shape agree bit for bit
+    (this also serves as a race detector for the CTA-pair kernels), at 1 chunk and at 8 chunks."""
+    dev = torch.device("cuda:0")
+    for name, T in (("c2", 4096), ("c3", 32768)):
+        cfg = I.CONFIGS[name]
+        d = I.make_inputs(cfg, device=dev)
+        a = _run(cfg, d, None, want_tok=True)
+        la, dha, dwa, ta = a.loss.clone(), a.dhidden.clone(), a.dweight.clone(), a.loss_per_token.clone()
+        del a
+        b = _run(cfg, d, None, want_tok=True)
+        assert torch.equal(la, b.loss) and torch.equal(ta, b.loss_per_token)
+        assert torch.equal(dha, b.dhidden) and torch.equal(dwa, b.dweight)
+        del b, d
