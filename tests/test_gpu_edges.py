@@ -65,3 +65,23 @@ def test_bounded_wait_expires_and_context_survives():
     assert op.status()[0] == 0
     o = kdkl_oracle(h.double().numpy(), W.double().numpy(), idx.numpy(), val.numpy(), want_grads=False)
     assert abs(op.loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
+
+
+def test_large_logits_and_small_temperature():
+    """Logits of standard deviation ~12 after the temperature (softmax close to one-hot on many rows):
+    the online max / sum-exp must neither overflow nor lose the loss to cancellation."""
+    dev = torch.device("cuda:0")
+    T, H, V, K, tau = 200, 128, 5000, 12, 0.5
+    h, W, idx, val = _case(T, H, V, K, seed=77)
+    h = (h.float() * 6).to(torch.bfloat16)
+    val = val * 4
+    op = B.FusedChunkedKL(T, H, V, K, chunk=64, temperature=tau, device=dev, want_per_token=True)
+    op.forward(h.to(dev), W.to(dev), idx.to(dev), val.to(dev))
+    op.backward(h.to(dev), W.to(dev))
+    assert op.status()[0] == 0
+    o = kdkl_oracle(h.double().numpy(), W.double().numpy(), idx.numpy(), val.numpy(), tau=tau)
+    assert o["logZ"].max() > 30
+    assert abs(op.loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
+    np.testing.assert_allclose(op.loss_per_token.cpu().double().numpy(), o["loss_tok"], rtol=1e-4, atol=1e-3)
+    assert _fro(op.dhidden.float().cpu().double().numpy(), o["dH"]) <= 1e-2
+    assert _fro(op.dweight.cpu().double().numpy(), o["dW"]) <= 1e-2
