@@ -359,3 +359,51 @@ class ShardedFusedChunkedKL:
 
     def status(self):
         return kdkl_status(self.workspace)
+
+
+class TokenShardedFusedKL:
+    """One rank of the token-sharded (data-parallel) loss: this rank holds T_local tokens and the whole head.
+
+    Rows are independent given the weight, so the only exchanges are three sums over ranks: the number of
+    counted tokens (before forward: it is the divisor of the mean), the loss, and the fp32 dweight.
+    dhidden needs no communication. ``all_reduce_sum(tensor)`` defaults to torch.distributed (NCCL).
+    """
+
+    def __init__(self, T_local, H, V, K, chunk=0, temperature=1.0, device="cuda", all_reduce_sum=None):
+        self.T, self.H, self.V, self.K = T_local, H, V, K
+        self.chunk, self.temperature, self.device = chunk, temperature, device
+        self.workspace = torch.empty(kdkl_workspace_bytes(T_local, H, V, K, chunk), dtype=torch.uint8, device=device)
+        self.loss = torch.zeros(1, dtype=torch.float32, device=device)
+        self.dhidden = torch.empty(T_local, H, dtype=torch.bfloat16, device=device)
+        self.dweight = torch.empty(V, H, dtype=torch.float32, device=device)
+        self._all_reduce_sum = all_reduce_sum or ShardedFusedChunkedKL._dist_all_reduce
+        self.opt = None
+
+    def count_tokens(self, loss_mask=None):
+        """Global number of counted tokens (one small all-reduce and a host read)."""
+        n = torch.tensor([float(self.T if loss_mask is None else int(loss_mask.sum().item()))], device=self.device)
+        self._all_reduce_sum(n)
+        return float(n.item())
+
+    def forward_local(self, hidden, weight, topk_idx, topk_val, n_global, teacher_lse=None, loss_mask=None):
+        self.opt = make_options(denom_override=n_global)      # every rank divides by the global count
+        kdkl_forward(hidden, weight, topk_idx, topk_val, self.workspace, self.loss, teacher_lse=teacher_lse,
+                     loss_mask=loss_mask, chunk=self.chunk, temperature=self.temperature, opt=self.opt)
+
+    def forward(self, hidden, weight, topk_idx, topk_val, teacher_lse=None, loss_mask=None):
+        n_global = self.count_tokens(loss_mask)
+        self.forward_local(hidden, weight, topk_idx, topk_val, n_global, teacher_lse, loss_mask)
+        self._all_reduce_sum(self.loss)                        # partial means add up to the global mean
+        return self.loss
+
+    def backward_local(self, hidden, weight, loss_mask=None, grad_loss=1.0):
+        kdkl_backward(hidden, weight, self.K, self.workspace, self.dhidden, self.dweight, loss_mask=loss_mask,
+                      chunk=self.chunk, temperature=self.temperature, opt=self.opt, grad_loss=grad_loss)
+
+    def backward(self, hidden, weight, loss_mask=None, grad_loss=1.0):
+        self.backward_local(hidden, weight, loss_mask, grad_loss)
+        self._all_reduce_sum(self.dweight)                     # the data-parallel gradient reduction
+        return self.dhidden, self.dweight
+
+    def status(self):
+        return kdkl_status(self.workspace)

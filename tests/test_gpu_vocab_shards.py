@@ -84,3 +84,35 @@ def test_sharded_c1_two_halves_equals_unsharded_loss():
     # dW slices are computed from the same G values: only the rounding of log Z can differ
     assert _fro(dW.cpu().double().numpy(), full.dweight.cpu().double().numpy()) < 2e-3
     assert _fro(dH.cpu().double().numpy(), full.dhidden.cpu().double().numpy()) < 2e-3
+
+
+def test_token_shards_match_oracle():
+    """Data-parallel form: uneven token slices, the global denominator on every rank, dW and loss summed."""
+    T, H, V, K, tau = 300, 136, 2100, 7, 1.0
+    g = torch.Generator().manual_seed(51)
+    d = {"hidden": torch.randn(T, H, generator=g).to(torch.bfloat16),
+         "weight": (torch.randn(V, H, generator=g) / H ** 0.5).to(torch.bfloat16),
+         "topk_idx": torch.stack([torch.randperm(V, generator=g)[:K] for _ in range(T)]).to(torch.int32),
+         "topk_val": (torch.randn(T, K, generator=g) * 3 ** 0.5).float(),
+         "mask": (torch.rand(T, generator=g) >= 0.2).to(torch.uint8)}
+    dev = torch.device("cuda:0")
+    gd = {k: v.to(dev) for k, v in d.items()}
+    bounds = [0, 77, 200, T]
+    n_global = float(d["mask"].sum().item())
+    ranks = []
+    for r in range(3):
+        a, b = bounds[r], bounds[r + 1]
+        op = B.TokenShardedFusedKL(b - a, H, V, K, chunk=64, temperature=tau, device=dev, all_reduce_sum=lambda t: t)
+        sl = {k: (v[a:b].contiguous() if k != "weight" else v) for k, v in gd.items()}
+        op.forward_local(sl["hidden"], sl["weight"], sl["topk_idx"], sl["topk_val"], n_global, loss_mask=sl["mask"])
+        op.backward_local(sl["hidden"], sl["weight"], loss_mask=sl["mask"])
+        assert op.status()[0] == 0
+        ranks.append(op)
+    loss = sum(op.loss.item() for op in ranks)                       # what the all-reduces deliver
+    dW = sum(op.dweight for op in ranks)
+    dH = torch.cat([op.dhidden for op in ranks], 0)
+    o = kdkl_oracle(d["hidden"].double().numpy(), d["weight"].double().numpy(), d["topk_idx"].numpy(),
+                    d["topk_val"].numpy(), tau=tau, mask=d["mask"].numpy())
+    assert abs(loss - o["loss"]) <= 1e-3 * abs(o["loss"])
+    assert _fro(dW.cpu().double().numpy(), o["dW"]) <= 1e-2
+    assert _fro(dH.float().cpu().double().numpy(), o["dH"]) <= 1e-2
