@@ -77,3 +77,18 @@ def test_host_side_argument_checks_without_a_gpu():
     assert L.kdkl_gemm_bf16(P, P, P, 64, 64, 60, 0, 0, None, None) == -2
     assert L.kdkl_wait_selftest(P, 0, None) == -5
     assert L.kdkl_logz_noalloc(P, P, 8, 64, 262144 + 256, 1.0, P, None) == -4
+
+
+def test_header_is_plain_c99(tmp_path):
+    """The boundary is a C ABI: the header must compile as C, with no C++ or torch types."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        import pytest
+        pytest.skip("no gcc")
+    src = tmp_path / "use.c"
+    src.write_text('#include "kdkl.h"\nint main(void) { kdkl_options o; o.struct_size = (int32_t)sizeof(o); '
+                   'return kdkl_workspace_bytes(1, 8, 8, 1, 0, &o) == 0; }\n')
+    subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only",
+                    "-I", os.path.join(ROOT, "include"), str(src)], check=True)
