@@ -331,6 +331,33 @@ def main():
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
         del arena
 
+    # the HBM-bound companion op (hidden-state feature loss, one pass: 2 reads + 1 write of [T,H] bf16), timed at
+    # 32768 tokens so that its 6*T*H bytes are several times the L2 whatever T the main workload has
+    feature = None
+    if rank == 0:
+        fT = 32768
+        fcfg = I.Config("feature", T=fT, H=H, V=V, K=K, chunk=cfg.chunk)
+        fs, fr = I.hidden(fcfg, device=dev), I.teacher_hidden(fcfg, device=dev)
+        fws = torch.empty(B.kdkl_feature_loss_workspace_bytes(fT), dtype=torch.uint8, device=dev)
+        fl, fd = torch.zeros(1, device=dev), torch.empty_like(fs)
+        feature = {"T": fT, "H": H, "algorithmic_bytes": 6 * fT * H,
+                   "hbm_peak_GBps": float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))}
+        for kind, kname in ((B.FEATURE_MSE, "mse"), (B.FEATURE_COSINE, "cosine")):
+            for _ in range(3):
+                B.kdkl_feature_loss(fs, fr, fws, fl, kind=kind, dstudent=fd)
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            f0.record()
+            f_iters = 2 if args.capture else 20
+            for _ in range(f_iters):
+                B.kdkl_feature_loss(fs, fr, fws, fl, kind=kind, dstudent=fd)
+            f1.record()
+            torch.cuda.synchronize()
+            f_ms = f0.elapsed_time(f1) / f_iters
+            gbps = 6 * fT * H / (f_ms * 1e-3) / 1e9
+            feature[kname] = {"ms": f_ms, "GBps": gbps, "frac_of_hbm_copy": gbps / feature["hbm_peak_GBps"],
+                              "loss": float(fl.item())}
+        del fs, fr, fd, fws
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -366,6 +393,7 @@ def main():
                      "traffic": traffic, "ms_per_launch": stages[dom]["ms_per_launch"],
                      "flops_per_launch": flops_per_launch},
         "stages": stages,
+        "feature_loss": feature,
         "cpu_baseline": cpu_baseline,
     }
     print(json.dumps(line), flush=True)

@@ -208,6 +208,32 @@ int kdkl_teacher_topk(const void* hidden_bf16, const void* weight_bf16, int64_t 
                       float temperature, void* workspace, size_t workspace_bytes, int32_t* topk_idx,
                       float* topk_val, float* lse, void* cuda_stream);
 
+#define KDKL_FEATURE_MSE 0
+#define KDKL_FEATURE_COSINE 1
+
+/* Hidden-state feature loss that the paper recommends adding to the logit KL (section "Additional
+ * Ablations", paragraph "Loss design": a mean-squared-error variant and a cosine variant; no formula is
+ * printed, these are the textbook ones). Per token t, student row s and teacher row r of width H:
+ *   KDKL_FEATURE_MSE     f_t = (1/H) sum_h (s_h - r_h)^2
+ *   KDKL_FEATURE_COSINE  f_t = 1 - <s,r> / (|s| |r|)        (f_t = 1, zero gradient, when |s||r| <= 1e-12)
+ *   loss = weight * sum_t mask_t f_t / N,  N = number of mask = 1 tokens (denom_override > 0 replaces it;
+ *   N = 0 gives loss 0 and zero gradients), reduced in a fixed order (bitwise reproducible).
+ * Loss and gradient come out of one pass over the inputs (the op is bound by memory traffic):
+ *   dstudent_bf16 [T, H] or NULL = loss only: grad_loss * d loss / d student, rounded once to bf16;
+ *     accumulate = 0 overwrites it (ignored tokens' rows are set to zero), accumulate = 1 adds to what it
+ *     holds, e.g. the dHidden that kdkl_backward wrote for the same hidden states (ignored rows untouched).
+ *   student_bf16, teacher_bf16 [T, H]: device, row-major, 16-byte aligned, H % 8 == 0; rows of ignored
+ *     tokens are never read. loss_mask [T] u8 or NULL = all counted. loss_out [1], loss_per_token [T] or
+ *     NULL (f_t, 0 on ignored tokens): device fp32. Must not alias one another.
+ *   workspace: device, 16-byte aligned, kdkl_feature_loss_workspace_bytes(T). Enqueue-only, two kernels (three with a mask).
+ * Returns KDKL_OK or KDKL_ERR_NULL / _SHAPE / _ARG (unknown kind, non-finite weight or grad_loss,
+ * accumulate not 0/1) / _ALIGN / _WORKSPACE / _ARCH / _CUDA. */
+size_t kdkl_feature_loss_workspace_bytes(int64_t T);
+int kdkl_feature_loss(const void* student_bf16, const void* teacher_bf16, const uint8_t* loss_mask, int64_t T,
+                      int64_t H, int32_t kind, float weight, float grad_loss, float denom_override,
+                      int32_t accumulate, void* workspace, size_t workspace_bytes, float* loss_out,
+                      float* loss_per_token, void* dstudent_bf16, void* cuda_stream);
+
 /* Exercises the bounded wait every kernel of this library uses on its mbarriers: one thread waits on
  * a barrier that nothing completes, gives up after limit_ns (1 .. 1e9) and the kernel returns normally.
  * status: device int32[2], zeroed by the caller; afterwards {KDKL_ERR_TIMEOUT, 99}. The context stays

@@ -27,7 +27,10 @@ EXPORTS = [
     "kdkl_host_arena_bytes", "kdkl_forward_backward_host", "kdkl_profile_stages", "kdkl_gemm_bf16", "kdkl_last_error",
     "kdkl_last_launch_count", "kdkl_logz_noalloc", "kdkl_forward_shard", "kdkl_forward_finish",
     "kdkl_wait_selftest", "kdkl_teacher_topk", "kdkl_teacher_topk_workspace_bytes",
+    "kdkl_feature_loss", "kdkl_feature_loss_workspace_bytes",
 ]
+
+FEATURE_MSE, FEATURE_COSINE = 0, 1
 
 
 class KdklError(RuntimeError):
@@ -85,6 +88,10 @@ def lib() -> ctypes.CDLL:
     L.kdkl_teacher_topk_workspace_bytes.argtypes = [i64, i64, i64, i32]
     L.kdkl_teacher_topk.restype = ctypes.c_int
     L.kdkl_teacher_topk.argtypes = [vp, vp, i64, i64, i64, i32, f32, vp, sz, vp, vp, vp, vp]
+    L.kdkl_feature_loss_workspace_bytes.restype = sz
+    L.kdkl_feature_loss_workspace_bytes.argtypes = [i64]
+    L.kdkl_feature_loss.restype = ctypes.c_int
+    L.kdkl_feature_loss.argtypes = [vp, vp, vp, i64, i64, i32, f32, f32, f32, i32, vp, sz, vp, vp, vp, vp]
     L.kdkl_wait_selftest.restype = ctypes.c_int
     L.kdkl_wait_selftest.argtypes = [vp, i64, vp]
     L.kdkl_last_error.restype = ctypes.c_char_p
@@ -246,6 +253,19 @@ def kdkl_teacher_topk(hidden, weight, K, temperature=1.0, workspace=None):
     _check(lib().kdkl_teacher_topk(_ptr(hidden), _ptr(weight), T, H, V, K, temperature, _ptr(workspace),
                                    workspace.numel(), _ptr(idx), _ptr(val), _ptr(lse), _stream()))
     return idx, val, lse, workspace
+
+
+def kdkl_feature_loss_workspace_bytes(T) -> int:
+    return lib().kdkl_feature_loss_workspace_bytes(T)
+
+
+def kdkl_feature_loss(student, teacher, workspace, loss_out, *, kind=FEATURE_MSE, loss_mask=None, weight=1.0,
+                      grad_loss=1.0, denom_override=0.0, accumulate=0, loss_per_token=None, dstudent=None) -> None:
+    """Hidden-state feature loss (MSE or cosine) and its gradient in one pass; see include/kdkl.h."""
+    T, H = student.shape
+    _check(lib().kdkl_feature_loss(_ptr(student), _ptr(teacher), _ptr(loss_mask), T, H, kind, weight, grad_loss,
+                                   denom_override, accumulate, _ptr(workspace), workspace.numel(), _ptr(loss_out),
+                                   _ptr(loss_per_token), _ptr(dstudent), _stream()))
 
 
 def kdkl_wait_selftest(status, limit_ns: int) -> None:

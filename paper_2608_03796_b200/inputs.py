@@ -25,7 +25,7 @@ from typing import Optional
 import torch
 
 # stream ids
-S_HIDDEN, S_WEIGHT, S_TIDX, S_TVAL, S_TOFF, S_DOC, S_MASS, S_ROWS = 1, 2, 3, 4, 5, 6, 7, 8
+S_HIDDEN, S_WEIGHT, S_TIDX, S_TVAL, S_TOFF, S_DOC, S_MASS, S_ROWS, S_THID = 1, 2, 3, 4, 5, 6, 7, 8, 9
 
 _MASK64 = (1 << 64) - 1
 
@@ -133,6 +133,19 @@ def hidden(cfg: Config, rows: Optional[torch.Tensor] = None, device="cpu") -> to
     col = torch.arange(cfg.H, dtype=torch.int64, device=device)
     return _blocked(lambda rb: bf16_bits(normal(cfg.seed, S_HIDDEN, rb[:, None] * cfg.H + col[None, :])),
                     r, cfg.H)
+
+
+def teacher_hidden(cfg: Config, rows: Optional[torch.Tensor] = None, device="cpu") -> torch.Tensor:
+    """Cached teacher hidden states for the feature loss, bf16 [len(rows), H]: 0.8 x the student's
+    N(0,1) draw + 0.6 x an independent N(0,1) draw, i.e. unit variance and correlation 0.8 with the
+    student row (a student that already tracks its teacher, as in healing)."""
+    r = _rows(cfg.T, rows, device)
+    col = torch.arange(cfg.H, dtype=torch.int64, device=device)
+
+    def block(rb):
+        at = rb[:, None] * cfg.H + col[None, :]
+        return bf16_bits(0.8 * normal(cfg.seed, S_HIDDEN, at) + 0.6 * normal(cfg.seed, S_THID, at))
+    return _blocked(block, r, cfg.H)
 
 
 def weight(cfg: Config, rows: Optional[torch.Tensor] = None, device="cpu") -> torch.Tensor:

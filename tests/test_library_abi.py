@@ -77,6 +77,17 @@ def test_host_side_argument_checks_without_a_gpu():
     assert L.kdkl_gemm_bf16(P, P, P, 64, 64, 60, 0, 0, None, None) == -2
     assert L.kdkl_wait_selftest(P, 0, None) == -5
     assert L.kdkl_logz_noalloc(P, P, 8, 64, 262144 + 256, 1.0, P, None) == -4
+    # feature loss
+    fws = binding.kdkl_feature_loss_workspace_bytes(T)
+    assert fws >= 256 + 4 * T and fws % 16 == 0
+
+    def feat(s=P, r=P, T=T, H=H, kind=0, weight=1.0, acc=0, wsp=Q, wsb=fws, loss=P, dst=P):
+        return L.kdkl_feature_loss(s, r, None, T, H, kind, weight, 1.0, 0.0, acc, wsp, wsb, loss, None, dst, None)
+    assert feat(s=None) == -1 and feat(r=None) == -1 and feat(loss=None) == -1 and feat(wsp=None) == -1
+    assert feat(T=0) == -2 and feat(H=12) == -2
+    assert feat(kind=2) == -5 and feat(acc=3) == -5 and feat(weight=float("nan")) == -5
+    assert feat(s=P + 8) == -3 and feat(dst=P + 2) == -3
+    assert feat(wsb=fws - 1) == -4
 
 
 def test_header_is_plain_c99(tmp_path):
