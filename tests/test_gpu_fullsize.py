@@ -127,3 +127,24 @@ def test_fullsize_runs_are_bitwise_reproducible():
         assert torch.equal(la, b.loss) and torch.equal(ta, b.loss_per_token)
         assert torch.equal(dha, b.dhidden) and torch.equal(dwa, b.dweight)
         del b, d
+
+
+def test_rows_do_not_depend_on_sequence_length():
+    """The generators are prefix-consistent and tokens are independent given the head, so the first
+    4096 tokens of the 32K run must reproduce the 4K run's per-token loss and log Z bit for bit, and its
+    dHidden rows up to the 1/N factor (4096 vs 32768 counted tokens; the factor enters through an fp32
+    exponent offset, so single bf16 roundings may differ)."""
+    dev = torch.device("cuda:0")
+    c2, c3 = I.CONFIGS["c2"], I.CONFIGS["c3"]
+    d3 = I.make_inputs(c3, device=dev)
+    d2 = I.make_inputs(c2, device=dev)
+    assert torch.equal(d3["hidden"][:c2.T], d2["hidden"]) and torch.equal(d3["topk_idx"][:c2.T], d2["topk_idx"])
+    a = _run(c2, d2, None)
+    tok2, dh2 = a.loss_per_token.clone(), a.dhidden.clone()
+    lz2 = a.saved_state()[0].clone()
+    del a
+    b = _run(c3, d3, None)
+    assert torch.equal(b.loss_per_token[:c2.T], tok2)
+    assert torch.equal(b.saved_state()[0][:c2.T], lz2)
+    x, y = b.dhidden[:c2.T].double() * 8.0, dh2.double()
+    assert ((x - y).norm() / y.norm()).item() < 2e-3
