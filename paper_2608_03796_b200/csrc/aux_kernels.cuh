@@ -179,8 +179,11 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
 // adds the sparse terms and writes the per-token loss  L_t = Hent_t - C_t + M_t log Z_t
 // (Eq. "decomp"), with C_t = sum_k p_k z_k / tau from the gathered logits. Also un-permutes the
 // gathered logits / columns into the caller's slot order.
-// Block = 32 rows x 8 partial lanes; partial arrays are [n_tiles, part_stride] so reads coalesce.
-__global__ void __launch_bounds__(256)
+// Block = 32 rows x COMBINE_WARPS partial lanes; partial arrays are [n_tiles, part_stride] so reads
+// coalesce. 32 lanes per row (1024 threads) keep 32 x 32 partial pairs in flight per block: the kernel
+// reads chunk x n_tiles x 8 bytes (16 MiB at chunk 4096, V = 131072) and is bound by memory latency.
+constexpr int COMBINE_WARPS = 32;
+__global__ void __launch_bounds__(COMBINE_WARPS * 32)
 combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_s, long long part_stride,
                int n_tiles, int rows, long long row0, int K, float inv_tau, const int* __restrict__ nvalid,
                const float* __restrict__ p_sorted, const uint16_t* __restrict__ perm, const float* __restrict__ zg,
@@ -188,13 +191,13 @@ combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_
                const uint8_t* __restrict__ mask, float* __restrict__ lz2, float* __restrict__ logZ_nat,
                float* __restrict__ loss_tok, float* __restrict__ loss_tok_user, float* __restrict__ g_logits,
                int* __restrict__ g_idx, int v0, float* __restrict__ shard_stats, long long T_total, WsHeader* hdr) {
-  __shared__ float sm_m[8][32], sm_s[8][32];
+  __shared__ float sm_m[COMBINE_WARPS][32], sm_s[COMBINE_WARPS][32];
   __shared__ float sm_lz[32];
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int r = blockIdx.x * 32 + tx;       // row within the chunk
   float m = -INFINITY, s = 0.f;
   if (r < rows) {
-    for (int nt = ty; nt < n_tiles; nt += 8) {
+    for (int nt = ty; nt < n_tiles; nt += COMBINE_WARPS) {
       const float pm = part_m[(long long)nt * part_stride + r];
       const float ps = part_s[(long long)nt * part_stride + r];
       const float mn = fmaxf(m, pm);
@@ -206,7 +209,7 @@ combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_
   __syncthreads();
   if (ty == 0 && r < rows) {
     float mm = sm_m[0][tx], ss = sm_s[0][tx];
-    for (int i = 1; i < 8; ++i) {           // fixed order
+    for (int i = 1; i < COMBINE_WARPS; ++i) {   // fixed order
       const float pm = sm_m[i][tx], ps = sm_s[i][tx];
       if (pm == -INFINITY) continue;
       const float mn = fmaxf(mm, pm);
@@ -219,9 +222,10 @@ combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_
     logZ_nat[row0 + r] = l2 * kLn2;
   }
   __syncthreads();
-  // sparse terms: warp ty handles rows ty*4 .. ty*4+3 of this block
-  for (int i = 0; i < 4; ++i) {
-    const int rr = blockIdx.x * 32 + ty * 4 + i;
+  // sparse terms: warp ty handles rows ty*RPW .. ty*RPW+RPW-1 of this block
+  constexpr int RPW = 32 / COMBINE_WARPS;
+  for (int i = 0; i < RPW; ++i) {
+    const int rr = blockIdx.x * 32 + ty * RPW + i;
     if (rr >= rows) break;
     const long long t = row0 + rr;
     const int nv = nvalid[t];
@@ -241,12 +245,12 @@ combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_
     c = warp_sum(c) * inv_tau;
     if (shard_stats != nullptr) {
       // a vocabulary shard: hand the local log-normaliser and cross term to the cross-shard reduction
-      if (tx == 0) { shard_stats[t] = sm_lz[ty * 4 + i]; shard_stats[T_total + t] = c; }
+      if (tx == 0) { shard_stats[t] = sm_lz[ty * RPW + i]; shard_stats[T_total + t] = c; }
       continue;
     }
     if (tx == 0) {
       const bool counted = mask == nullptr || mask[t] != 0;
-      const float lz = sm_lz[ty * 4 + i] * kLn2;
+      const float lz = sm_lz[ty * RPW + i] * kLn2;
       float L = 0.f;
       if (counted) {
         L = Hent[t] - c + Mv[t] * lz;

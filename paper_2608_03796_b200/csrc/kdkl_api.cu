@@ -315,7 +315,7 @@ static int forward_impl(const void* hidden, const void* weight, const int32_t* t
     if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA /*no output map*/, p, di.sm_count, st))) return rc;
     stage_mark(ST_COMBINE, st);
 
-    combine_kernel<<<(unsigned)((rows + 31) / 32), 256, 0, st>>>(
+    combine_kernel<<<(unsigned)((rows + 31) / 32), COMBINE_WARPS * 32, 0, st>>>(
         at<float>(ws, L.part_m), at<float>(ws, L.part_s), L.Cpad, (int)L.n_tiles_v, (int)rows, s0, K, inv_tau,
         at<int>(ws, L.nvalid), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<float>(ws, L.zg),
         at<int>(ws, L.colread), at<float>(ws, L.M), at<float>(ws, L.Hent), loss_mask, at<float>(ws, L.lz2),
