@@ -73,7 +73,9 @@ size_t kdkl_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t 
  *                                duplicates within a row add
  *   topk_val      [T, K]  fp32   teacher values (see teacher_mode)
  *   teacher_lse   [T] fp32 or NULL   full-vocabulary teacher logsumexp at temperature tau
- *   loss_mask     [T] uint8 or NULL  1 = counted, 0 = ignored (teacher row is never read)
+ *   loss_mask     [T] uint8 or NULL  1 = counted, 0 = ignored (teacher row is never read). Row tiles
+ *                                (256 consecutive tokens of a chunk) without a counted token are skipped
+ *                                by every tensor-core sweep, forward and backward: padding costs nothing
  *   chunk         tokens per chunk, 0 = default; the result does not depend on it
  *   loss_out      [1] fp32  mean loss
  *   loss_per_token [T] fp32 or NULL  (0 at ignored tokens)
@@ -134,7 +136,8 @@ int kdkl_forward_finish(const float* all_stats, int32_t n_shards, const uint8_t*
 int kdkl_status(const void* workspace, void* cuda_stream, int32_t* code, int64_t* detail);
 
 /* Saved per-token scalars of Algorithm 1 inside a workspace forward has filled (device pointers
- * into the workspace; valid until the workspace is reused): log Z of z/tau and the retained mass M. */
+ * into the workspace; valid until the workspace is reused): log Z of z/tau and the retained mass M
+ * (both 0 at ignored tokens). */
 int kdkl_saved_state(void* workspace, int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk,
                      const kdkl_options* opt, const float** logZ, const float** mass);
 

@@ -174,6 +174,27 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
   if (lane == 0) { nvalid[t] = nv; Mout[t] = msum; Hent[t] = hsum; }
 }
 
+// ------------------------------------------------------------------------------------ live row tiles
+// live[c * tiles_per_chunk + i] = 1 when at least one token of rows [c*chunk + i*tile_rows, ... + tile_rows)
+// (clipped to the chunk and to T) is counted. The GEMM kernels skip row tiles whose flag is 0: a padding
+// tail or a run of ignored tokens costs no tensor-core work. One warp per tile.
+__global__ void __launch_bounds__(256)
+tile_live_kernel(const uint8_t* __restrict__ mask, long long T, long long chunk, int tile_rows, int tiles_per_chunk,
+                 long long n_flags, uint8_t* __restrict__ live) {
+  const long long f = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (f >= n_flags) return;
+  const int lane = threadIdx.x & 31;
+  const long long c = f / tiles_per_chunk, i = f - c * tiles_per_chunk;
+  const long long r0 = c * chunk + i * tile_rows;
+  long long r1 = r0 + tile_rows;
+  if (r1 > (c + 1) * chunk) r1 = (c + 1) * chunk;
+  if (r1 > T) r1 = T;
+  int any = 0;
+  for (long long r = r0 + lane; r < r1; r += 32) any |= mask[r] != 0;
+  any = __any_sync(0xffffffffu, any);
+  if (lane == 0) live[f] = any ? 1 : 0;
+}
+
 // ------------------------------------------------------------------------------------ combine
 // Per chunk. Merges the per-vocab-tile (max, sum) partials of every row into the log-normaliser,
 // adds the sparse terms and writes the per-token loss  L_t = Hent_t - C_t + M_t log Z_t
@@ -196,7 +217,10 @@ combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int r = blockIdx.x * 32 + tx;       // row within the chunk
   float m = -INFINITY, s = 0.f;
-  if (r < rows) {
+  // ignored tokens: their partials may not exist (a row tile with no counted token is skipped by the
+  // GEMM), so nothing is read for them and their log Z is reported as 0
+  const bool row_counted = r < rows && (mask == nullptr || mask[row0 + r] != 0);
+  if (row_counted) {
     for (int nt = ty; nt < n_tiles; nt += COMBINE_WARPS) {
       const float pm = part_m[(long long)nt * part_stride + r];
       const float ps = part_s[(long long)nt * part_stride + r];
@@ -216,7 +240,7 @@ combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_
       ss = ss * exp2f(mm - mn) + ps * exp2f(pm - mn);
       mm = mn;
     }
-    const float l2 = mm + log2f(ss);
+    const float l2 = row_counted ? mm + log2f(ss) : 0.f;
     sm_lz[tx] = l2;
     lz2[row0 + r] = l2;
     logZ_nat[row0 + r] = l2 * kLn2;

@@ -62,6 +62,13 @@ struct GemmParams {
   int split_rows;
   int* status;               // device status word pair {code, where}
   const int* go;             // optional: kernel returns at once when *go == 0
+  // Skipping work for ignored tokens (both optional, one flag per TILE_M rows, 0 = every token of
+  // that row tile is ignored). m_live [m_tiles]: a dead row tile of D is not computed - LSE / TOPK
+  // write nothing for it, the store epilogues write zeros (nothing when accumulating). k_live
+  // [ceil(K / TILE_M)]: dead k-blocks of the contraction are not loaded or multiplied (their A
+  // columns are zeros by construction); a unit's first k-block is always processed.
+  const uint8_t* m_live;
+  const uint8_t* k_live;
   // EPI_STORE_F32: 1 -> output += D (TMA reduce-add), 0 -> output = D. Outputs go through tmC.
   int accumulate;
   // EPI_LSE / EPI_DLOGITS: all row-indexed pointers are already offset to this chunk's row 0
@@ -185,6 +192,19 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     else           { nt = tile % p.n_tiles; mt = tile / p.n_tiles; }
   };
 
+  // Dead k-blocks: the flags of the first 64 row tiles of the contraction are read once into a bit
+  // mask (a load per k-block would sit on the issue path of the producer and the MMA thread); row
+  // tiles past the 64th (chunks beyond 64 * TILE_M tokens) are never skipped.
+  unsigned long long k_dead = 0ull;
+  if (p.k_live != nullptr && lane == 0 && warp < 2) {
+    const int nkt = (p.K + TILE_M - 1) / TILE_M;
+    for (int t = 0; t < nkt && t < 64; ++t) k_dead |= (unsigned long long)(p.k_live[t] == 0) << t;
+  }
+  auto kb_dead = [&](int kb, int kb0) {
+    const int t = (kb * BK) / TILE_M;
+    return kb != kb0 && t < 64 && ((k_dead >> t) & 1ull);
+  };
+
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -198,9 +218,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int tile, split, kb0, kb1, mt, nt;
         unit_decode(unit, tile, split, kb0, kb1);
         tile_coords(tile, mt, nt);
+        if (p.m_live != nullptr && !p.m_live[mt]) continue;   // dead row tile: all three roles skip it alike
         const int m0 = mt * TILE_M + (int)cta_rank * BM;      // this CTA's rows of A
         const int n0 = nt * BN + (int)cta_rank * B_ROWS;      // this CTA's rows of B
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (kb_dead(kb, kb0)) continue;
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
@@ -226,6 +248,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
           issued |= 1u << s;
           last_par = (last_par & ~(1u << s)) | (ph << s);
+          ++it;
         }
       }
       if (!ok) {
@@ -252,15 +275,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       auto commit = [&](uint32_t bar) { if (NCTA == 2) umma_commit_pair(bar); else umma_commit(bar); };
       uint32_t it = 0, lt = 0;
       bool ok = true;
-      for (int unit = worker; unit < num_units && ok; unit += num_workers, ++lt) {
-        int tile, split, kb0, kb1;
+      for (int unit = worker; unit < num_units && ok; unit += num_workers) {
+        int tile, split, kb0, kb1, mt, nt;
         unit_decode(unit, tile, split, kb0, kb1);
+        tile_coords(tile, mt, nt);
+        if (p.m_live != nullptr && !p.m_live[mt]) continue;
         const uint32_t acc = lt & 1u;
         const uint32_t aph = (lt >> 1) & 1u;
         if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + acc * BN;
-        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (kb_dead(kb, kb0)) continue;
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, 3)) { ok = false; break; }
@@ -276,8 +302,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             mma(tmem_d, ad, bd, (kb > kb0 || j > 0) ? 1u : 0u);
           }
           commit(empty_bar(s));                // frees the stage (in both CTAs) when these MMAs have read it
+          ++it;
         }
         if (ok) commit(tfull_bar(acc));        // accumulator complete (signalled in both CTAs)
+        ++lt;
       }
     }
   } else {
@@ -287,10 +315,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     constexpr bool kBf16Out = (EPI == EPI_STORE_BF16 || EPI == EPI_DLOGITS);
     uint32_t lt = 0, nbox = 0;
     bool ok = true;
-    for (int unit = worker; unit < num_units && ok; unit += num_workers, ++lt) {
+    for (int unit = worker; unit < num_units && ok; unit += num_workers) {
       int tile, split, kb0, kb1, mt, nt;
       unit_decode(unit, tile, split, kb0, kb1);
       tile_coords(tile, mt, nt);
+      // A dead row tile (every token ignored) was skipped by the producer and the MMA issuer: no
+      // accumulator belongs to it. LSE / TOPK have nothing to write; a store epilogue writes zeros,
+      // or nothing when it would add them.
+      const bool dead = p.m_live != nullptr && !p.m_live[mt];
+      if (dead && (EPI == EPI_LSE || EPI == EPI_TOPK || (EPI == EPI_STORE_F32 && p.accumulate))) continue;
       const int m0 = mt * TILE_M + (int)cta_rank * BM, n0 = nt * BN;   // this CTA's 128 x 256 part of D
       const int row = m0 + row_in_tile;
       const bool row_ok = row < p.M;
@@ -303,7 +336,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       float row_b = 0.f, row_off = -INFINITY, row_thr = INFINITY;
       if (EPI == EPI_TOPK) { if (row_ok) row_thr = p.thr[row]; }
       if (EPI == EPI_LSE || EPI == EPI_DLOGITS) {
-        if (row_ok) {
+        if (row_ok && !dead) {
           idxrow = p.idx_sorted + (long long)row * p.Ktop;
           nv = p.nvalid[row];
           cur = lower_bound_i32(idxrow, nv, n0);
@@ -317,9 +350,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
 
       // the decision to go on is taken by the whole warp: tcgen05.ld below is warp-collective
-      const bool arrived = mbar_wait(tfull_bar(acc), aph, abort_flag, p.status, 4);
-      if (!__all_sync(0xffffffffu, arrived)) { ok = false; break; }
-      tc_fence_after();
+      if (!dead) {
+        const bool arrived = mbar_wait(tfull_bar(acc), aph, abort_flag, p.status, 4);
+        if (!__all_sync(0xffffffffu, arrived)) { ok = false; break; }
+        tc_fence_after();
+      }
       const uint32_t taddr = tmem_base + (uint32_t(lg * 32) << 16) + acc * BN;
 
       float m_run = -INFINITY, s_run = 0.f;
@@ -333,8 +368,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (col0 >= p.N && (!kBf16Out || (w & 1) == 0)) break;
         uint32_t r[32];
         __syncwarp();
-        tmem_ld32(taddr + w * 32, r);
-        tmem_ld_wait();
+        if (!dead) {
+          tmem_ld32(taddr + w * 32, r);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = 0u;
+        }
         const bool full_w = col0 + 32 <= p.N;
 
         if (EPI == EPI_LSE) {
@@ -401,6 +441,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (EPI == EPI_STORE_BF16) {
 #pragma unroll
               for (int j = 0; j < 16; ++j) v[j] = pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+            } else if (dead) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) v[j] = 0u;
             } else {  // EPI_DLOGITS
               // a_t * 2^(s - lz2) = 2^(s + (log2 a_t - lz2)): the row coefficient rides in the exponent
               // (a_t = 0 for ignored tokens gives -inf, hence exact zeros)
@@ -441,12 +484,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       }
+      if (dead) continue;                      // no accumulator stage was used
       // accumulator stage is free again
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
         if (NCTA == 2) mbar_arrive_cluster(leader_bar(tempty_bar(acc))); else mbar_arrive(tempty_bar(acc));
       }
+      ++lt;
 
       if (EPI == EPI_LSE) {
         if (row_ok) {

@@ -181,7 +181,8 @@ struct WsLayout {
   long long C, Cpad, Vpad, n_tiles_v;
   int dh_splits;             // split-K factor of the dH GEMM at full chunks
   size_t hdr, idx_sorted, p_sorted, perm, zg, colread, nvalid, M, Hent, lz2, logZ, loss_tok, coefA, coefB;
-  size_t part_m, part_s, G, dh_part, total;
+  size_t part_m, part_s, G, dh_part, live, total;
+  long long tiles_per_chunk, n_live;   // live-row-tile flags: one per kTileM rows of every chunk
 };
 
 static WsLayout ws_layout(long long T, long long H, long long V, int K, long long chunk) {
@@ -212,6 +213,9 @@ static WsLayout ws_layout(long long T, long long H, long long V, int K, long lon
   L.G = take((size_t)L.Cpad * L.Vpad * 2);
   L.dh_splits = choose_k_splits(((L.C + kTileM - 1) / kTileM) * ((H + BN - 1) / BN), (V + BK - 1) / BK);
   L.dh_part = take(L.dh_splits > 1 ? (size_t)L.dh_splits * L.Cpad * H * 4 : 0);
+  L.tiles_per_chunk = (L.C + kTileM - 1) / kTileM;
+  L.n_live = ((T + L.C - 1) / L.C) * L.tiles_per_chunk;
+  L.live = take((size_t)L.n_live);
   L.total = o;
   return L;
 }
@@ -291,11 +295,21 @@ static int forward_impl(const void* hidden, const void* weight, const int32_t* t
       at<int>(ws, L.idx_sorted), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<int>(ws, L.nvalid),
       at<float>(ws, L.M), at<float>(ws, L.Hent), hdr);
   KDKL_LAUNCHED("prep_kernel");
+  // with a mask: which row tiles hold at least one counted token (the others are skipped by every GEMM,
+  // forward and backward; the flags stay in the workspace for kdkl_backward)
+  const uint8_t* live = nullptr;
+  if (loss_mask != nullptr) {
+    tile_live_kernel<<<(unsigned)((L.n_live + 7) / 8), 256, 0, st>>>(loss_mask, T, L.C, kTileM, (int)L.tiles_per_chunk,
+                                                                    L.n_live, at<uint8_t>(ws, L.live));
+    KDKL_LAUNCHED("tile_live_kernel");
+    live = at<uint8_t>(ws, L.live);
+  }
 
   CUtensorMap tmW;
   if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, kBRows))) return rc;
 
-  for (long long s0 = 0; s0 < T; s0 += L.C) {
+  long long fci = 0;
+  for (long long s0 = 0; s0 < T; s0 += L.C, ++fci) {
     const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
     CUtensorMap tmA;
     const __nv_bfloat16* hA = reinterpret_cast<const __nv_bfloat16*>(hidden) + s0 * H;
@@ -311,6 +325,7 @@ static int forward_impl(const void* hidden, const void* weight, const int32_t* t
     p.part_m = at<float>(ws, L.part_m); p.part_s = at<float>(ws, L.part_s); p.part_stride = L.Cpad;
     p.zg = at<float>(ws, L.zg) + s0 * K;
     p.colread = at<int>(ws, L.colread) + s0 * K;
+    p.m_live = live ? live + fci * L.tiles_per_chunk : nullptr;
     stage_mark(ST_F1, st);
     if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA /*no output map*/, p, di.sm_count, st))) return rc;
     stage_mark(ST_COMBINE, st);
@@ -408,9 +423,12 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
   CUtensorMap tmdW;
   if ((rc = make_tmap_out_f32(&tmdW, dweight, (uint64_t)H, (uint64_t)V, (uint64_t)H))) return rc;
 
+  // live-row-tile flags written by the forward call (same mask)
+  const uint8_t* live = loss_mask != nullptr ? at<uint8_t>(ws, L.live) : nullptr;
   long long ci = 0;
   for (long long s0 = 0; s0 < T; s0 += L.C, ++ci) {
     const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
+    const uint8_t* live_c = live ? live + ci * L.tiles_per_chunk : nullptr;
     const __nv_bfloat16* hA = reinterpret_cast<const __nv_bfloat16*>(hidden) + s0 * H;
     CUtensorMap tmA, tmG, tmGmn, tmhmn;
     if ((rc = make_tmap_bf16(&tmA, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, BK, BM))) return rc;
@@ -429,6 +447,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p.coefA = at<float>(ws, L.coefA) + s0;
     p.coefB = at<float>(ws, L.coefB) + s0;
     p.neg_a = grad_loss < 0.f ? 1 : 0;
+    p.m_live = live_c;                 // dead row tiles of G are written as zeros without being computed
     CUtensorMap tmGout;
     if ((rc = make_tmap_out_bf16(&tmGout, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad))) return rc;
     stage_mark(ST_B1, st);
@@ -443,6 +462,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p2.m_tiles = (int)((rows + kTileM - 1) / kTileM); p2.n_tiles = (int)((H + BN - 1) / BN); p2.m_inner = 0;
     p2.status = &hdr->status; p2.go = go;
     p2.accumulate = 0;
+    p2.m_live = live_c;                // their dH rows are zeros
     // a short last chunk may want a different split; never more than the workspace was sized for
     int sp = choose_k_splits((long long)p2.m_tiles * p2.n_tiles, (V + BK - 1) / BK);
     if (sp > L.dh_splits) sp = L.dh_splits;
@@ -479,6 +499,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p3.m_tiles = (int)((V + kTileM - 1) / kTileM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0; p3.k_splits = 1;
     p3.status = &hdr->status; p3.go = go;
     p3.accumulate = (ci > 0 || o.accumulate_dweight) ? 1 : 0;
+    p3.k_live = live_c;                // and their zero rows of G are left out of the contraction over tokens
     stage_mark(ST_B3, st);
     if ((rc = launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, tmdW, p3, di.sm_count, st))) return rc;
   }

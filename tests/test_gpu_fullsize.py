@@ -63,7 +63,8 @@ def test_fullsize_sampled_parity(name, n_rows, partial_mass):
     lt = full.loss_per_token[Rd].cpu().double().numpy()
     np.testing.assert_allclose(lt, o["loss_tok"], rtol=0, atol=TOK_ATOL)
     lz, M = full.saved_state()
-    np.testing.assert_allclose(lz[Rd].cpu().double().numpy(), o["logZ"], rtol=0, atol=TOK_ATOL)
+    np.testing.assert_allclose(lz[Rd].cpu().double().numpy()[counted], o["logZ"][counted], rtol=0, atol=TOK_ATOL)
+    assert not lz[Rd].cpu().numpy()[~counted].any()          # log Z of ignored tokens is reported as 0
     np.testing.assert_allclose(M[Rd].cpu().double().numpy()[counted], o["M"][counted], rtol=0, atol=1e-5)
     usable = (idxR >= 0) & (idxR < cfg.V) & counted[:, None]
     gi = full.gathered_idx[Rd].cpu().numpy()

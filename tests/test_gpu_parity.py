@@ -59,7 +59,8 @@ def _compare(op, o, d, check_grads=True):
     lt = op.loss_per_token.cpu().double().numpy()
     np.testing.assert_allclose(lt, o["loss_tok"], rtol=0, atol=TOK_ATOL)
     lz, M = op.saved_state()
-    np.testing.assert_allclose(lz.cpu().double().numpy(), o["logZ"], rtol=0, atol=TOK_ATOL)
+    np.testing.assert_allclose(lz.cpu().double().numpy()[counted], o["logZ"][counted], rtol=0, atol=TOK_ATOL)
+    assert not lz.cpu().numpy()[~counted].any()            # ignored tokens: log Z is reported as 0
     np.testing.assert_allclose(M.cpu().double().numpy()[counted], o["M"][counted], rtol=0, atol=1e-5)
     # gathered columns: bit-exact wherever the slot holds a usable index of a counted token
     idx = d["topk_idx"].numpy()
@@ -165,6 +166,40 @@ def test_k1_and_large_k():
     _compare(_run(d, 40, 128, 1000, 1, 0, 1.0), _oracle(d, 1.0), d)
     d = _small_case(33, 64, 2048, 600, seed=14)              # K above the usual 100, not a power of two
     _compare(_run(d, 33, 64, 2048, 600, 0, 0.9), _oracle(d, 0.9), d)
+
+
+@pytest.mark.parametrize("chunk,accumulate", [(600, 0), (600, 1), (0, 0), (256, 0), (300, 0)])
+def test_row_tiles_without_counted_tokens_are_skipped(chunk, accumulate):
+    """Runs of ignored tokens that cover whole row tiles (a padding tail, a dead first tile, a whole dead
+    chunk): those tiles are not computed at all, yet every output must be as if they had been - zero
+    dHidden rows, untouched dWeight contributions, per-token loss 0 - and the rest must match the oracle."""
+    T, H, V, K = 1300, 72, 1001, 7
+    d = _small_case(T, H, V, K, seed=123)
+    mask = torch.ones(T, dtype=torch.uint8)
+    mask[0:260] = 0            # first 256-row tile of the first chunk dead (whatever the chunk size)
+    mask[600:1200] = 0         # with chunk = 600: the whole second chunk; with one chunk: tiles 768..1023 dead
+    mask[1290:] = 0            # a short ignored tail inside a live tile
+    mask[5] = 1 if chunk == 300 else 0     # chunk 300: a single counted token keeps the first tile alive
+    d["mask"] = mask
+    d["topk_idx"][mask == 0] = -1
+    d["topk_val"][mask == 0] = float("nan")
+    dev = torch.device("cuda:0")
+    opt = B.make_options(accumulate_dweight=accumulate)
+    op = B.FusedChunkedKL(T, H, V, K, chunk=chunk, temperature=1.0, opt=opt, device=dev, want_gathered=True,
+                          want_per_token=True)
+    g = {k: (v.to(dev) if v is not None else None) for k, v in d.items()}
+    base = torch.randn(V, H, generator=torch.Generator().manual_seed(1)) * 1e-3
+    op.dhidden.fill_(float("nan"))
+    if accumulate:
+        op.dweight.copy_(base)
+    else:
+        op.dweight.fill_(float("nan"))
+    op.forward(g["hidden"], g["weight"], g["topk_idx"], g["topk_val"], loss_mask=g["mask"])
+    op.backward(g["hidden"], g["weight"], loss_mask=g["mask"])
+    o = _oracle(d, 1.0)
+    if accumulate:
+        o["dW"] = o["dW"] + base.double().numpy()
+    _compare(op, o, d)
 
 
 def test_negative_upstream_gradient():
