@@ -116,3 +116,48 @@ def test_token_shards_match_oracle():
     assert abs(loss - o["loss"]) <= 1e-3 * abs(o["loss"])
     assert _fro(dW.cpu().double().numpy(), o["dW"]) <= 1e-2
     assert _fro(dH.float().cpu().double().numpy(), o["dH"]) <= 1e-2
+
+
+@pytest.mark.parametrize("seed", list(range(2000, 2016)))
+def test_random_shardings_match_oracle(seed):
+    """Seeded random shapes, 2-4 shards at random (ragged, possibly tiny) boundaries, masks with dead
+    runs, duplicates / empty slots, partial teacher mass: every rank's loss, the summed dHidden and the
+    concatenated dWeight against the full-vocabulary oracle."""
+    r = np.random.default_rng(seed)
+    T = int(r.choice([5, 130, 300, 700]))
+    H = 8 * int(r.integers(1, 30))
+    K = int(r.choice([1, 4, 16, 40]))
+    V = int(r.integers(max(4 * K, 64), 3000))
+    R = int(r.integers(2, 5))
+    cuts = sorted(int(x) for x in r.choice(np.arange(1, V), size=R - 1, replace=False))
+    bounds = [0] + cuts + [V]
+    tau = float(r.choice([0.7, 1.0, 2.0]))
+    chunk = int(r.choice([0, 64, 100, 256]))
+    g = torch.Generator().manual_seed(seed)
+    idx = (torch.randint(0, V, (T, K), generator=g) if r.random() < 0.3
+           else torch.stack([torch.randperm(V, generator=g)[:K] for _ in range(T)])).to(torch.int32)
+    if r.random() < 0.5:
+        idx[torch.rand(T, K, generator=g) < 0.1] = -1
+    mask = None
+    if r.random() < 0.6:
+        mask = (torch.rand(T, generator=g) >= 0.15).to(torch.uint8)
+        if T >= 600:
+            mask[100:100 + int(r.integers(256, 450))] = 0
+    d = {"hidden": torch.randn(T, H, generator=g).to(torch.bfloat16),
+         "weight": (torch.randn(V, H, generator=g) / H ** 0.5).to(torch.bfloat16),
+         "topk_idx": idx.contiguous(), "topk_val": (torch.randn(T, K, generator=g) * 3 ** 0.5).float(), "mask": mask}
+    lse = None
+    if r.random() < 0.5:
+        lse = torch.logsumexp(d["topk_val"].double() / tau, 1).float() + torch.rand(T, generator=g) * 0.4
+    ranks, dH, dW = _run_sharded(d, T, H, V, K, bounds, chunk, tau, lse=lse)
+    o = kdkl_oracle(d["hidden"].double().numpy(), d["weight"].double().numpy(), d["topk_idx"].numpy(),
+                    d["topk_val"].numpy(), tau=tau, mask=None if mask is None else mask.numpy(),
+                    teacher_lse=None if lse is None else lse.double().numpy())
+    for op in ranks:
+        assert abs(op.loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"]) + 1e-6
+        np.testing.assert_allclose(op.loss_per_token.cpu().double().numpy(), o["loss_tok"], rtol=0, atol=2e-4)
+        assert torch.equal(op.loss_per_token, ranks[0].loss_per_token)      # identical bits on every rank
+    assert _fro(dH.cpu().double().numpy(), o["dH"]) <= 1e-2
+    assert _fro(dW.cpu().double().numpy(), o["dW"]) <= 1e-2
+    if mask is not None:
+        assert not dH[mask == 0].abs().sum().item()
