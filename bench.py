@@ -228,6 +228,8 @@ def main():
     torch.cuda.synchronize()
     torch.cuda.reset_peak_memory_stats()
     base_mem = torch.cuda.memory_allocated()
+    torch.cuda.empty_cache()                        # idle blocks left by the input generators go back first
+    free_before = torch.cuda.mem_get_info()[0]      # driver's view, for a cross-check of the allocator's peak
     op = B.FusedChunkedKL(T, H, V, K, chunk=cfg.chunk, temperature=cfg.tau, device=dev)
 
     def step():
@@ -249,18 +251,24 @@ def main():
         torch.cuda.synchronize()
 
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     barrier()
     with ClockSampler(local_rank) as clk:
         ev0.record()
-        for _ in range(args.steps):
+        for i in range(args.steps):
             step()
+            step_ev[i].record()
         ev1.record()
         barrier()
     ms_total = ev0.elapsed_time(ev1)
+    marks = [ev0] + step_ev
+    per_step = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps))
+    ms_median, ms_min = per_step[len(per_step) // 2], per_step[0]
     ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
     loss_val = float(op.loss.item())
     peak_mem = torch.cuda.max_memory_allocated()
+    driver_delta = free_before - torch.cuda.mem_get_info()[0]   # what the op's buffers took from the device
     ws_bytes = op.workspace.numel()
 
     # peak memory versus sequence length for this shape, from the allocation sizes alone (inputs + outputs +
@@ -373,7 +381,8 @@ def main():
     step_tflops = cfg.flops / (ms_step * 1e-3) / 1e12
     line = {
         "metric": METRIC, "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
-        "warmup": n_warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": n_warm, "ms_per_step": ms_step, "ms_per_step_median": ms_median, "ms_per_step_min": ms_min,
+        "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": workload_name(cfg), "l2": f"inputs larger than L2 (weight {V * H * 2 / 2**20:.0f} MiB, dW {V * H * 4 / 2**20:.0f} MiB per step)",
                    "per_rank_tokens": T, "parallelism": f"independent batches x{world}"},
@@ -383,6 +392,7 @@ def main():
                                                                      FALLBACK_PEAKS["bf16_tflops_sustained"])),
         "peaks": peaks.get("_source"),
         "peak_mem_gb": peak_mem / 1e9, "workspace_gb": ws_bytes / 1e9, "input_mem_gb": base_mem / 1e9,
+        "op_mem_gb_allocator": (peak_mem - base_mem) / 1e9, "op_mem_gb_driver": driver_delta / 1e9,
         "peak_mem_gb_vs_tokens": mem_model,
         "loss": loss_val,
         "clocks": clk.summary(),

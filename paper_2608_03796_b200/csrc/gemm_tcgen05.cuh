@@ -32,6 +32,7 @@ namespace kdkl {
 constexpr int BM = 128, BN = 256, BK = 64;   // per-CTA accumulator: 128 TMEM lanes x 256 fp32 columns
 constexpr int UMMA_K = 16;
 constexpr int GEMM_THREADS = 192;
+constexpr int MAX_LIVE_KB = 512;               // k-block skipping is available for contractions up to 512 k-blocks
 constexpr int TMEM_COLS = 512;
 constexpr int STAGING_WARP_BYTES = 2 * 4096;   // per epilogue warp: two 32-row x 128-byte output boxes
 constexpr int STAGING_BYTES = 4 * STAGING_WARP_BYTES;
@@ -48,7 +49,8 @@ struct GemmCfg {
   static constexpr int B_STAGE_BYTES = B_ROWS * BK * 2;  // 32 / 16 KiB
   static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
   static constexpr int STAGES = 4;   // measured: 3 starves the tensor pipe, 5 and 6 are no faster than 4
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ +
+                                    2 * MAX_LIVE_KB /*live k-block list*/;
 };
 
 enum { EPI_STORE_F32 = 0, EPI_STORE_BF16 = 1, EPI_LSE = 2, EPI_DLOGITS = 3, EPI_TOPK = 4 };
@@ -65,8 +67,9 @@ struct GemmParams {
   // Skipping work for ignored tokens (both optional, one flag per TILE_M rows, 0 = every token of
   // that row tile is ignored). m_live [m_tiles]: a dead row tile of D is not computed - LSE / TOPK
   // write nothing for it, the store epilogues write zeros (nothing when accumulating). k_live
-  // [ceil(K / TILE_M)]: dead k-blocks of the contraction are not loaded or multiplied (their A
-  // columns are zeros by construction); a unit's first k-block is always processed.
+  // [ceil(K / TILE_M)] (at most 32 flags, k_splits must be 1): dead k-blocks of the contraction are not
+  // loaded or multiplied (their A columns are zeros by construction); if all are dead the first one is
+  // processed, so that the accumulator is defined.
   const uint8_t* m_live;
   const uint8_t* k_live;
   // EPI_STORE_F32: 1 -> output += D (TMA reduce-add), 0 -> output = D. Outputs go through tmC.
@@ -122,6 +125,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+__device__ __forceinline__ int kblocks_all(int K) { return (K + BK - 1) / BK; }
+
 template <int EPI, bool A_MN, bool B_MN, int NCTA>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -169,6 +174,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (NCTA == 2) { tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS); tmem_relinquish_pair(); }
     else           { tmem_alloc(smem_u32(tmem_slot), TMEM_COLS); tmem_relinquish(); }
   }
+  // Dead k-blocks: one warp turns the row-tile flags into the ascending list of live k-blocks in shared
+  // memory, once per kernel. The two single-thread loops below then run over that list with exactly
+  // the loop shape of the unskipped case (a test per k-block inside those loops costs whole percents
+  // of the kernel even when it is never taken).
+  const bool kskip = p.k_live != nullptr;
+  uint16_t* live_kb = reinterpret_cast<uint16_t*>(smem_al + STAGES * STAGE_BYTES + STAGING_BYTES + 256);
+  volatile int* n_live_kb = reinterpret_cast<volatile int*>(tmem_slot + 2);
+  if (kskip && warp == 2) {
+    const int nkt = (p.K + TILE_M - 1) / TILE_M;
+    const uint32_t live_tiles = __ballot_sync(0xffffffffu, lane < nkt && p.k_live[lane] != 0);
+    if (lane == 0) {
+      int n = 0;
+      for (int kb = 0; kb < kblocks_all(p.K); ++kb)
+        if ((live_tiles >> ((kb * BK) / TILE_M)) & 1u) live_kb[n++] = (uint16_t)kb;
+      if (n == 0) live_kb[n++] = 0;
+      *n_live_kb = n;
+    }
+  }
   tc_fence_before();
   __syncthreads();
   if (NCTA == 2) cluster_sync_all();   // the peer's barriers exist before anything arrives on them
@@ -192,19 +215,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     else           { nt = tile % p.n_tiles; mt = tile / p.n_tiles; }
   };
 
-  // Dead k-blocks: the flags of the first 64 row tiles of the contraction are read once into a bit
-  // mask (a load per k-block would sit on the issue path of the producer and the MMA thread); row
-  // tiles past the 64th (chunks beyond 64 * TILE_M tokens) are never skipped.
-  unsigned long long k_dead = 0ull;
-  if (p.k_live != nullptr && lane == 0 && warp < 2) {
-    const int nkt = (p.K + TILE_M - 1) / TILE_M;
-    for (int t = 0; t < nkt && t < 64; ++t) k_dead |= (unsigned long long)(p.k_live[t] == 0) << t;
-  }
-  auto kb_dead = [&](int kb, int kb0) {
-    const int t = (kb * BK) / TILE_M;
-    return kb != kb0 && t < 64 && ((k_dead >> t) & 1ull);
-  };
-
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -221,8 +231,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (p.m_live != nullptr && !p.m_live[mt]) continue;   // dead row tile: all three roles skip it alike
         const int m0 = mt * TILE_M + (int)cta_rank * BM;      // this CTA's rows of A
         const int n0 = nt * BN + (int)cta_rank * B_ROWS;      // this CTA's rows of B
-        for (int kb = kb0; kb < kb1; ++kb) {
-          if (kb_dead(kb, kb0)) continue;
+        const int nkb = kskip ? *n_live_kb : kb1 - kb0;
+        for (int i = 0; i < nkb; ++i, ++it) {
+          const int kb = kskip ? (int)live_kb[i] : kb0 + i;
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
@@ -248,7 +259,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
           issued |= 1u << s;
           last_par = (last_par & ~(1u << s)) | (ph << s);
-          ++it;
         }
       }
       if (!ok) {
@@ -273,6 +283,19 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (NCTA == 2) umma_bf16_pair(d, ad, bd, idesc, accf); else umma_bf16(d, ad, bd, idesc, accf);
       };
       auto commit = [&](uint32_t bar) { if (NCTA == 2) umma_commit_pair(bar); else umma_commit(bar); };
+      // This single thread feeds the tensor pipe: every instruction here is on the critical path, so the
+      // shared-memory descriptors are not rebuilt per instruction. Their upper words and the layout bits
+      // of the lower words are constants; the 14-bit address field advances by STAGE_BYTES / 16 per
+      // stage and by a fixed step per K = 16 slice (all addresses stay below 256 KiB: no carry).
+      constexpr uint32_t A_LBO = A_MN ? BK * 128 : 0, B_LBO = B_MN ? BK * 128 : 0;
+      constexpr uint32_t A_STEP = (A_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+      constexpr uint32_t B_STEP = (B_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+      constexpr uint32_t STAGE_STEP = STAGE_BYTES >> 4;
+      const uint64_t a_proto = make_smem_desc(smem_base, A_LBO, 1024);
+      const uint64_t b_proto = make_smem_desc(smem_base + A_STAGE_BYTES, B_LBO, 1024);
+      const uint32_t a_hi = (uint32_t)(a_proto >> 32), a_lo0 = (uint32_t)a_proto;
+      const uint32_t b_hi = (uint32_t)(b_proto >> 32), b_lo0 = (uint32_t)b_proto;
+      auto desc = [](uint32_t lo, uint32_t hi) { return (static_cast<uint64_t>(hi) << 32) | lo; };
       uint32_t it = 0, lt = 0;
       bool ok = true;
       for (int unit = worker; unit < num_units && ok; unit += num_workers) {
@@ -285,24 +308,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + acc * BN;
-        for (int kb = kb0; kb < kb1; ++kb) {
-          if (kb_dead(kb, kb0)) continue;
-          const int s = it % STAGES;
+        uint32_t accf = 0u;                    // the unit's first MMA overwrites the accumulator
+        const int nkb = kskip ? *n_live_kb : kb1 - kb0;
+        for (int i = 0; i < nkb; ++i, ++it) {
+          const uint32_t s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, 3)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_base + s * STAGE_BYTES;
-          const uint32_t sb = sa + A_STAGE_BYTES;
+          const uint32_t alo = a_lo0 + s * STAGE_STEP, blo = b_lo0 + s * STAGE_STEP;
 #pragma unroll
           for (int j = 0; j < BK / UMMA_K; ++j) {
-            const uint64_t ad = A_MN ? make_smem_desc(sa + j * (UMMA_K * 128), BK * 128, 1024)
-                                     : make_smem_desc(sa + j * (UMMA_K * 2), 0, 1024);
-            const uint64_t bd = B_MN ? make_smem_desc(sb + j * (UMMA_K * 128), BK * 128, 1024)
-                                     : make_smem_desc(sb + j * (UMMA_K * 2), 0, 1024);
-            mma(tmem_d, ad, bd, (kb > kb0 || j > 0) ? 1u : 0u);
+            mma(tmem_d, desc(alo + j * A_STEP, a_hi), desc(blo + j * B_STEP, b_hi), accf);
+            accf = 1u;
           }
           commit(empty_bar(s));                // frees the stage (in both CTAs) when these MMAs have read it
-          ++it;
         }
         if (ok) commit(tfull_bar(acc));        // accumulator complete (signalled in both CTAs)
         ++lt;
@@ -322,9 +341,30 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       // A dead row tile (every token ignored) was skipped by the producer and the MMA issuer: no
       // accumulator belongs to it. LSE / TOPK have nothing to write; a store epilogue writes zeros,
       // or nothing when it would add them.
-      const bool dead = p.m_live != nullptr && !p.m_live[mt];
-      if (dead && (EPI == EPI_LSE || EPI == EPI_TOPK || (EPI == EPI_STORE_F32 && p.accumulate))) continue;
       const int m0 = mt * TILE_M + (int)cta_rank * BM, n0 = nt * BN;   // this CTA's 128 x 256 part of D
+      if (p.m_live != nullptr && !p.m_live[mt]) {
+        if (EPI == EPI_STORE_F32 || EPI == EPI_STORE_BF16 || EPI == EPI_DLOGITS) {
+          if (!(EPI == EPI_STORE_F32 && p.accumulate) && m0 + lg * 32 < p.M) {
+            // zero boxes through the same staging / bulk-group protocol as the regular output path
+            constexpr int BOX_COLS = (EPI == EPI_STORE_F32) ? 32 : 64;
+            for (int c0 = n0; c0 < n0 + BN && c0 < p.N; c0 += BOX_COLS) {
+              const uint32_t sbox = staging0 + (warp - 2) * STAGING_WARP_BYTES + (nbox & 1u) * 4096u;
+              if (lane == 0) bulk_wait_read<1>();
+              __syncwarp();
+#pragma unroll
+              for (int c = 0; c < 8; ++c) st_shared_v4(sbox + lane * 128 + (c << 4), 0u, 0u, 0u, 0u);
+              fence_proxy_async_smem();
+              __syncwarp();
+              if (lane == 0) {
+                tma_store_2d(&tmC, sbox, c0, m0 + lg * 32 + split * p.split_rows);
+                bulk_commit();
+              }
+              ++nbox;
+            }
+          }
+        }
+        continue;
+      }
       const int row = m0 + row_in_tile;
       const bool row_ok = row < p.M;
       const uint32_t acc = lt & 1u;
@@ -336,7 +376,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       float row_b = 0.f, row_off = -INFINITY, row_thr = INFINITY;
       if (EPI == EPI_TOPK) { if (row_ok) row_thr = p.thr[row]; }
       if (EPI == EPI_LSE || EPI == EPI_DLOGITS) {
-        if (row_ok && !dead) {
+        if (row_ok) {
           idxrow = p.idx_sorted + (long long)row * p.Ktop;
           nv = p.nvalid[row];
           cur = lower_bound_i32(idxrow, nv, n0);
@@ -350,11 +390,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
 
       // the decision to go on is taken by the whole warp: tcgen05.ld below is warp-collective
-      if (!dead) {
-        const bool arrived = mbar_wait(tfull_bar(acc), aph, abort_flag, p.status, 4);
-        if (!__all_sync(0xffffffffu, arrived)) { ok = false; break; }
-        tc_fence_after();
-      }
+      const bool arrived = mbar_wait(tfull_bar(acc), aph, abort_flag, p.status, 4);
+      if (!__all_sync(0xffffffffu, arrived)) { ok = false; break; }
+      tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(lg * 32) << 16) + acc * BN;
 
       float m_run = -INFINITY, s_run = 0.f;
@@ -368,13 +406,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (col0 >= p.N && (!kBf16Out || (w & 1) == 0)) break;
         uint32_t r[32];
         __syncwarp();
-        if (!dead) {
-          tmem_ld32(taddr + w * 32, r);
-          tmem_ld_wait();
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) r[j] = 0u;
-        }
+        tmem_ld32(taddr + w * 32, r);
+        tmem_ld_wait();
         const bool full_w = col0 + 32 <= p.N;
 
         if (EPI == EPI_LSE) {
@@ -441,9 +474,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (EPI == EPI_STORE_BF16) {
 #pragma unroll
               for (int j = 0; j < 16; ++j) v[j] = pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-            } else if (dead) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) v[j] = 0u;
             } else {  // EPI_DLOGITS
               // a_t * 2^(s - lz2) = 2^(s + (log2 a_t - lz2)): the row coefficient rides in the exponent
               // (a_t = 0 for ignored tokens gives -inf, hence exact zeros)
@@ -484,7 +514,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       }
-      if (dead) continue;                      // no accumulator stage was used
       // accumulator stage is free again
       tc_fence_before();
       __syncwarp();

@@ -499,7 +499,8 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p3.m_tiles = (int)((V + kTileM - 1) / kTileM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0; p3.k_splits = 1;
     p3.status = &hdr->status; p3.go = go;
     p3.accumulate = (ci > 0 || o.accumulate_dweight) ? 1 : 0;
-    p3.k_live = live_c;                // and their zero rows of G are left out of the contraction over tokens
+    // and their zero rows of G are left out of the contraction over tokens (the kernel takes up to 32 flags)
+    p3.k_live = (rows <= 32ll * kTileM && (rows + BK - 1) / BK <= MAX_LIVE_KB) ? live_c : nullptr;
     stage_mark(ST_B3, st);
     if ((rc = launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, tmdW, p3, di.sm_count, st))) return rc;
   }

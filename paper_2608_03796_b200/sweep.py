@@ -50,8 +50,11 @@ def worker(method: str, name: str, steps: int) -> dict:
     cfg = _cfg(name)
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
+    torch.zeros(1, device=dev)                      # context up before the driver's free-memory reading
+    free0 = torch.cuda.mem_get_info()[0]
     d = I.make_inputs(cfg, device=dev)
     torch.cuda.synchronize()
+    torch.cuda.empty_cache()                        # idle blocks left by the input generators go back to the driver
     torch.cuda.reset_peak_memory_stats()
     out = {"method": method, "workload": name, "T": cfg.T, "H": cfg.H, "V": cfg.V, "K": cfg.K, "chunk": cfg.chunk,
            "input_gb": torch.cuda.memory_allocated() / 1e9}
@@ -142,7 +145,8 @@ def worker(method: str, name: str, steps: int) -> dict:
         out.update(ms_per_iter=ms, it_per_s=1e3 / ms, tokens_per_s=cfg.T / (ms * 1e-3),
                    tflops=(0.5 if method == "teacher" else 1.0) * cfg.flops / (ms * 1e-3) / 1e12,   # teacher: 2 sweeps
                    loss=float(loss.item()),
-                   peak_gb=torch.cuda.max_memory_allocated() / 1e9)
+                   peak_gb=torch.cuda.max_memory_allocated() / 1e9,
+                   driver_delta_gb=(free0 - torch.cuda.mem_get_info()[0]) / 1e9)
         if method == "fused":
             code, _ = op.status()
             out["status"] = code
@@ -201,19 +205,20 @@ def main():
                  "Command: `python -m paper_2608_03796_b200.sweep --out " + args.out + "`", "",
                  f"Peaks used: bf16 burst {burst} / sustained {sust} TFLOP/s "
                  f"({'measured' if peaks else 'fallback'}). FLOPs counted as 8*T*H*V per iteration.", "",
-                 "| method | workload | T | ms/iter | it/s | tokens/s | TFLOP/s | % burst | % sustained | peak GB | workspace GB | loss | ‖dH‖ | ‖dW‖ |",
-                 "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|"]
+                 "| method | workload | T | ms/iter | it/s | tokens/s | TFLOP/s | % burst | % sustained | peak GB | driver Δ GB | workspace GB | loss | ‖dH‖ | ‖dW‖ |",
+                 "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|"]
         for r in rows:
             if "ms_per_iter" in r:
                 lines.append(f"| {r['method']} | {r['workload']} | {r['T']} | {r['ms_per_iter']:.2f} | {r['it_per_s']:.3f} | "
                              f"{r['tokens_per_s']:.0f} | {r['tflops']:.0f} | {100 * r['tflops'] / burst:.1f} | "
-                             f"{100 * r['tflops'] / sust:.1f} | {r['peak_gb']:.2f} | {r.get('workspace_gb', 0):.2f} | "
+                             f"{100 * r['tflops'] / sust:.1f} | {r['peak_gb']:.2f} | {r.get('driver_delta_gb', float('nan')):.2f} | "
+                             f"{r.get('workspace_gb', 0):.2f} | "
                              f"{r.get('loss', float('nan')):.5f} | {r.get('dh_norm', float('nan')):.4e} | "
                              f"{r.get('dw_norm', float('nan')):.4e} |")
             elif r.get("oom"):
-                lines.append(f"| {r['method']} | {r['workload']} | {r['T']} | out of memory | | | | | | > {r['peak_gb']:.1f} | | | | |")
+                lines.append(f"| {r['method']} | {r['workload']} | {r['T']} | out of memory | | | | | | > {r['peak_gb']:.1f} | | | | | |")
             else:
-                lines.append(f"| {r['method']} | {r['workload']} | | failed: {r.get('failed', '')[:80]} | | | | | | | | | | |")
+                lines.append(f"| {r['method']} | {r['workload']} | | failed: {r.get('failed', '')[:80]} | | | | | | | | | | | |")
         # least-squares line through the fused peaks of the H=4096 / V=131072 family
         pts = [(r["T"], r["peak_gb"]) for r in rows if r["method"] == "fused" and "ms_per_iter" in r
                and r["H"] == 4096 and r["V"] == 131072 and r["T"] >= 32768]
@@ -243,6 +248,9 @@ def main():
             lines += ["", f"Forward-chunked comparator: {slope * 1e6:.0f} KB/token (logits and their gradient held in full, "
                           f"{slope * 1e9 / rows[0]['V']:.1f} bytes per logit); {min(ratios):.2f}x-{max(ratios):.2f}x the fused "
                           "path's time at every length measured, so on this part there is no length below which it wins."]
+        lines += ["", "peak GB is torch's peak allocated memory (inputs, outputs and workspace are all torch allocations); "
+                      "driver Δ GB is the drop in the driver's free memory over the run (cudaMemGetInfo), which also holds "
+                      "the caching allocator's rounding and idle blocks, so it bounds the peak from above."]
         lines += ["", "The last three columns cross-check the methods against each other on the same inputs: loss, and the "
                       "Frobenius norms of dHidden and dWeight, agree to 4-5 digits.",
                   "", "Context (the paper's loss-only benchmark, 2 x H200 with tensor parallelism 2, each rank holding half "
