@@ -1,0 +1,106 @@
+"""torch.autograd entry to the fused chunked KL loss (and the optional feature loss).
+
+    loss = fused_chunked_kl(hidden, weight, topk_idx, topk_val, teacher_lse=None, loss_mask=None,
+                            chunk=4096, temperature=1.0)
+    loss.backward()          # hidden.grad [T,H] bf16, weight.grad [V,H] bf16 (rounded from the fp32 dW)
+
+Marshalling only: forward runs kdkl_forward, backward runs kdkl_backward with the upstream gradient
+as `grad_loss`; nothing of the loss arithmetic happens in torch ops. The upstream gradient of a scalar
+loss is read to the host once (`grad.item()`), since the C entry point takes it as a plain float.
+Workspace and gradient buffers are cached per shape on the function object, so repeated steps allocate
+nothing. `weight_grad_fp32=True` hands back the fp32 dW buffer itself (Megatron-style main_grad use)
+instead of a bf16 copy; with `dweight_out` given, dW is accumulated into that fp32 tensor in place.
+"""
+from __future__ import annotations
+
+from typing import Optional
+
+import torch
+
+from . import binding as B
+
+_cache: dict = {}
+
+
+def _holder(T, H, V, K, chunk, tau, accumulate, device) -> B.FusedChunkedKL:
+    key = (T, H, V, K, chunk, tau, accumulate, str(device))
+    op = _cache.get(key)
+    if op is None:
+        op = B.FusedChunkedKL(T, H, V, K, chunk=chunk, temperature=tau,
+                              opt=B.make_options(accumulate_dweight=accumulate), device=device)
+        _cache[key] = op
+    return op
+
+
+class _FusedChunkedKL(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, chunk, temperature, dweight_out,
+                weight_grad_fp32):
+        T, H = hidden.shape
+        V, K = weight.shape[0], topk_idx.shape[1]
+        op = _holder(T, H, V, K, int(chunk), float(temperature), 1 if dweight_out is not None else 0, hidden.device)
+        op.forward(hidden, weight, topk_idx, topk_val, teacher_lse=teacher_lse, loss_mask=loss_mask)
+        ctx.op, ctx.mask = op, loss_mask
+        ctx.dweight_out, ctx.weight_grad_fp32 = dweight_out, weight_grad_fp32
+        ctx.save_for_backward(hidden, weight)
+        return op.loss.clone().squeeze(0)
+
+    @staticmethod
+    def backward(ctx, grad):
+        hidden, weight = ctx.saved_tensors
+        op = ctx.op
+        if ctx.dweight_out is not None:
+            saved, op.dweight = op.dweight, ctx.dweight_out       # dW += into the caller's fp32 buffer
+        try:
+            op.backward(hidden, weight, loss_mask=ctx.mask, grad_loss=float(grad.item()))
+        finally:
+            if ctx.dweight_out is not None:
+                op.dweight = saved
+        code, detail = op.status()
+        if code not in (0, -10):                                  # -10: out-of-range teacher indices were ignored
+            raise B.KdklError(code, f"device status, detail {detail}")
+        if ctx.dweight_out is not None:
+            dW = None
+        elif ctx.weight_grad_fp32:
+            dW = op.dweight
+        else:
+            dW = op.dweight.to(weight.dtype)
+        return op.dhidden.clone(), dW, None, None, None, None, None, None, None, None
+
+
+def fused_chunked_kl(hidden, weight, topk_idx, topk_val, teacher_lse: Optional[torch.Tensor] = None,
+                     loss_mask: Optional[torch.Tensor] = None, chunk: int = 4096, temperature: float = 1.0,
+                     dweight_out: Optional[torch.Tensor] = None, weight_grad_fp32: bool = False) -> torch.Tensor:
+    """Mean forward KL between the cached top-K teacher and softmax(hidden @ weight.T / temperature)."""
+    return _FusedChunkedKL.apply(hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, chunk, temperature,
+                                 dweight_out, weight_grad_fp32)
+
+
+class _FeatureLoss(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, student, teacher, loss_mask, kind, weight):
+        T, H = student.shape
+        ws = torch.empty(B.kdkl_feature_loss_workspace_bytes(T), dtype=torch.uint8, device=student.device)
+        loss = torch.zeros(1, dtype=torch.float32, device=student.device)
+        grad = torch.empty_like(student)
+        # loss and d loss / d student come out of the same pass, for an upstream gradient of 1
+        B.kdkl_feature_loss(student, teacher, ws, loss, kind=kind, loss_mask=loss_mask, weight=weight, dstudent=grad)
+        ctx.save_for_backward(student, teacher, grad, ws)
+        ctx.args = (loss_mask, kind, weight)
+        return loss.squeeze(0)
+
+    @staticmethod
+    def backward(ctx, g):
+        student, teacher, grad, ws = ctx.saved_tensors
+        gl = float(g.item())
+        if gl != 1.0:                              # any other upstream gradient: one more pass of the kernel
+            loss_mask, kind, weight = ctx.args
+            scratch = torch.zeros(1, dtype=torch.float32, device=student.device)
+            B.kdkl_feature_loss(student, teacher, ws, scratch, kind=kind, loss_mask=loss_mask, weight=weight,
+                                grad_loss=gl, dstudent=grad)
+        return grad, None, None, None, None
+
+
+def feature_loss(student, teacher, loss_mask=None, kind=B.FEATURE_MSE, weight=1.0) -> torch.Tensor:
+    """Hidden-state feature loss (MSE or cosine) between student and cached teacher hidden states."""
+    return _FeatureLoss.apply(student, teacher, loss_mask, kind, weight)

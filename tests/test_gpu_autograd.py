@@ -1,0 +1,60 @@
+"""The torch.autograd entry: loss.backward() through the fused kernels against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle.feature_oracle import KIND_COSINE, feature_loss_oracle
+from oracle.kdkl_oracle import kdkl_oracle
+from paper_2608_03796_b200 import inputs as I
+from paper_2608_03796_b200.autograd import feature_loss, fused_chunked_kl
+
+pytestmark = pytest.mark.gpu
+
+
+def _fro(a, b):
+    return np.linalg.norm(a - b) / np.linalg.norm(b)
+
+
+def test_loss_backward_matches_oracle_and_combines_with_the_feature_loss():
+    dev = torch.device("cuda:0")
+    cfg = I.CONFIGS["c1"]
+    d = I.make_inputs(cfg, device=dev)
+    r = I.teacher_hidden(cfg, device=dev)
+    h = d["hidden"].clone().requires_grad_(True)
+    W = d["weight"].clone().requires_grad_(True)
+    kl = fused_chunked_kl(h, W, d["topk_idx"], d["topk_val"], chunk=cfg.chunk, temperature=cfg.tau)
+    ft = feature_loss(h, r, kind=KIND_COSINE, weight=0.3)
+    total = 2.0 * kl + ft                                 # upstream gradients 2 and 1
+    total.backward()
+    hn, Wn = d["hidden"].cpu().double().numpy(), d["weight"].cpu().double().numpy()
+    ok = kdkl_oracle(hn, Wn, d["topk_idx"].cpu().numpy(), d["topk_val"].cpu().numpy(), tau=cfg.tau, grad_loss=2.0)
+    of = feature_loss_oracle(hn, r.cpu().double().numpy(), KIND_COSINE, weight=0.3)
+    want = 2.0 * ok["loss"] + of["loss"]
+    assert abs(total.item() - want) <= 1e-3 * abs(want)
+    assert h.grad.dtype == torch.bfloat16 and W.grad.dtype == torch.bfloat16
+    assert _fro(h.grad.float().cpu().double().numpy(), ok["dH"] + of["dS"]) <= 1e-2
+    assert _fro(W.grad.float().cpu().double().numpy(), ok["dW"]) <= 1e-2
+
+
+def test_main_grad_accumulation_and_second_step_reuses_buffers():
+    dev = torch.device("cuda:0")
+    cfg = I.CONFIGS["c1"]
+    d = I.make_inputs(cfg, device=dev)
+    main_grad = torch.zeros(cfg.V, cfg.H, dtype=torch.float32, device=dev)
+    o = kdkl_oracle(d["hidden"].cpu().double().numpy(), d["weight"].cpu().double().numpy(),
+                    d["topk_idx"].cpu().numpy(), d["topk_val"].cpu().numpy(), tau=cfg.tau)
+    before = None
+    for step in range(2):
+        h = d["hidden"].clone().requires_grad_(True)
+        W = d["weight"].clone().requires_grad_(True)
+        loss = fused_chunked_kl(h, W, d["topk_idx"], d["topk_val"], chunk=cfg.chunk, temperature=cfg.tau,
+                                dweight_out=main_grad)
+        loss.backward()
+        assert W.grad is None                               # dW went into main_grad instead
+        assert abs(loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
+        if step == 0:
+            torch.cuda.synchronize()
+            before = torch.cuda.memory_allocated()
+    torch.cuda.synchronize()
+    assert torch.cuda.memory_allocated() <= before + 2 * d["hidden"].numel() * 2 + 4096   # no new workspace
+    assert _fro(main_grad.cpu().double().numpy(), 2.0 * o["dW"]) <= 1e-2                  # two steps accumulated
