@@ -107,8 +107,33 @@ def _check(rc: int):
         raise KdklError(rc, lib().kdkl_last_error().decode() if rc == -7 else "")
 
 
-def _ptr(t: Optional[torch.Tensor]):
-    return None if t is None else ctypes.c_void_p(t.data_ptr())
+def _dptr(t: Optional[torch.Tensor], dtype=None, shape=None, name="tensor"):
+    """Device pointer of a contiguous CUDA tensor, optionally of a given dtype and shape. Anything else is
+    refused here: the library would hand the address to a kernel as it is, and a narrower element type or a
+    smaller tensor than the kernel assumes would be read out of bounds."""
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise TypeError(f"kdkl: {name}: expected a CUDA tensor, got a tensor on {t.device}")
+    if not t.is_contiguous():
+        raise TypeError(f"kdkl: {name}: expected a contiguous tensor")
+    if dtype is not None and t.dtype not in (dtype if isinstance(dtype, tuple) else (dtype,)):
+        raise TypeError(f"kdkl: {name}: expected dtype {dtype}, got {t.dtype}")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise TypeError(f"kdkl: {name}: expected shape {tuple(shape)}, got {tuple(t.shape)}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+_BF16, _F32, _I32, _U8 = torch.bfloat16, torch.float32, torch.int32, torch.uint8
+
+
+def _hptr(t: Optional[torch.Tensor]):
+    """Host pointer of a contiguous CPU tensor (the host-buffer entry point)."""
+    if t is None:
+        return None
+    if t.is_cuda or not t.is_contiguous():
+        raise TypeError("kdkl: expected a contiguous host tensor")
+    return ctypes.c_void_p(t.data_ptr())
 
 
 def _stream():
@@ -133,19 +158,26 @@ def kdkl_forward(hidden, weight, topk_idx, topk_val, workspace, loss_out, *, tea
     T, H = hidden.shape
     V = weight.shape[0]
     K = topk_idx.shape[1]
-    _check(lib().kdkl_forward(_ptr(hidden), _ptr(weight), _ptr(topk_idx), _ptr(topk_val), _ptr(teacher_lse),
-                              _ptr(loss_mask), T, H, V, K, chunk, temperature, _opt_ptr(opt), _ptr(workspace),
-                              workspace.numel() * workspace.element_size(), _ptr(loss_out), _ptr(loss_per_token),
-                              _ptr(gathered_logits), _ptr(gathered_idx), _stream()))
+    _check(lib().kdkl_forward(_dptr(hidden, _BF16, (T, H), "hidden"), _dptr(weight, _BF16, (V, H), "weight"),
+                              _dptr(topk_idx, _I32, (T, K), "topk_idx"), _dptr(topk_val, _F32, (T, K), "topk_val"),
+                              _dptr(teacher_lse, _F32, (T,), "teacher_lse"), _dptr(loss_mask, _U8, (T,), "loss_mask"),
+                              T, H, V, K, chunk, temperature, _opt_ptr(opt), _dptr(workspace, _U8, None, "workspace"),
+                              workspace.numel(), _dptr(loss_out, _F32, (1,), "loss_out"),
+                              _dptr(loss_per_token, _F32, (T,), "loss_per_token"),
+                              _dptr(gathered_logits, _F32, (T, K), "gathered_logits"),
+                              _dptr(gathered_idx, _I32, (T, K), "gathered_idx"), _stream()))
 
 
 def kdkl_backward(hidden, weight, K, workspace, dhidden, dweight, *, loss_mask=None, chunk=0, temperature=1.0,
                   opt=None, grad_loss=1.0) -> None:
     T, H = hidden.shape
     V = weight.shape[0]
-    _check(lib().kdkl_backward(_ptr(hidden), _ptr(weight), _ptr(loss_mask), T, H, V, K, chunk, temperature,
-                               _opt_ptr(opt), grad_loss, _ptr(workspace),
-                               workspace.numel() * workspace.element_size(), _ptr(dhidden), _ptr(dweight), _stream()))
+    dh_dtype = _F32 if (opt is not None and opt.dhidden_dtype == 1) else _BF16
+    _check(lib().kdkl_backward(_dptr(hidden, _BF16, (T, H), "hidden"), _dptr(weight, _BF16, (V, H), "weight"),
+                               _dptr(loss_mask, _U8, (T,), "loss_mask"), T, H, V, K, chunk, temperature,
+                               _opt_ptr(opt), grad_loss, _dptr(workspace, _U8, None, "workspace"), workspace.numel(),
+                               _dptr(dhidden, dh_dtype, (T, H), "dhidden"), _dptr(dweight, _F32, (V, H), "dweight"),
+                               _stream()))
 
 
 def kdkl_forward_shard(hidden, weight_local, topk_idx, topk_val, workspace, shard_stats, *, vocab_offset, V_total,
@@ -155,33 +187,39 @@ def kdkl_forward_shard(hidden, weight_local, topk_idx, topk_val, workspace, shar
     T, H = hidden.shape
     V_local = weight_local.shape[0]
     K = topk_idx.shape[1]
-    _check(lib().kdkl_forward_shard(_ptr(hidden), _ptr(weight_local), _ptr(topk_idx), _ptr(topk_val),
-                                    _ptr(teacher_lse), _ptr(loss_mask), T, H, V_local, vocab_offset, V_total, K, chunk,
-                                    temperature, _opt_ptr(opt), _ptr(workspace),
-                                    workspace.numel() * workspace.element_size(), _ptr(shard_stats),
-                                    _ptr(gathered_logits), _ptr(gathered_idx), _stream()))
+    _check(lib().kdkl_forward_shard(_dptr(hidden, _BF16, (T, H), "hidden"),
+                                    _dptr(weight_local, _BF16, (V_local, H), "weight_local"),
+                                    _dptr(topk_idx, _I32, (T, K), "topk_idx"), _dptr(topk_val, _F32, (T, K), "topk_val"),
+                                    _dptr(teacher_lse, _F32, (T,), "teacher_lse"),
+                                    _dptr(loss_mask, _U8, (T,), "loss_mask"), T, H, V_local, vocab_offset, V_total, K,
+                                    chunk, temperature, _opt_ptr(opt), _dptr(workspace, _U8, None, "workspace"),
+                                    workspace.numel(), _dptr(shard_stats, _F32, (2, T), "shard_stats"),
+                                    _dptr(gathered_logits, _F32, (T, K), "gathered_logits"),
+                                    _dptr(gathered_idx, _I32, (T, K), "gathered_idx"), _stream()))
 
 
 def kdkl_forward_finish(all_stats, n_shards, T, H, V_local, K, workspace, loss_out, *, loss_mask=None, chunk=0,
                         temperature=1.0, opt=None, loss_per_token=None) -> None:
     """Completes the sharded forward from the gathered statistics [n_shards, 2, T]."""
-    _check(lib().kdkl_forward_finish(_ptr(all_stats), n_shards, _ptr(loss_mask), T, H, V_local, K, chunk, temperature,
-                                     _opt_ptr(opt), _ptr(workspace), workspace.numel() * workspace.element_size(),
-                                     _ptr(loss_out), _ptr(loss_per_token), _stream()))
+    _check(lib().kdkl_forward_finish(_dptr(all_stats, _F32, (n_shards, 2, T), "all_stats"), n_shards,
+                                     _dptr(loss_mask, _U8, (T,), "loss_mask"), T, H, V_local, K, chunk, temperature,
+                                     _opt_ptr(opt), _dptr(workspace, _U8, None, "workspace"), workspace.numel(),
+                                     _dptr(loss_out, _F32, (1,), "loss_out"),
+                                     _dptr(loss_per_token, _F32, (T,), "loss_per_token"), _stream()))
 
 
 def kdkl_status(workspace):
     """(code, [site_or_row, counted_tokens, ignored_indices]); synchronises the current stream."""
     code = ctypes.c_int32(0)
     detail = (ctypes.c_int64 * 3)()
-    _check(lib().kdkl_status(_ptr(workspace), _stream(), ctypes.byref(code), detail))
+    _check(lib().kdkl_status(_dptr(workspace), _stream(), ctypes.byref(code), detail))
     return code.value, list(detail)
 
 
 def kdkl_saved_state(workspace, T, H, V, K, chunk=0, opt=None):
     """Views of the saved log Z [T] and retained mass M [T] inside the workspace."""
     a, b = ctypes.c_void_p(), ctypes.c_void_p()
-    _check(lib().kdkl_saved_state(_ptr(workspace), T, H, V, K, chunk, _opt_ptr(opt), ctypes.byref(a), ctypes.byref(b)))
+    _check(lib().kdkl_saved_state(_dptr(workspace), T, H, V, K, chunk, _opt_ptr(opt), ctypes.byref(a), ctypes.byref(b)))
     base = workspace.data_ptr()
     ws_f = workspace.view(torch.uint8)
     def view(p):
@@ -201,11 +239,11 @@ def kdkl_forward_backward_host(hidden, weight, topk_idx, topk_val, arena, loss_o
     T, H = hidden.shape
     V = weight.shape[0]
     K = topk_idx.shape[1]
-    _check(lib().kdkl_forward_backward_host(_ptr(hidden), _ptr(weight), _ptr(topk_idx), _ptr(topk_val),
-                                            _ptr(teacher_lse), _ptr(loss_mask), T, H, V, K, chunk, temperature,
-                                            _opt_ptr(opt), grad_loss, _ptr(arena),
-                                            arena.numel() * arena.element_size(), _ptr(loss_out), _ptr(dhidden_out),
-                                            _ptr(dweight_out), _stream()))
+    _check(lib().kdkl_forward_backward_host(_hptr(hidden), _hptr(weight), _hptr(topk_idx), _hptr(topk_val),
+                                            _hptr(teacher_lse), _hptr(loss_mask), T, H, V, K, chunk, temperature,
+                                            _opt_ptr(opt), grad_loss, _dptr(arena),
+                                            arena.numel() * arena.element_size(), _hptr(loss_out), _hptr(dhidden_out),
+                                            _hptr(dweight_out), _stream()))
 
 
 STAGES = ["prep", "fwd_gemm_lse", "combine", "loss_reduce", "bwd_coef", "bwd_gemm_dlogits", "dhidden_gemm",
@@ -220,15 +258,15 @@ def kdkl_profile_stages(hidden, weight, topk_idx, topk_val, workspace, loss_out,
     K = topk_idx.shape[1]
     ms = (ctypes.c_float * 8)()
     nl = (ctypes.c_int32 * 8)()
-    _check(lib().kdkl_profile_stages(_ptr(hidden), _ptr(weight), _ptr(topk_idx), _ptr(topk_val), _ptr(teacher_lse),
-                                     _ptr(loss_mask), T, H, V, K, chunk, temperature, _opt_ptr(opt), grad_loss,
-                                     _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(loss_out),
-                                     _ptr(dhidden), _ptr(dweight), _stream(), ms, nl))
+    _check(lib().kdkl_profile_stages(_dptr(hidden), _dptr(weight), _dptr(topk_idx), _dptr(topk_val), _dptr(teacher_lse),
+                                     _dptr(loss_mask), T, H, V, K, chunk, temperature, _opt_ptr(opt), grad_loss,
+                                     _dptr(workspace), workspace.numel() * workspace.element_size(), _dptr(loss_out),
+                                     _dptr(dhidden), _dptr(dweight), _stream(), ms, nl))
     return {STAGES[i]: (float(ms[i]), int(nl[i])) for i in range(8)}
 
 
 def kdkl_gemm_bf16(A, B, C, M, N, K, a_mn=0, b_mn=0, status=None) -> None:
-    _check(lib().kdkl_gemm_bf16(_ptr(A), _ptr(B), _ptr(C), M, N, K, a_mn, b_mn, _ptr(status), _stream()))
+    _check(lib().kdkl_gemm_bf16(_dptr(A), _dptr(B), _dptr(C), M, N, K, a_mn, b_mn, _dptr(status), _stream()))
 
 
 def kdkl_logz_noalloc(hidden, weight, logz_out, temperature=1.0) -> None:
@@ -237,7 +275,7 @@ def kdkl_logz_noalloc(hidden, weight, logz_out, temperature=1.0) -> None:
     pool owns the device, a latency-critical callback). Calls sharing a GPU must not overlap."""
     T, H = hidden.shape
     V = weight.shape[0]
-    _check(lib().kdkl_logz_noalloc(_ptr(hidden), _ptr(weight), T, H, V, temperature, _ptr(logz_out), _stream()))
+    _check(lib().kdkl_logz_noalloc(_dptr(hidden), _dptr(weight), T, H, V, temperature, _dptr(logz_out), _stream()))
 
 
 def kdkl_teacher_topk(hidden, weight, K, temperature=1.0, workspace=None):
@@ -250,8 +288,8 @@ def kdkl_teacher_topk(hidden, weight, K, temperature=1.0, workspace=None):
     idx = torch.empty(T, K, dtype=torch.int32, device=hidden.device)
     val = torch.empty(T, K, dtype=torch.float32, device=hidden.device)
     lse = torch.empty(T, dtype=torch.float32, device=hidden.device)
-    _check(lib().kdkl_teacher_topk(_ptr(hidden), _ptr(weight), T, H, V, K, temperature, _ptr(workspace),
-                                   workspace.numel(), _ptr(idx), _ptr(val), _ptr(lse), _stream()))
+    _check(lib().kdkl_teacher_topk(_dptr(hidden), _dptr(weight), T, H, V, K, temperature, _dptr(workspace),
+                                   workspace.numel(), _dptr(idx), _dptr(val), _dptr(lse), _stream()))
     return idx, val, lse, workspace
 
 
@@ -263,14 +301,17 @@ def kdkl_feature_loss(student, teacher, workspace, loss_out, *, kind=FEATURE_MSE
                       grad_loss=1.0, denom_override=0.0, accumulate=0, loss_per_token=None, dstudent=None) -> None:
     """Hidden-state feature loss (MSE or cosine) and its gradient in one pass; see include/kdkl.h."""
     T, H = student.shape
-    _check(lib().kdkl_feature_loss(_ptr(student), _ptr(teacher), _ptr(loss_mask), T, H, kind, weight, grad_loss,
-                                   denom_override, accumulate, _ptr(workspace), workspace.numel(), _ptr(loss_out),
-                                   _ptr(loss_per_token), _ptr(dstudent), _stream()))
+    _check(lib().kdkl_feature_loss(_dptr(student, _BF16, (T, H), "student"), _dptr(teacher, _BF16, (T, H), "teacher"),
+                                   _dptr(loss_mask, _U8, (T,), "loss_mask"), T, H, kind, weight, grad_loss,
+                                   denom_override, accumulate, _dptr(workspace, _U8, None, "workspace"),
+                                   workspace.numel(), _dptr(loss_out, _F32, (1,), "loss_out"),
+                                   _dptr(loss_per_token, _F32, (T,), "loss_per_token"),
+                                   _dptr(dstudent, _BF16, (T, H), "dstudent"), _stream()))
 
 
 def kdkl_wait_selftest(status, limit_ns: int) -> None:
     """A wait nobody satisfies must expire into status = {KDKL_ERR_TIMEOUT, 99} (see include/kdkl.h)."""
-    _check(lib().kdkl_wait_selftest(_ptr(status), limit_ns, _stream()))
+    _check(lib().kdkl_wait_selftest(_dptr(status), limit_ns, _stream()))
 
 
 def kdkl_last_launch_count() -> int:

@@ -103,3 +103,27 @@ def test_header_is_plain_c99(tmp_path):
                    'return kdkl_workspace_bytes(1, 8, 8, 1, 0, &o) == 0; }\n')
     subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only",
                     "-I", os.path.join(ROOT, "include"), str(src)], check=True)
+
+
+def test_binding_refuses_host_tensors_where_device_pointers_are_expected():
+    """A CPU tensor (or a strided view) handed to a device entry point must raise before the library sees
+    the address: there is no CPU path to fall back to, and a kernel must never get a host pointer."""
+    import pytest
+    import torch
+    from paper_2608_03796_b200 import autograd
+    entry.build()
+    h = torch.zeros(8, 64, dtype=torch.bfloat16)
+    W = torch.zeros(128, 64, dtype=torch.bfloat16)
+    idx = torch.zeros(8, 4, dtype=torch.int32)
+    val = torch.zeros(8, 4)
+    ws = torch.empty(binding.kdkl_workspace_bytes(8, 64, 128, 4), dtype=torch.uint8)
+    loss = torch.zeros(1)
+    with pytest.raises(TypeError):
+        binding.kdkl_forward(h, W, idx, val, ws, loss)
+    with pytest.raises(TypeError):
+        binding.kdkl_feature_loss(h, h, ws, loss)
+    with pytest.raises(TypeError):
+        autograd.fused_chunked_kl(h.requires_grad_(False), W, idx, val)
+    assert binding._dptr(None) is None and binding._hptr(None) is None
+    with pytest.raises(TypeError):
+        binding._hptr(torch.zeros(4, 4).t())          # strided view
