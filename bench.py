@@ -336,7 +336,9 @@ def main():
         d2h = 4 + dh_h.numel() * 2 + dw_h.numel() * 4
         assert abs(float(loss_h.item()) - loss_val) <= 1e-5 * abs(loss_val)
         e2e = {"value": whole_job_tokens_per_s(T, world, e_ms), "unit": "tokens/s", "ms_per_step": e_ms,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
+               "what": "every input (hidden, weight, teacher record, mask) from pinned host memory and loss, dHidden, "
+                       "dWeight back to the host each step: bound by the host link"}
         del arena
 
     # the HBM-bound companion op (hidden-state feature loss, one pass: 2 reads + 1 write of [T,H] bf16), timed at
@@ -365,6 +367,36 @@ def main():
             feature[kname] = {"ms": f_ms, "GBps": gbps, "frac_of_hbm_copy": gbps / feature["hbm_peak_GBps"],
                               "loss": float(fl.item())}
         del fs, fr, fd, fws
+
+    # the step as the offline pipeline feeds it: only the batch's cached teacher record (and mask) comes from the
+    # host every step; hidden states, weight and gradients stay on the device, as in a training loop
+    e2e_record = None
+    if not args.no_e2e and not args.capture:
+        staging = torch.empty(B.kdkl_record_staging_bytes(T, K), dtype=torch.uint8, device=dev)
+        rec = {k: (d[k].cpu().pin_memory() if d[k] is not None else None) for k in ("topk_idx", "topk_val", "mask")}
+        loss_h2 = torch.zeros(1, dtype=torch.float32).pin_memory()
+
+        def record_step():
+            B.kdkl_step_host_record(d["hidden"], d["weight"], rec["topk_idx"], rec["topk_val"], staging, op.workspace,
+                                    loss_h2, op.dhidden, op.dweight, loss_mask_host=rec["mask"], chunk=cfg.chunk,
+                                    temperature=cfg.tau)
+        record_step()
+        barrier()
+        t0 = time.perf_counter()
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        r0.record()
+        for _ in range(args.steps):
+            record_step()
+        r1.record()
+        barrier()
+        r_ms = max(r0.elapsed_time(r1), 1e3 * (time.perf_counter() - t0)) / args.steps
+        r_ms = max_over_ranks(r_ms, world, dev)
+        assert abs(float(loss_h2.item()) - loss_val) <= 1e-5 * abs(loss_val)
+        e2e_record = {"value": whole_job_tokens_per_s(T, world, r_ms), "unit": "tokens/s", "ms_per_step": r_ms,
+                      "h2d_bytes_per_step": sum(v.numel() * v.element_size() for v in rec.values() if v is not None),
+                      "d2h_bytes_per_step": 4, "steps": args.steps,
+                      "what": "teacher record (+ mask) from pinned host memory each step; hidden, weight, gradients resident"}
+        del staging
 
     if rank != 0:
         if world > 1:
@@ -398,6 +430,7 @@ def main():
         "clocks": clk.summary(),
         "gpu_launches": launches_per_step * args.steps,
         "e2e": e2e,
+        "e2e_record_from_host": e2e_record,
         "roofline": {"bound": "tensor", "kernel": dom, "achieved": dom_tflops, "peak": peak, "unit": "TFLOP/s",
                      "frac": dom_tflops / peak, "peak_kind": f"{peak_key} ({peaks.get('_source')})",
                      "traffic": traffic, "ms_per_launch": stages[dom]["ms_per_launch"],

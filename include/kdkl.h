@@ -155,6 +155,22 @@ int kdkl_forward_backward_host(const void* hidden_bf16, const void* weight_bf16,
                                size_t arena_bytes, float* loss_out, void* dhidden_out, float* dweight_out,
                                void* cuda_stream);
 
+/* One step the way the offline pipeline of the paper feeds it (section "Offline Distillation with a Top-K
+ * Teacher": the teacher's top-K record is cached ahead of time and read back per batch): the record of this
+ * batch - topk_idx, topk_val, optional teacher_lse, optional loss_mask - arrives from HOST memory (pinned for
+ * full copy speed), while the student's hidden states, the head weight, both gradients and the workspace live
+ * on the DEVICE, as they do inside a training loop. Copies the record into `staging` (device,
+ * kdkl_record_staging_bytes(T, K) bytes, 256-byte aligned), runs kdkl_forward and kdkl_backward on the stream,
+ * copies the loss to loss_out (HOST, 4 bytes) and synchronises the stream before returning. Errors as the
+ * two calls; device-detected conditions through kdkl_status(workspace). */
+size_t kdkl_record_staging_bytes(int64_t T, int32_t K);
+int kdkl_step_host_record(const void* hidden_bf16, const void* weight_bf16, const int32_t* topk_idx_host,
+                          const float* topk_val_host, const float* teacher_lse_host, const uint8_t* loss_mask_host,
+                          int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, float temperature,
+                          const kdkl_options* opt, float grad_loss, void* staging, size_t staging_bytes,
+                          void* workspace, size_t workspace_bytes, float* loss_out_host, void* dhidden,
+                          float* dweight, void* cuda_stream);
+
 /* Forward + backward on DEVICE buffers with a CUDA event between every kernel; synchronises and
  * returns, per stage, the summed device time in ms and the number of launches. Stages:
  * 0 teacher prep, 1 forward GEMM + online log-sum-exp + gather, 2 partial combine, 3 loss reduce,

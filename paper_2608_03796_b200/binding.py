@@ -27,7 +27,7 @@ EXPORTS = [
     "kdkl_host_arena_bytes", "kdkl_forward_backward_host", "kdkl_profile_stages", "kdkl_gemm_bf16", "kdkl_last_error",
     "kdkl_last_launch_count", "kdkl_logz_noalloc", "kdkl_forward_shard", "kdkl_forward_finish",
     "kdkl_wait_selftest", "kdkl_teacher_topk", "kdkl_teacher_topk_workspace_bytes",
-    "kdkl_feature_loss", "kdkl_feature_loss_workspace_bytes",
+    "kdkl_feature_loss", "kdkl_feature_loss_workspace_bytes", "kdkl_step_host_record", "kdkl_record_staging_bytes",
 ]
 
 FEATURE_MSE, FEATURE_COSINE = 0, 1
@@ -77,6 +77,11 @@ def lib() -> ctypes.CDLL:
     L.kdkl_forward_backward_host.restype = ctypes.c_int
     L.kdkl_forward_backward_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, f32, vp, sz,
                                              vp, vp, vp, vp]
+    L.kdkl_record_staging_bytes.restype = sz
+    L.kdkl_record_staging_bytes.argtypes = [i64, i32]
+    L.kdkl_step_host_record.restype = ctypes.c_int
+    L.kdkl_step_host_record.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, f32, vp, sz, vp, sz,
+                                        vp, vp, vp, vp]
     L.kdkl_profile_stages.restype = ctypes.c_int
     L.kdkl_profile_stages.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, f32, vp, sz,
                                       vp, vp, vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
@@ -244,6 +249,26 @@ def kdkl_forward_backward_host(hidden, weight, topk_idx, topk_val, arena, loss_o
                                             _opt_ptr(opt), grad_loss, _dptr(arena),
                                             arena.numel() * arena.element_size(), _hptr(loss_out), _hptr(dhidden_out),
                                             _hptr(dweight_out), _stream()))
+
+
+def kdkl_record_staging_bytes(T, K) -> int:
+    return lib().kdkl_record_staging_bytes(T, K)
+
+
+def kdkl_step_host_record(hidden, weight, topk_idx_host, topk_val_host, staging, workspace, loss_out_host, dhidden,
+                          dweight, *, teacher_lse_host=None, loss_mask_host=None, chunk=0, temperature=1.0, opt=None,
+                          grad_loss=1.0) -> None:
+    """One step with the cached teacher record (and mask) in HOST memory and everything else on the device."""
+    T, H = hidden.shape
+    V = weight.shape[0]
+    K = topk_idx_host.shape[1]
+    dh_dtype = _F32 if (opt is not None and opt.dhidden_dtype == 1) else _BF16
+    _check(lib().kdkl_step_host_record(
+        _dptr(hidden, _BF16, (T, H), "hidden"), _dptr(weight, _BF16, (V, H), "weight"), _hptr(topk_idx_host),
+        _hptr(topk_val_host), _hptr(teacher_lse_host), _hptr(loss_mask_host), T, H, V, K, chunk, temperature,
+        _opt_ptr(opt), grad_loss, _dptr(staging, _U8, None, "staging"), staging.numel(),
+        _dptr(workspace, _U8, None, "workspace"), workspace.numel(), _hptr(loss_out_host),
+        _dptr(dhidden, dh_dtype, (T, H), "dhidden"), _dptr(dweight, _F32, (V, H), "dweight"), _stream()))
 
 
 STAGES = ["prep", "fwd_gemm_lse", "combine", "loss_reduce", "bwd_coef", "bwd_gemm_dlogits", "dhidden_gemm",

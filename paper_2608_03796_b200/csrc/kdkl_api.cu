@@ -591,6 +591,58 @@ int kdkl_forward_backward_host(const void* hidden, const void* weight, const int
   return KDKL_OK;
 }
 
+// ------------------------------------------------------------------ step with the teacher record on the host
+struct StagingLayout { size_t idx, val, lse, mask, loss, total; };
+static StagingLayout staging_layout(long long T, int K) {
+  StagingLayout S;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = up(o + bytes, 256); return at; };
+  S.idx = take((size_t)T * K * 4);
+  S.val = take((size_t)T * K * 4);
+  S.lse = take((size_t)T * 4);
+  S.mask = take((size_t)T);
+  S.loss = take(256);
+  S.total = o;
+  return S;
+}
+
+size_t kdkl_record_staging_bytes(int64_t T, int32_t K) {
+  if (T < 1 || K < 1) return 0;
+  return staging_layout(T, K).total;
+}
+
+int kdkl_step_host_record(const void* hidden, const void* weight, const int32_t* topk_idx_host,
+                          const float* topk_val_host, const float* teacher_lse_host, const uint8_t* loss_mask_host,
+                          int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, float tau, const kdkl_options* opt,
+                          float grad_loss, void* staging, size_t staging_bytes, void* ws, size_t ws_bytes,
+                          float* loss_out_host, void* dhidden, float* dweight, void* cuda_stream) {
+  if (!topk_idx_host || !topk_val_host || !staging || !loss_out_host) return KDKL_ERR_NULL;
+  if (T < 1 || K < 1) return KDKL_ERR_SHAPE;
+  if ((uintptr_t)staging & 255) return KDKL_ERR_ALIGN;
+  const StagingLayout S = staging_layout(T, K);
+  if (staging_bytes < S.total) return KDKL_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  uint8_t* d = reinterpret_cast<uint8_t*>(staging);
+  KDKL_CUDA(cudaMemcpyAsync(d + S.idx, topk_idx_host, (size_t)T * K * 4, cudaMemcpyHostToDevice, st));
+  KDKL_CUDA(cudaMemcpyAsync(d + S.val, topk_val_host, (size_t)T * K * 4, cudaMemcpyHostToDevice, st));
+  if (teacher_lse_host)
+    KDKL_CUDA(cudaMemcpyAsync(d + S.lse, teacher_lse_host, (size_t)T * 4, cudaMemcpyHostToDevice, st));
+  if (loss_mask_host) KDKL_CUDA(cudaMemcpyAsync(d + S.mask, loss_mask_host, (size_t)T, cudaMemcpyHostToDevice, st));
+  const uint8_t* mask_d = loss_mask_host ? d + S.mask : nullptr;
+  int rc = kdkl_forward(hidden, weight, reinterpret_cast<int32_t*>(d + S.idx), reinterpret_cast<float*>(d + S.val),
+                        teacher_lse_host ? reinterpret_cast<float*>(d + S.lse) : nullptr, mask_d, T, H, V, K, chunk, tau,
+                        opt, ws, ws_bytes, reinterpret_cast<float*>(d + S.loss), nullptr, nullptr, nullptr, cuda_stream);
+  if (rc) return rc;
+  const int64_t fl = g_launches;
+  rc = kdkl_backward(hidden, weight, mask_d, T, H, V, K, chunk, tau, opt, grad_loss, ws, ws_bytes, dhidden, dweight,
+                     cuda_stream);
+  if (rc) return rc;
+  g_launches += fl;
+  KDKL_CUDA(cudaMemcpyAsync(loss_out_host, d + S.loss, 4, cudaMemcpyDeviceToHost, st));
+  KDKL_CUDA(cudaStreamSynchronize(st));
+  return KDKL_OK;
+}
+
 // ------------------------------------------------------------------ per-stage profile
 int kdkl_profile_stages(const void* hidden, const void* weight, const int32_t* topk_idx, const float* topk_val,
                         const float* teacher_lse, const uint8_t* loss_mask, int64_t T, int64_t H, int64_t V, int32_t K,

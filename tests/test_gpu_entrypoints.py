@@ -39,6 +39,36 @@ def test_host_buffer_call_equals_device_calls_bitwise():
     assert e.value.code == -4
 
 
+def test_step_with_the_teacher_record_on_the_host_equals_device_calls_bitwise():
+    """Teacher record + mask from pinned host memory, everything else resident: same bits as the device calls."""
+    import dataclasses
+    dev = torch.device("cuda:0")
+    cfg = dataclasses.replace(I.CONFIGS["c5"], T=1300, H=256, V=4104, chunk=512)       # with the packing mask
+    d = I.make_inputs(cfg)
+    lse = I.partial_mass_lse(cfg, torch.nan_to_num(d["topk_val"]))
+    g = {k: (v.to(dev) if v is not None else None) for k, v in d.items()}
+    op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev)
+    op.forward(g["hidden"], g["weight"], g["topk_idx"], g["topk_val"], teacher_lse=lse.to(dev), loss_mask=g["mask"])
+    op.backward(g["hidden"], g["weight"], loss_mask=g["mask"], grad_loss=0.5)
+    assert op.status()[0] == 0
+    want = (op.loss.item(), op.dhidden.clone(), op.dweight.clone())
+    staging = torch.empty(B.kdkl_record_staging_bytes(cfg.T, cfg.K), dtype=torch.uint8, device=dev)
+    ws = torch.empty_like(op.workspace)
+    dh = torch.full_like(op.dhidden, float("nan"))
+    dw = torch.full_like(op.dweight, float("nan"))
+    loss_h = torch.zeros(1).pin_memory()
+    B.kdkl_step_host_record(g["hidden"], g["weight"], d["topk_idx"].pin_memory(), d["topk_val"].pin_memory(), staging,
+                            ws, loss_h, dh, dw, teacher_lse_host=lse.pin_memory(), loss_mask_host=d["mask"].pin_memory(),
+                            chunk=cfg.chunk, temperature=cfg.tau, grad_loss=0.5)
+    assert B.kdkl_status(ws)[0] == 0
+    assert loss_h.item() == want[0] and torch.equal(dh, want[1]) and torch.equal(dw, want[2])
+    assert B.kdkl_last_launch_count() == op.launches
+    with pytest.raises(B.KdklError) as e:
+        B.kdkl_step_host_record(g["hidden"], g["weight"], d["topk_idx"].pin_memory(), d["topk_val"].pin_memory(),
+                                staging[:1024], ws, loss_h, dh, dw, chunk=cfg.chunk, temperature=cfg.tau)
+    assert e.value.code == -4
+
+
 def test_profile_stages_accounts_for_every_launch_and_changes_nothing():
     cfg = I.CONFIGS["c1"]
     d = I.make_inputs(cfg)
