@@ -32,7 +32,8 @@ namespace kdkl {
 constexpr int BM = 128, BN = 256, BK = 64;   // per-CTA accumulator: 128 TMEM lanes x 256 fp32 columns
 constexpr int UMMA_K = 16;
 constexpr int GEMM_THREADS = 192;
-constexpr int MAX_LIVE_KB = 512;               // k-block skipping is available for contractions up to 512 k-blocks
+constexpr int MAX_LIVE_KB = 128;               // k-block skipping: 32 row-tile flags = at most 8192 tokens = 128 k-blocks
+constexpr int MAX_LIVE_M = 256;                // row-tile skipping for launches of up to 256 row tiles
 constexpr int TMEM_COLS = 512;
 constexpr int STAGING_WARP_BYTES = 2 * 4096;   // per epilogue warp: two 32-row x 128-byte output boxes
 constexpr int STAGING_BYTES = 4 * STAGING_WARP_BYTES;
@@ -50,7 +51,7 @@ struct GemmCfg {
   static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
   static constexpr int STAGES = 4;   // measured: 3 starves the tensor pipe, 5 and 6 are no faster than 4
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ +
-                                    2 * MAX_LIVE_KB /*live k-block list*/;
+                                    2 * MAX_LIVE_KB /*live k-block list*/ + 2 * MAX_LIVE_M /*live row-tile list*/;
 };
 
 enum { EPI_STORE_F32 = 0, EPI_STORE_BF16 = 1, EPI_LSE = 2, EPI_DLOGITS = 3, EPI_TOPK = 4 };
@@ -65,8 +66,9 @@ struct GemmParams {
   int* status;               // device status word pair {code, where}
   const int* go;             // optional: kernel returns at once when *go == 0
   // Skipping work for ignored tokens (both optional, one flag per TILE_M rows, 0 = every token of
-  // that row tile is ignored). m_live [m_tiles]: a dead row tile of D is not computed - LSE / TOPK
-  // write nothing for it, the store epilogues write zeros (nothing when accumulating). k_live
+  // that row tile is ignored). m_live [m_tiles] (m_tiles <= MAX_LIVE_M): a dead row tile of D is not
+  // computed - LSE / TOPK write nothing for it, the store epilogues write zeros (nothing when
+  // accumulating); the work units are numbered over the live tiles only, so the workers stay balanced. k_live
   // [ceil(K / TILE_M)] (at most 32 flags, k_splits must be 1): dead k-blocks of the contraction are not
   // loaded or multiplied (their A columns are zeros by construction); if all are dead the first one is
   // processed, so that the accumulator is defined.
@@ -192,13 +194,34 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       *n_live_kb = n;
     }
   }
+  // Dead row tiles: another warp writes the live row tiles (ascending) to the front of a list and the
+  // dead ones to its back. Units are then numbered over the live tiles only - with the static
+  // round-robin assignment, skipping dead units in place would leave some workers with twice the work.
+  const bool mskip = p.m_live != nullptr;
+  uint16_t* live_m = live_kb + MAX_LIVE_KB;
+  volatile int* n_live_m = reinterpret_cast<volatile int*>(tmem_slot + 3);
+  if (mskip && warp == 3) {
+    int n = 0, nd = 0;
+    for (int base = 0; base < p.m_tiles; base += 32) {
+      const int t = base + lane;
+      const uint32_t bits = __ballot_sync(0xffffffffu, t < p.m_tiles && p.m_live[t] != 0);
+      if (lane == 0) {
+        for (int j = 0; j < 32 && base + j < p.m_tiles; ++j) {
+          if ((bits >> j) & 1u) live_m[n++] = (uint16_t)(base + j);
+          else live_m[p.m_tiles - 1 - nd++] = (uint16_t)(base + j);
+        }
+      }
+    }
+    if (lane == 0) *n_live_m = n;
+  }
   tc_fence_before();
   __syncthreads();
   if (NCTA == 2) cluster_sync_all();   // the peer's barriers exist before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int num_tiles = p.m_tiles * p.n_tiles;
+  const int m_count = mskip ? *n_live_m : p.m_tiles;      // row tiles that are computed
+  const int num_tiles = m_count * p.n_tiles;
   const int kblocks = (p.K + BK - 1) / BK;
   // work units: unit u = split * num_tiles + tile; a unit contracts k-blocks [kb0, kb1)
   const int num_units = num_tiles * p.k_splits;
@@ -211,8 +234,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   };
 
   auto tile_coords = [&](int tile, int& mt, int& nt) {
-    if (p.m_inner) { mt = tile % p.m_tiles; nt = tile / p.m_tiles; }
+    if (p.m_inner) { mt = tile % m_count; nt = tile / m_count; }
     else           { nt = tile % p.n_tiles; mt = tile / p.n_tiles; }
+    if (mskip) mt = live_m[mt];
   };
 
   if (warp == 0) {
@@ -228,7 +252,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int tile, split, kb0, kb1, mt, nt;
         unit_decode(unit, tile, split, kb0, kb1);
         tile_coords(tile, mt, nt);
-        if (p.m_live != nullptr && !p.m_live[mt]) continue;   // dead row tile: all three roles skip it alike
         const int m0 = mt * TILE_M + (int)cta_rank * BM;      // this CTA's rows of A
         const int n0 = nt * BN + (int)cta_rank * B_ROWS;      // this CTA's rows of B
         const int nkb = kskip ? *n_live_kb : kb1 - kb0;
@@ -302,7 +325,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int tile, split, kb0, kb1, mt, nt;
         unit_decode(unit, tile, split, kb0, kb1);
         tile_coords(tile, mt, nt);
-        if (p.m_live != nullptr && !p.m_live[mt]) continue;
         const uint32_t acc = lt & 1u;
         const uint32_t aph = (lt >> 1) & 1u;
         if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
@@ -334,37 +356,42 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     constexpr bool kBf16Out = (EPI == EPI_STORE_BF16 || EPI == EPI_DLOGITS);
     uint32_t lt = 0, nbox = 0;
     bool ok = true;
+    // Dead row tiles (every token ignored) belong to no work unit. LSE / TOPK have nothing to write for
+    // them; a store epilogue writes their part of the output as zeros (nothing when it would add them),
+    // for every split's slab, before it turns to the computed tiles.
+    if (mskip && (EPI == EPI_STORE_F32 || EPI == EPI_STORE_BF16 || EPI == EPI_DLOGITS) &&
+        !(EPI == EPI_STORE_F32 && p.accumulate)) {
+      const int n_dead = p.m_tiles - m_count;
+      const int zero_units = n_dead * p.n_tiles * p.k_splits;
+      constexpr int BOX_COLS = (EPI == EPI_STORE_F32) ? 32 : 64;
+      for (int zu = worker; zu < zero_units; zu += num_workers) {
+        const int split = zu / (n_dead * p.n_tiles);
+        const int rem = zu - split * (n_dead * p.n_tiles);
+        const int mt = live_m[m_count + rem / p.n_tiles], nt = rem % p.n_tiles;
+        const int r0 = mt * TILE_M + (int)cta_rank * BM + lg * 32, n0 = nt * BN;
+        if (r0 >= p.M) continue;
+        // zero boxes through the same staging / bulk-group protocol as the regular output path
+        for (int c0 = n0; c0 < n0 + BN && c0 < p.N; c0 += BOX_COLS) {
+          const uint32_t sbox = staging0 + (warp - 2) * STAGING_WARP_BYTES + (nbox & 1u) * 4096u;
+          if (lane == 0) bulk_wait_read<1>();
+          __syncwarp();
+#pragma unroll
+          for (int c = 0; c < 8; ++c) st_shared_v4(sbox + lane * 128 + (c << 4), 0u, 0u, 0u, 0u);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&tmC, sbox, c0, r0 + split * p.split_rows);
+            bulk_commit();
+          }
+          ++nbox;
+        }
+      }
+    }
     for (int unit = worker; unit < num_units && ok; unit += num_workers) {
       int tile, split, kb0, kb1, mt, nt;
       unit_decode(unit, tile, split, kb0, kb1);
       tile_coords(tile, mt, nt);
-      // A dead row tile (every token ignored) was skipped by the producer and the MMA issuer: no
-      // accumulator belongs to it. LSE / TOPK have nothing to write; a store epilogue writes zeros,
-      // or nothing when it would add them.
       const int m0 = mt * TILE_M + (int)cta_rank * BM, n0 = nt * BN;   // this CTA's 128 x 256 part of D
-      if (p.m_live != nullptr && !p.m_live[mt]) {
-        if (EPI == EPI_STORE_F32 || EPI == EPI_STORE_BF16 || EPI == EPI_DLOGITS) {
-          if (!(EPI == EPI_STORE_F32 && p.accumulate) && m0 + lg * 32 < p.M) {
-            // zero boxes through the same staging / bulk-group protocol as the regular output path
-            constexpr int BOX_COLS = (EPI == EPI_STORE_F32) ? 32 : 64;
-            for (int c0 = n0; c0 < n0 + BN && c0 < p.N; c0 += BOX_COLS) {
-              const uint32_t sbox = staging0 + (warp - 2) * STAGING_WARP_BYTES + (nbox & 1u) * 4096u;
-              if (lane == 0) bulk_wait_read<1>();
-              __syncwarp();
-#pragma unroll
-              for (int c = 0; c < 8; ++c) st_shared_v4(sbox + lane * 128 + (c << 4), 0u, 0u, 0u, 0u);
-              fence_proxy_async_smem();
-              __syncwarp();
-              if (lane == 0) {
-                tma_store_2d(&tmC, sbox, c0, m0 + lg * 32 + split * p.split_rows);
-                bulk_commit();
-              }
-              ++nbox;
-            }
-          }
-        }
-        continue;
-      }
       const int row = m0 + row_in_tile;
       const bool row_ok = row < p.M;
       const uint32_t acc = lt & 1u;

@@ -325,7 +325,7 @@ static int forward_impl(const void* hidden, const void* weight, const int32_t* t
     p.part_m = at<float>(ws, L.part_m); p.part_s = at<float>(ws, L.part_s); p.part_stride = L.Cpad;
     p.zg = at<float>(ws, L.zg) + s0 * K;
     p.colread = at<int>(ws, L.colread) + s0 * K;
-    p.m_live = live ? live + fci * L.tiles_per_chunk : nullptr;
+    p.m_live = (live && p.m_tiles <= MAX_LIVE_M) ? live + fci * L.tiles_per_chunk : nullptr;
     stage_mark(ST_F1, st);
     if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA /*no output map*/, p, di.sm_count, st))) return rc;
     stage_mark(ST_COMBINE, st);
@@ -447,7 +447,9 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p.coefA = at<float>(ws, L.coefA) + s0;
     p.coefB = at<float>(ws, L.coefB) + s0;
     p.neg_a = grad_loss < 0.f ? 1 : 0;
-    p.m_live = live_c;                 // dead row tiles of G are written as zeros without being computed
+    // dead row tiles of G are written as zeros without being computed (up to MAX_LIVE_M row tiles per chunk)
+    const uint8_t* live_m = (live_c && p.m_tiles <= MAX_LIVE_M) ? live_c : nullptr;
+    p.m_live = live_m;
     CUtensorMap tmGout;
     if ((rc = make_tmap_out_bf16(&tmGout, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad))) return rc;
     stage_mark(ST_B1, st);
@@ -462,7 +464,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p2.m_tiles = (int)((rows + kTileM - 1) / kTileM); p2.n_tiles = (int)((H + BN - 1) / BN); p2.m_inner = 0;
     p2.status = &hdr->status; p2.go = go;
     p2.accumulate = 0;
-    p2.m_live = live_c;                // their dH rows are zeros
+    p2.m_live = live_m;                // their dH rows are zeros
     // a short last chunk may want a different split; never more than the workspace was sized for
     int sp = choose_k_splits((long long)p2.m_tiles * p2.n_tiles, (V + BK - 1) / BK);
     if (sp > L.dh_splits) sp = L.dh_splits;
