@@ -60,3 +60,33 @@ def test_step_replays_from_a_cuda_graph():
     e2.record()
     torch.cuda.synchronize()
     print(f"c1 step: eager {e0.elapsed_time(e1) / 20:.3f} ms, graph replay {e1.elapsed_time(e2) / 20:.3f} ms")
+
+
+def test_runs_on_a_side_stream_with_identical_bits():
+    """Everything is enqueued on the caller's stream: a step issued on a non-default stream, with unrelated
+    work on the default stream at the same time, gives the bits of a step on the default stream."""
+    from paper_2608_03796_b200 import inputs as I
+    dev = torch.device("cuda:0")
+    cfg = I.CONFIGS["c1"]
+    d = I.make_inputs(cfg, device=dev)
+    op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev,
+                          want_per_token=True)
+    op.forward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"])
+    op.backward(d["hidden"], d["weight"])
+    torch.cuda.synchronize()
+    ref = (op.loss.clone(), op.loss_per_token.clone(), op.dhidden.clone(), op.dweight.clone())
+    for t in (op.loss, op.loss_per_token, op.dhidden, op.dweight):
+        t.zero_()
+    side = torch.cuda.Stream()
+    noise = torch.randn(4096, 4096, device=dev)
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        op.forward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"])
+        op.backward(d["hidden"], d["weight"])
+    for _ in range(4):
+        noise = noise @ noise.T * 1e-4                    # keeps the default stream busy meanwhile
+    side.synchronize()
+    torch.cuda.synchronize()
+    assert op.status()[0] == 0
+    assert torch.equal(op.loss, ref[0]) and torch.equal(op.loss_per_token, ref[1])
+    assert torch.equal(op.dhidden, ref[2]) and torch.equal(op.dweight, ref[3])
