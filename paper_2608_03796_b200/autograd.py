@@ -22,6 +22,11 @@ from . import binding as B
 _cache: dict = {}
 
 
+def clear_cache() -> None:
+    """Drops the cached workspaces and gradient buffers (one set per shape seen so far)."""
+    _cache.clear()
+
+
 def _holder(T, H, V, K, chunk, tau, accumulate, device) -> B.FusedChunkedKL:
     key = (T, H, V, K, chunk, tau, accumulate, str(device))
     op = _cache.get(key)
