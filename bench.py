@@ -280,6 +280,26 @@ def main():
         return (fixed + per_t + B.kdkl_workspace_bytes(tokens, H, V, K, cfg.chunk)) / 1e9
     mem_model = {str(t): round(allocation_gb(t), 3) for t in (4096, 32768, 65536, 131072, 262144)}
 
+    # the single-pass step (kdkl_forward_backward: three projections instead of four, same memory, same outputs up
+    # to one more bf16 rounding inside G), timed like the headline; reported beside it, not instead of it
+    def step1():
+        op.forward_backward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], loss_mask=d["mask"])
+    for _ in range(n_warm):
+        step1()
+    sp0, sp1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sp0.record()
+    for _ in range(args.steps):
+        step1()
+    sp1.record()
+    barrier()
+    sp_ms = max_over_ranks(sp0.elapsed_time(sp1), world, dev) / args.steps
+    assert op.status()[0] == 0 and abs(float(op.loss.item()) - loss_val) <= 1e-6 * abs(loss_val)
+    single_pass = {"ms_per_step": sp_ms, "tokens_per_s": whole_job_tokens_per_s(T, world, sp_ms),
+                   "flops_executed": 0.75 * cfg.flops, "tflops_executed_per_gpu": 0.75 * cfg.flops / (sp_ms * 1e-3) / 1e12,
+                   "launches_per_step": op.launches,
+                   "what": "forward + backward in one call without the second projection (6*T*H*V flops)"}
+
     # per-kernel times, live, with an event between kernels (a separate short run)
     stage_acc = {}
     n_prof = 1 if args.capture else 3
@@ -429,6 +449,7 @@ def main():
         "loss": loss_val,
         "clocks": clk.summary(),
         "gpu_launches": launches_per_step * args.steps,
+        "single_pass": single_pass,
         "e2e": e2e,
         "e2e_record_from_host": e2e_record,
         "roofline": {"bound": "tensor", "kernel": dom, "achieved": dom_tflops, "peak": peak, "unit": "TFLOP/s",

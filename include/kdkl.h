@@ -102,6 +102,22 @@ int kdkl_backward(const void* hidden_bf16, const void* weight_bf16, const uint8_
                   const kdkl_options* opt, float grad_loss, void* workspace, size_t workspace_bytes,
                   void* dhidden, float* dweight, void* cuda_stream);
 
+/* Forward and backward in one call, with three projections instead of four. The paper's backward recomputes
+ * each chunk's logits (Algorithm 1, "Backward": a second output projection) because it runs as a separate
+ * autograd phase; when the gradient is wanted right away - the loss is the last operation of a training step -
+ * the forward sweep of a chunk can leave the unnormalised exponentials 2^(z log2e / tau - 64) in the chunk's
+ * [chunk, V] bf16 buffer, and as soon as the chunk's log Z is known they are turned, in place, into
+ * G = (M q - p) g / tau (Eq. "grad"). Same workspace, same peak memory, same outputs as kdkl_forward followed
+ * by kdkl_backward up to one more bf16 rounding inside G (scaled logits beyond about +190 overflow the stored
+ * exponential and are reported as KDKL_ERR_NONFINITE through the loss). 6 T H V flops instead of 8 T H V.
+ * Arguments as the two calls; grad_loss must be known here. The workspace afterwards holds the same saved
+ * state (kdkl_saved_state, kdkl_status). Not available for vocabulary shards (log Z needs the exchange first). */
+int kdkl_forward_backward(const void* hidden_bf16, const void* weight_bf16, const int32_t* topk_idx,
+                          const float* topk_val, const float* teacher_lse, const uint8_t* loss_mask, int64_t T,
+                          int64_t H, int64_t V, int32_t K, int64_t chunk, float temperature, const kdkl_options* opt,
+                          float grad_loss, void* workspace, size_t workspace_bytes, float* loss_out,
+                          float* loss_per_token, void* dhidden, float* dweight, void* cuda_stream);
+
 /* Vocabulary-sharded use (the paper's tensor-parallel variant: section "Full Chunked KL Computation", last
  * sentences, and Algorithm 1's "distributed max", "reduce sigma", "reduce dh across shards").
  * Rank r holds the weight rows [vocab_offset, vocab_offset + V_local) of a vocabulary of V_total entries;

@@ -40,11 +40,17 @@ def _holder(T, H, V, K, chunk, tau, accumulate, device) -> B.FusedChunkedKL:
 class _FusedChunkedKL(torch.autograd.Function):
     @staticmethod
     def forward(ctx, hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, chunk, temperature, dweight_out,
-                weight_grad_fp32):
+                weight_grad_fp32, single_pass):
         T, H = hidden.shape
         V, K = weight.shape[0], topk_idx.shape[1]
+        # single pass: the gradients for an upstream gradient of 1 come out of the forward call (three projections
+        # instead of four); it writes dW itself, so it is not combined with accumulation into a caller's buffer
+        ctx.done = bool(single_pass) and dweight_out is None
         op = _holder(T, H, V, K, int(chunk), float(temperature), 1 if dweight_out is not None else 0, hidden.device)
-        op.forward(hidden, weight, topk_idx, topk_val, teacher_lse=teacher_lse, loss_mask=loss_mask)
+        if ctx.done:
+            op.forward_backward(hidden, weight, topk_idx, topk_val, teacher_lse=teacher_lse, loss_mask=loss_mask)
+        else:
+            op.forward(hidden, weight, topk_idx, topk_val, teacher_lse=teacher_lse, loss_mask=loss_mask)
         ctx.op, ctx.mask = op, loss_mask
         ctx.dweight_out, ctx.weight_grad_fp32 = dweight_out, weight_grad_fp32
         ctx.save_for_backward(hidden, weight)
@@ -54,13 +60,15 @@ class _FusedChunkedKL(torch.autograd.Function):
     def backward(ctx, grad):
         hidden, weight = ctx.saved_tensors
         op = ctx.op
-        if ctx.dweight_out is not None:
-            saved, op.dweight = op.dweight, ctx.dweight_out       # dW += into the caller's fp32 buffer
-        try:
-            op.backward(hidden, weight, loss_mask=ctx.mask, grad_loss=float(grad.item()))
-        finally:
+        gl = float(grad.item())
+        if not (ctx.done and gl == 1.0):                          # any other upstream gradient: the recompute path
             if ctx.dweight_out is not None:
-                op.dweight = saved
+                saved, op.dweight = op.dweight, ctx.dweight_out   # dW += into the caller's fp32 buffer
+            try:
+                op.backward(hidden, weight, loss_mask=ctx.mask, grad_loss=gl)
+            finally:
+                if ctx.dweight_out is not None:
+                    op.dweight = saved
         code, detail = op.status()
         if code not in (0, -10):                                  # -10: out-of-range teacher indices were ignored
             raise B.KdklError(code, f"device status, detail {detail}")
@@ -70,15 +78,17 @@ class _FusedChunkedKL(torch.autograd.Function):
             dW = op.dweight
         else:
             dW = op.dweight.to(weight.dtype)
-        return op.dhidden.clone(), dW, None, None, None, None, None, None, None, None
+        return op.dhidden.clone(), dW, None, None, None, None, None, None, None, None, None
 
 
 def fused_chunked_kl(hidden, weight, topk_idx, topk_val, teacher_lse: Optional[torch.Tensor] = None,
                      loss_mask: Optional[torch.Tensor] = None, chunk: int = 4096, temperature: float = 1.0,
-                     dweight_out: Optional[torch.Tensor] = None, weight_grad_fp32: bool = False) -> torch.Tensor:
-    """Mean forward KL between the cached top-K teacher and softmax(hidden @ weight.T / temperature)."""
+                     dweight_out: Optional[torch.Tensor] = None, weight_grad_fp32: bool = False,
+                     single_pass: bool = False) -> torch.Tensor:
+    """Mean forward KL between the cached top-K teacher and softmax(hidden @ weight.T / temperature).
+    single_pass=True computes the gradients during the forward call (kdkl_forward_backward)."""
     return _FusedChunkedKL.apply(hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, chunk, temperature,
-                                 dweight_out, weight_grad_fp32)
+                                 dweight_out, weight_grad_fp32, single_pass)
 
 
 class _FeatureLoss(torch.autograd.Function):

@@ -28,6 +28,7 @@ EXPORTS = [
     "kdkl_last_launch_count", "kdkl_logz_noalloc", "kdkl_forward_shard", "kdkl_forward_finish",
     "kdkl_wait_selftest", "kdkl_teacher_topk", "kdkl_teacher_topk_workspace_bytes",
     "kdkl_feature_loss", "kdkl_feature_loss_workspace_bytes", "kdkl_step_host_record", "kdkl_record_staging_bytes",
+    "kdkl_forward_backward",
 ]
 
 FEATURE_MSE, FEATURE_COSINE = 0, 1
@@ -77,6 +78,9 @@ def lib() -> ctypes.CDLL:
     L.kdkl_forward_backward_host.restype = ctypes.c_int
     L.kdkl_forward_backward_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, f32, vp, sz,
                                              vp, vp, vp, vp]
+    L.kdkl_forward_backward.restype = ctypes.c_int
+    L.kdkl_forward_backward.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, f32, vp, sz, vp, vp,
+                                        vp, vp, vp]
     L.kdkl_record_staging_bytes.restype = sz
     L.kdkl_record_staging_bytes.argtypes = [i64, i32]
     L.kdkl_step_host_record.restype = ctypes.c_int
@@ -183,6 +187,23 @@ def kdkl_backward(hidden, weight, K, workspace, dhidden, dweight, *, loss_mask=N
                                _opt_ptr(opt), grad_loss, _dptr(workspace, _U8, None, "workspace"), workspace.numel(),
                                _dptr(dhidden, dh_dtype, (T, H), "dhidden"), _dptr(dweight, _F32, (V, H), "dweight"),
                                _stream()))
+
+
+def kdkl_forward_backward(hidden, weight, topk_idx, topk_val, workspace, loss_out, dhidden, dweight, *,
+                          teacher_lse=None, loss_mask=None, chunk=0, temperature=1.0, opt=None, grad_loss=1.0,
+                          loss_per_token=None) -> None:
+    """Single-pass forward + backward: three projections instead of four (see include/kdkl.h)."""
+    T, H = hidden.shape
+    V = weight.shape[0]
+    K = topk_idx.shape[1]
+    dh_dtype = _F32 if (opt is not None and opt.dhidden_dtype == 1) else _BF16
+    _check(lib().kdkl_forward_backward(
+        _dptr(hidden, _BF16, (T, H), "hidden"), _dptr(weight, _BF16, (V, H), "weight"),
+        _dptr(topk_idx, _I32, (T, K), "topk_idx"), _dptr(topk_val, _F32, (T, K), "topk_val"),
+        _dptr(teacher_lse, _F32, (T,), "teacher_lse"), _dptr(loss_mask, _U8, (T,), "loss_mask"), T, H, V, K, chunk,
+        temperature, _opt_ptr(opt), grad_loss, _dptr(workspace, _U8, None, "workspace"), workspace.numel(),
+        _dptr(loss_out, _F32, (1,), "loss_out"), _dptr(loss_per_token, _F32, (T,), "loss_per_token"),
+        _dptr(dhidden, dh_dtype, (T, H), "dhidden"), _dptr(dweight, _F32, (V, H), "dweight"), _stream()))
 
 
 def kdkl_forward_shard(hidden, weight_local, topk_idx, topk_val, workspace, shard_stats, *, vocab_offset, V_total,
@@ -374,6 +395,15 @@ class FusedChunkedKL:
                       chunk=self.chunk, temperature=self.temperature, opt=self.opt, grad_loss=grad_loss)
         self.launches += kdkl_last_launch_count()
         return self.dhidden, self.dweight
+
+    def forward_backward(self, hidden, weight, topk_idx, topk_val, teacher_lse=None, loss_mask=None, grad_loss=1.0):
+        """Single-pass step (three projections): loss, dhidden and dweight from one call."""
+        kdkl_forward_backward(hidden, weight, topk_idx, topk_val, self.workspace, self.loss, self.dhidden,
+                              self.dweight, teacher_lse=teacher_lse, loss_mask=loss_mask, chunk=self.chunk,
+                              temperature=self.temperature, opt=self.opt, grad_loss=grad_loss,
+                              loss_per_token=self.loss_per_token)
+        self.launches = kdkl_last_launch_count()
+        return self.loss, self.dhidden, self.dweight
 
     def status(self):
         return kdkl_status(self.workspace)

@@ -174,6 +174,96 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
   if (lane == 0) { nvalid[t] = nv; Mout[t] = msum; Hent[t] = hsum; }
 }
 
+// ------------------------------------------------------------------------------------ single-pass step
+// The single-pass forward + backward needs the divisor of the mean before the first chunk (the
+// two-call path learns it at the end of forward): N = number of counted tokens, or the override.
+__global__ void __launch_bounds__(1024)
+count_tokens_kernel(const uint8_t* __restrict__ mask, long long T, float denom_override, WsHeader* hdr) {
+  __shared__ long long part[32];
+  long long c = 0;
+  if (mask) { for (long long t = threadIdx.x; t < T; t += 1024) c += mask[t] != 0; }
+  else if (threadIdx.x == 0) c = T;
+  for (int o = 16; o; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = c;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    long long n = 0;
+    for (int i = 0; i < 32; ++i) n += part[i];
+    hdr->n_tokens = n;
+    hdr->denom = denom_override > 0.f ? denom_override : (float)n;
+  }
+}
+
+// a_t = g_t M_t / tau, b_t = g_t / tau with g_t = grad_loss * mask_t / N (Eq. "grad"), from the header's divisor.
+__global__ void step_coef_kernel(const float* __restrict__ Mv, const uint8_t* __restrict__ mask, long long T,
+                                 float grad_loss, float inv_tau, float* __restrict__ coefA,
+                                 float* __restrict__ coefB, const WsHeader* __restrict__ hdr) {
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= T) return;
+  const float denom = hdr->denom;
+  const bool counted = mask == nullptr || mask[t] != 0;
+  const float g = (counted && denom > 0.f) ? grad_loss / denom : 0.f;
+  coefA[t] = g * Mv[t] * inv_tau;
+  coefB[t] = g * inv_tau;
+}
+
+// In place, per chunk: the forward sweep left e = 2^(s - bias) (bf16) in the G buffer; with log Z known,
+//   G = a_t * 2^(s - lz2_t) - b_t p = (a_t * 2^(bias - lz2_t)) * e - b_t p at the support      (Eq. "grad")
+// One block per (row, 8192-column segment): the dense scaling is a streaming pass (read + write of the
+// chunk's G: the op is bound by HBM), then the row's support entries inside the segment are patched.
+constexpr int E2G_SEG = 8192;                  // columns per block: 256 threads x 4 vectors of 8
+__global__ void __launch_bounds__(256)
+e_to_g_kernel(__nv_bfloat16* __restrict__ G, long long ldg /* elements per row */, int n_cols /* multiple of 8 */,
+              const float* __restrict__ coefA, const float* __restrict__ coefB, const float* __restrict__ lz2,
+              const int* __restrict__ idx_sorted, const float* __restrict__ p_sorted, const int* __restrict__ nvalid,
+              int Ktop, float bias, int n_seg) {
+  const long long row = blockIdx.x / n_seg;
+  const int c_begin = (int)(blockIdx.x - row * n_seg) * E2G_SEG;
+  const int c_end = c_begin + E2G_SEG < n_cols ? c_begin + E2G_SEG : n_cols;
+  const float a = coefA[row];
+  uint4* g_row = reinterpret_cast<uint4*>(G + row * ldg);
+  const int v_begin = c_begin / 8, v_end = c_end / 8;
+  if (a == 0.f) {                              // ignored token (or zero upstream gradient): exact zeros, nothing read
+    for (int v = v_begin + threadIdx.x; v < v_end; v += 256) g_row[v] = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
+  const float scale = a * exp2f(bias - lz2[row]);
+  uint4 buf[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int v = v_begin + threadIdx.x + i * 256;
+    if (v < v_end) buf[i] = g_row[v];
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int v = v_begin + threadIdx.x + i * 256;
+    if (v < v_end) {
+      __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&buf[i]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 x = __bfloat1622float2(h2[j]);
+        h2[j] = __floats2bfloat162_rn(x.x * scale, x.y * scale);
+      }
+      g_row[v] = buf[i];
+    }
+  }
+  // support entries of this row that fall into the segment (sorted ascending, duplicates merged by prep)
+  const int nv = nvalid[row];
+  if (nv == 0) return;
+  __syncthreads();                             // the block's dense stores are visible to its own later loads
+  const int* ids = idx_sorted + row * Ktop;
+  int lo = 0, hi = nv;
+  while (lo < hi) { const int mid = (lo + hi) >> 1; if (ids[mid] < c_begin) lo = mid + 1; else hi = mid; }
+  const float b = coefB[row];
+  __nv_bfloat16* g_el = G + row * ldg;
+  for (int k = lo + threadIdx.x; k < nv; k += 256) {
+    const int col = ids[k];
+    if (col >= c_end) break;
+    const float pk = p_sorted[row * Ktop + k];
+    if (pk != 0.f) g_el[col] = __float2bfloat16_rn(__bfloat162float(g_el[col]) - b * pk);
+  }
+}
+
 // ------------------------------------------------------------------------------------ live row tiles
 // live[c * tiles_per_chunk + i] = 1 when at least one token of rows [c*chunk + i*tile_rows, ... + tile_rows)
 // (clipped to the chunk and to T) is counted. The GEMM kernels skip row tiles whose flag is 0: a padding

@@ -22,6 +22,8 @@
 //   EPI_DLOGITS     backward: G = a_t * exp(z/tau - logZ) - b_t * p at the support, cast to
 //                   bf16 (Eq. "grad", Algorithm 1 backward)
 //   EPI_TOPK        teacher cache: emits the (column, logit) pairs above a per-row threshold
+//   EPI_LSE_E       EPI_LSE that also stores the unnormalised exponentials 2^(z log2e / tau - 64) in bf16, for the
+//                   single-pass forward + backward (no second projection: G is made from them once log Z is known)
 #pragma once
 #include <cuda_bf16.h>
 
@@ -54,7 +56,11 @@ struct GemmCfg {
                                     2 * MAX_LIVE_KB /*live k-block list*/ + 2 * MAX_LIVE_M /*live row-tile list*/;
 };
 
-enum { EPI_STORE_F32 = 0, EPI_STORE_BF16 = 1, EPI_LSE = 2, EPI_DLOGITS = 3, EPI_TOPK = 4 };
+enum { EPI_STORE_F32 = 0, EPI_STORE_BF16 = 1, EPI_LSE = 2, EPI_DLOGITS = 3, EPI_TOPK = 4, EPI_LSE_E = 5 };
+
+// EPI_LSE_E stores e = 2^(z log2e / tau - kExpBias) in bf16: representable for scaled logits in about
+// [-62, 190] (bf16 has fp32's exponent range), i.e. far below any weight that matters and far above any sane logit.
+constexpr float kExpBias = 64.f;
 
 struct GemmParams {
   int M, N, K;               // valid extents of this launch
@@ -353,14 +359,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int lg = warp & 3;                   // TMEM lane group this warp may read
     const int row_in_tile = lg * 32 + lane;
-    constexpr bool kBf16Out = (EPI == EPI_STORE_BF16 || EPI == EPI_DLOGITS);
+    constexpr bool kBf16Out = (EPI == EPI_STORE_BF16 || EPI == EPI_DLOGITS || EPI == EPI_LSE_E);
+    constexpr bool kLse = (EPI == EPI_LSE || EPI == EPI_LSE_E);
+    constexpr bool kStore = (EPI == EPI_STORE_F32 || kBf16Out);
     uint32_t lt = 0, nbox = 0;
     bool ok = true;
     // Dead row tiles (every token ignored) belong to no work unit. LSE / TOPK have nothing to write for
     // them; a store epilogue writes their part of the output as zeros (nothing when it would add them),
     // for every split's slab, before it turns to the computed tiles.
-    if (mskip && (EPI == EPI_STORE_F32 || EPI == EPI_STORE_BF16 || EPI == EPI_DLOGITS) &&
-        !(EPI == EPI_STORE_F32 && p.accumulate)) {
+    if (mskip && kStore && !(EPI == EPI_STORE_F32 && p.accumulate)) {
       const int n_dead = p.m_tiles - m_count;
       const int zero_units = n_dead * p.n_tiles * p.k_splits;
       constexpr int BOX_COLS = (EPI == EPI_STORE_F32) ? 32 : 64;
@@ -402,7 +409,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int* idxrow = nullptr;
       float row_b = 0.f, row_off = -INFINITY, row_thr = INFINITY;
       if (EPI == EPI_TOPK) { if (row_ok) row_thr = p.thr[row]; }
-      if (EPI == EPI_LSE || EPI == EPI_DLOGITS) {
+      if (kLse || EPI == EPI_DLOGITS) {
         if (row_ok) {
           idxrow = p.idx_sorted + (long long)row * p.Ktop;
           nv = p.nvalid[row];
@@ -437,7 +444,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         tmem_ld_wait();
         const bool full_w = col0 + 32 <= p.N;
 
-        if (EPI == EPI_LSE) {
+        if (kLse) {
           if (row_ok) {
             // gather the student logit at every teacher index that falls in this window
             while (next_idx < col0 + 32) {
@@ -462,7 +469,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             s_run = s_run * ex2_approx(m_run - m_new) + acc_s;
             m_run = m_new;
           }
-        } else if (EPI == EPI_TOPK) {
+        }
+        if (EPI == EPI_TOPK) {
           if (row_ok) {
             // candidates of this window: a bit per column whose scaled logit reaches the row's threshold
             uint32_t hits = 0u;
@@ -481,7 +489,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               }
             }
           }
-        } else {
+        }
+        if (kStore) {
           // Output path: the warp's 32 rows x 128 bytes go to a swizzled shared-memory box (16-byte
           // chunk c of row i sits at chunk c ^ (i & 7), the layout a 128-byte-swizzle tensor map
           // expects) and leave with one TMA store / reduce-add; two boxes alternate.
@@ -501,6 +510,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (EPI == EPI_STORE_BF16) {
 #pragma unroll
               for (int j = 0; j < 16; ++j) v[j] = pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+            } else if (EPI == EPI_LSE_E) {
+              // unnormalised exponentials with a fixed bias: G = A_t * e - b_t p is formed from them later
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                v[j] = pack_bf16x2(ex2_approx(fmaf(__uint_as_float(r[2 * j]), p.scale_log2, -kExpBias)),
+                                   ex2_approx(fmaf(__uint_as_float(r[2 * j + 1]), p.scale_log2, -kExpBias)));
             } else {  // EPI_DLOGITS
               // a_t * 2^(s - lz2) = 2^(s + (log2 a_t - lz2)): the row coefficient rides in the exponent
               // (a_t = 0 for ignored tokens gives -inf, hence exact zeros)
@@ -549,7 +564,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
       ++lt;
 
-      if (EPI == EPI_LSE) {
+      if (kLse) {
         if (row_ok) {
           p.part_m[(long long)nt * p.part_stride + row] = m_run;
           p.part_s[(long long)nt * p.part_stride + row] = s_run;

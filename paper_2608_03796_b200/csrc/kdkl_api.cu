@@ -509,6 +509,151 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
   return KDKL_OK;
 }
 
+// ------------------------------------------------------------------ single-pass forward + backward
+// Same results as kdkl_forward followed by kdkl_backward (up to one more bf16 rounding inside G), with three
+// projections instead of four: the forward sweep of a chunk also stores the unnormalised exponentials of its
+// logits in the chunk's G buffer, and once the chunk's log Z is known they are turned into G in place.
+int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t* topk_idx, const float* topk_val,
+                          const float* teacher_lse, const uint8_t* loss_mask, int64_t T, int64_t H, int64_t V, int32_t K,
+                          int64_t chunk, float tau, const kdkl_options* opt, float grad_loss, void* ws, size_t ws_bytes,
+                          float* loss_out, float* loss_per_token, void* dhidden, float* dweight, void* cuda_stream) {
+  g_launches = 0;
+  if (!topk_idx || !topk_val || !loss_out || !dhidden || !dweight) return KDKL_ERR_NULL;
+  if (((uintptr_t)dhidden & 15) || ((uintptr_t)dweight & 15)) return KDKL_ERR_ALIGN;
+  kdkl_options o;
+  WsLayout L;
+  int rc = check_common(hidden, weight, T, H, V, K, chunk, tau, opt, ws, ws_bytes, &o, &L);
+  if (rc) return rc;
+  DeviceInfo di;
+  if ((rc = device_info(&di))) return rc;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  WsHeader* hdr = at<WsHeader>(ws, L.hdr);
+  const float inv_tau = 1.0f / tau;
+
+  stage_mark(ST_PREP, st);
+  header_reset_kernel<<<1, 32, 0, st>>>(hdr);
+  KDKL_LAUNCHED("header_reset_kernel");
+  const int Kpad = next_pow2(K);
+  const size_t prep_smem = (size_t)PREP_WARPS * Kpad * (4 + 4 + 2);
+  prep_kernel<<<(unsigned)((T + PREP_WARPS - 1) / PREP_WARPS), PREP_WARPS * 32, prep_smem, st>>>(
+      topk_idx, topk_val, teacher_lse, loss_mask, T, (int)V, 0, (int)V, K, Kpad, inv_tau, o.teacher_mode,
+      at<int>(ws, L.idx_sorted), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<int>(ws, L.nvalid),
+      at<float>(ws, L.M), at<float>(ws, L.Hent), hdr);
+  KDKL_LAUNCHED("prep_kernel");
+  const uint8_t* live = nullptr;
+  if (loss_mask != nullptr) {
+    tile_live_kernel<<<(unsigned)((L.n_live + 7) / 8), 256, 0, st>>>(loss_mask, T, L.C, kTileM, (int)L.tiles_per_chunk,
+                                                                    L.n_live, at<uint8_t>(ws, L.live));
+    KDKL_LAUNCHED("tile_live_kernel");
+    live = at<uint8_t>(ws, L.live);
+  }
+  // the divisor of the mean and the per-token gradient coefficients are needed before the first chunk here
+  count_tokens_kernel<<<1, 1024, 0, st>>>(loss_mask, T, o.denom_override, hdr);
+  KDKL_LAUNCHED("count_tokens_kernel");
+  step_coef_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(at<float>(ws, L.M), loss_mask, T, grad_loss, inv_tau,
+                                                                at<float>(ws, L.coefA), at<float>(ws, L.coefB), hdr);
+  KDKL_LAUNCHED("step_coef_kernel");
+
+  __nv_bfloat16* G = at<__nv_bfloat16>(ws, L.G);
+  CUtensorMap tmW, tmWmn, tmdW;
+  if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, kBRows))) return rc;
+  if ((rc = make_tmap_bf16(&tmWmn, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, 64, BK))) return rc;
+  if ((rc = make_tmap_out_f32(&tmdW, dweight, (uint64_t)H, (uint64_t)V, (uint64_t)H))) return rc;
+
+  long long ci = 0;
+  for (long long s0 = 0; s0 < T; s0 += L.C, ++ci) {
+    const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
+    const uint8_t* live_c = live ? live + ci * L.tiles_per_chunk : nullptr;
+    const __nv_bfloat16* hA = reinterpret_cast<const __nv_bfloat16*>(hidden) + s0 * H;
+    CUtensorMap tmA, tmGout, tmG, tmGmn, tmhmn, tmdH;
+    if ((rc = make_tmap_bf16(&tmA, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, BK, BM))) return rc;
+    if ((rc = make_tmap_out_bf16(&tmGout, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad))) return rc;
+
+    // F1': logits tile by tile -> online log-sum-exp partials, gathered teacher logits, and e = 2^(s - bias) into G
+    GemmParams p;
+    memset(&p, 0, sizeof(p));
+    p.M = (int)rows; p.N = (int)V; p.K = (int)H;
+    p.m_tiles = (int)((rows + kTileM - 1) / kTileM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1; p.k_splits = 1;
+    p.status = &hdr->status; p.go = nullptr;
+    p.scale_log2 = kLog2e * inv_tau; p.Ktop = K;
+    p.idx_sorted = at<int>(ws, L.idx_sorted) + s0 * K;
+    p.nvalid = at<int>(ws, L.nvalid) + s0;
+    p.part_m = at<float>(ws, L.part_m); p.part_s = at<float>(ws, L.part_s); p.part_stride = L.Cpad;
+    p.zg = at<float>(ws, L.zg) + s0 * K;
+    p.colread = at<int>(ws, L.colread) + s0 * K;
+    const uint8_t* live_m = (live_c && p.m_tiles <= MAX_LIVE_M) ? live_c : nullptr;
+    p.m_live = live_m;
+    stage_mark(ST_F1, st);
+    if ((rc = launch_gemm<EPI_LSE_E, false, false>(tmA, tmW, tmGout, p, di.sm_count, st))) return rc;
+    stage_mark(ST_COMBINE, st);
+    combine_kernel<<<(unsigned)((rows + 31) / 32), COMBINE_WARPS * 32, 0, st>>>(
+        at<float>(ws, L.part_m), at<float>(ws, L.part_s), L.Cpad, (int)L.n_tiles_v, (int)rows, s0, K, inv_tau,
+        at<int>(ws, L.nvalid), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<float>(ws, L.zg),
+        at<int>(ws, L.colread), at<float>(ws, L.M), at<float>(ws, L.Hent), loss_mask, at<float>(ws, L.lz2),
+        at<float>(ws, L.logZ), at<float>(ws, L.loss_tok), loss_per_token, nullptr, nullptr, 0, nullptr, T, hdr);
+    KDKL_LAUNCHED("combine_kernel");
+
+    // e -> G in place, now that the chunk's log Z is known
+    stage_mark(ST_B1, st);
+    const int n_cols = (int)(((V + 7) / 8) * 8);
+    const int n_seg = (n_cols + E2G_SEG - 1) / E2G_SEG;
+    e_to_g_kernel<<<(unsigned)(rows * n_seg), 256, 0, st>>>(
+        G, L.Vpad, n_cols, at<float>(ws, L.coefA) + s0, at<float>(ws, L.coefB) + s0, at<float>(ws, L.lz2) + s0,
+        at<int>(ws, L.idx_sorted) + s0 * K, at<float>(ws, L.p_sorted) + s0 * K, at<int>(ws, L.nvalid) + s0, K, kExpBias,
+        n_seg);
+    KDKL_LAUNCHED("e_to_g_kernel");
+
+    // dH[chunk] = G W and dW (+)= G^T h, exactly as in kdkl_backward
+    stage_mark(ST_B2, st);
+    if ((rc = make_tmap_bf16(&tmG, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, BK, BM))) return rc;
+    GemmParams p2;
+    memset(&p2, 0, sizeof(p2));
+    p2.M = (int)rows; p2.N = (int)H; p2.K = (int)V;
+    p2.m_tiles = (int)((rows + kTileM - 1) / kTileM); p2.n_tiles = (int)((H + BN - 1) / BN); p2.m_inner = 0;
+    p2.status = &hdr->status; p2.go = nullptr;
+    p2.m_live = live_m;
+    int sp = choose_k_splits((long long)p2.m_tiles * p2.n_tiles, (V + BK - 1) / BK);
+    if (sp > L.dh_splits) sp = L.dh_splits;
+    p2.k_splits = sp;
+    if (sp > 1) {
+      float* part = at<float>(ws, L.dh_part);
+      p2.split_rows = (int)L.Cpad;
+      if ((rc = make_tmap_out_f32(&tmdH, part, (uint64_t)H, (uint64_t)sp * L.Cpad, (uint64_t)H))) return rc;
+      if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
+      const long long n4 = rows * H / 4;
+      splitk_fixup_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(
+          part, (long long)L.Cpad * H, sp, n4,
+          o.dhidden_dtype == 0 ? reinterpret_cast<__nv_bfloat16*>(dhidden) + s0 * H : nullptr,
+          o.dhidden_dtype == 1 ? reinterpret_cast<float*>(dhidden) + s0 * H : nullptr, nullptr);
+      KDKL_LAUNCHED("splitk_fixup_kernel");
+    } else if (o.dhidden_dtype == 0) {
+      if ((rc = make_tmap_out_bf16(&tmdH, reinterpret_cast<__nv_bfloat16*>(dhidden) + s0 * H, (uint64_t)H,
+                                   (uint64_t)rows, (uint64_t)H))) return rc;
+      if ((rc = launch_gemm<EPI_STORE_BF16, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
+    } else {
+      if ((rc = make_tmap_out_f32(&tmdH, reinterpret_cast<float*>(dhidden) + s0 * H, (uint64_t)H, (uint64_t)rows,
+                                  (uint64_t)H))) return rc;
+      if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
+    }
+    if ((rc = make_tmap_bf16(&tmGmn, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, 64, BK))) return rc;
+    if ((rc = make_tmap_bf16(&tmhmn, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, 64, BK))) return rc;
+    GemmParams p3;
+    memset(&p3, 0, sizeof(p3));
+    p3.M = (int)V; p3.N = (int)H; p3.K = (int)rows;
+    p3.m_tiles = (int)((V + kTileM - 1) / kTileM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0; p3.k_splits = 1;
+    p3.status = &hdr->status; p3.go = nullptr;
+    p3.accumulate = (ci > 0 || o.accumulate_dweight) ? 1 : 0;
+    p3.k_live = (rows <= 32ll * kTileM && (rows + BK - 1) / BK <= MAX_LIVE_KB) ? live_c : nullptr;
+    stage_mark(ST_B3, st);
+    if ((rc = launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, tmdW, p3, di.sm_count, st))) return rc;
+  }
+  stage_mark(ST_REDUCE, st);
+  loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, tau, H, V, K,
+                                         loss_out, hdr);
+  KDKL_LAUNCHED("loss_reduce_kernel");
+  return KDKL_OK;
+}
+
 int kdkl_status(const void* ws, void* cuda_stream, int32_t* code, int64_t* detail) {
   if (!ws || !code) return KDKL_ERR_NULL;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);

@@ -58,3 +58,20 @@ def test_main_grad_accumulation_and_second_step_reuses_buffers():
     torch.cuda.synchronize()
     assert torch.cuda.memory_allocated() <= before + 2 * d["hidden"].numel() * 2 + 4096   # no new workspace
     assert _fro(main_grad.cpu().double().numpy(), 2.0 * o["dW"]) <= 1e-2                  # two steps accumulated
+
+
+def test_single_pass_autograd_matches_oracle():
+    dev = torch.device("cuda:0")
+    cfg = I.CONFIGS["c1"]
+    d = I.make_inputs(cfg, device=dev)
+    o = kdkl_oracle(d["hidden"].cpu().double().numpy(), d["weight"].cpu().double().numpy(),
+                    d["topk_idx"].cpu().numpy(), d["topk_val"].cpu().numpy(), tau=cfg.tau)
+    for scale in (1.0, 3.0):                               # 3.0 takes the recompute path in backward
+        h = d["hidden"].clone().requires_grad_(True)
+        W = d["weight"].clone().requires_grad_(True)
+        loss = fused_chunked_kl(h, W, d["topk_idx"], d["topk_val"], chunk=cfg.chunk, temperature=cfg.tau,
+                                single_pass=True)
+        (scale * loss).backward()
+        assert abs(loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
+        assert _fro(h.grad.float().cpu().double().numpy(), scale * o["dH"]) <= 1e-2
+        assert _fro(W.grad.float().cpu().double().numpy(), scale * o["dW"]) <= 1e-2

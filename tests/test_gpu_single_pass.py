@@ -1,0 +1,112 @@
+"""kdkl_forward_backward (single pass, three projections) against the fp64 oracle and against the two-call path.
+
+Same tolerances as the two-call path: the only arithmetic difference is one more bf16 rounding inside G
+(the stored exponential, 2^-9 relative), so the gradient error stays well inside the 1e-2 Frobenius bound;
+loss, per-token loss and log Z come from the same sweep and must be bitwise those of kdkl_forward.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle.kdkl_oracle import kdkl_oracle
+from paper_2608_03796_b200 import binding as B
+from paper_2608_03796_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+def _fro(a, b):
+    nb = np.linalg.norm(b)
+    return np.linalg.norm(a - b) / nb if nb > 0 else np.linalg.norm(a)
+
+
+def _case(T, H, V, K, seed, mask_mode=0, dup=False):
+    g = torch.Generator().manual_seed(seed)
+    h = torch.randn(T, H, generator=g).to(torch.bfloat16)
+    W = (torch.randn(V, H, generator=g) / H ** 0.5).to(torch.bfloat16)
+    idx = (torch.randint(0, V, (T, K), generator=g) if dup
+           else torch.stack([torch.randperm(V, generator=g)[:K] for _ in range(T)])).to(torch.int32)
+    val = (torch.randn(T, K, generator=g) * 3 ** 0.5).float()
+    mask = None
+    if mask_mode:
+        mask = (torch.rand(T, generator=g) >= 0.15).to(torch.uint8)
+        if mask_mode == 2 and T > 600:
+            mask[100:100 + 300] = 0                       # a dead run that covers a whole row tile
+        idx[mask == 0] = -1
+        val[mask == 0] = float("nan")
+    return h, W, idx.contiguous(), val.contiguous(), mask
+
+
+@pytest.mark.parametrize("T,H,V,K,chunk,tau,mask_mode,dup,opts", [
+    (256, 256, 4096, 16, 64, 1.0, 0, False, {}),
+    (261, 264, 4120, 9, 100, 1.3, 1, False, {"grad_loss": 0.7, "partial": True}),
+    (700, 72, 1001, 7, 256, 0.5, 2, True, {"grad_loss": -2.0}),
+    (1300, 128, 3000, 33, 0, 2.0, 2, False, {"dh32": 1, "accumulate": 1}),
+    (5, 8, 9, 9, 1, 1.0, 0, False, {}),
+])
+def test_single_pass_matches_oracle_and_two_call_path(T, H, V, K, chunk, tau, mask_mode, dup, opts):
+    dev = torch.device("cuda:0")
+    h, W, idx, val, mask = _case(T, H, V, K, seed=T + V, mask_mode=mask_mode, dup=dup)
+    gl = opts.get("grad_loss", 1.0)
+    lse = None
+    if opts.get("partial"):
+        lse = torch.logsumexp(torch.nan_to_num(val).double() / tau, 1).float() + 0.3
+    opt = B.make_options(dhidden_dtype=opts.get("dh32", 0), accumulate_dweight=opts.get("accumulate", 0))
+    to = lambda x: None if x is None else x.to(dev)
+    base = torch.randn(V, H, generator=torch.Generator().manual_seed(7)) * 1e-4
+    # two-call path
+    two = B.FusedChunkedKL(T, H, V, K, chunk=chunk, temperature=tau, opt=opt, device=dev, want_per_token=True)
+    two.dweight.copy_(base)
+    two.forward(to(h), to(W), to(idx), to(val), teacher_lse=to(lse), loss_mask=to(mask))
+    two.backward(to(h), to(W), loss_mask=to(mask), grad_loss=gl)
+    # single pass
+    one = B.FusedChunkedKL(T, H, V, K, chunk=chunk, temperature=tau, opt=opt, device=dev, want_per_token=True)
+    one.dhidden.fill_(float("nan"))
+    one.dweight.copy_(base) if opts.get("accumulate") else one.dweight.fill_(float("nan"))
+    one.forward_backward(to(h), to(W), to(idx), to(val), teacher_lse=to(lse), loss_mask=to(mask), grad_loss=gl)
+    assert one.status()[0] == 0 and two.status()[0] == 0
+    assert torch.equal(one.loss, two.loss) and torch.equal(one.loss_per_token, two.loss_per_token)
+    assert torch.equal(one.saved_state()[0], two.saved_state()[0])
+    mask_np = None if mask is None else mask.numpy()
+    with np.errstate(all="ignore"):
+        o = kdkl_oracle(h.double().numpy(), W.double().numpy(), idx.numpy(), val.numpy(), tau=tau, mask=mask_np,
+                        teacher_lse=None if lse is None else lse.double().numpy(), grad_loss=gl)
+    assert abs(one.loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
+    dH = one.dhidden.float().cpu().double().numpy()
+    dW = one.dweight.cpu().double().numpy()
+    want_dW = o["dW"] + (base.double().numpy() if opts.get("accumulate") else 0.0)
+    assert np.isfinite(dH).all() and np.isfinite(dW).all()
+    assert _fro(dH, o["dH"]) <= 1e-2 and _fro(dW, want_dW) <= 1e-2
+    if mask is not None:
+        assert not dH[mask_np == 0].any()
+    # and close to the two-call gradients (two independent roundings of G against one)
+    assert _fro(dH, two.dhidden.float().cpu().double().numpy()) <= 6e-3
+    assert _fro(dW, two.dweight.cpu().double().numpy()) <= 6e-3
+
+
+def test_single_pass_fullsize_sampled():
+    """The benchmark shape: per-token outputs bitwise equal to the two-call path, dH rows on sampled tokens
+    against the oracle, column sums of dW vanish, two runs bit for bit."""
+    dev = torch.device("cuda:0")
+    cfg = I.CONFIGS["c2"]
+    d = I.make_inputs(cfg, device=dev)
+    two = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev,
+                           want_per_token=True)
+    two.forward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"])
+    tok2 = two.loss_per_token.clone()
+    del two
+    one = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev,
+                           want_per_token=True)
+    one.forward_backward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"])
+    assert one.status()[0] == 0
+    assert torch.equal(one.loss_per_token, tok2)
+    first = (one.dhidden.clone(), one.dweight.clone())
+    one.forward_backward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"])
+    assert torch.equal(one.dhidden, first[0]) and torch.equal(one.dweight, first[1])
+    R = I.sample_rows(cfg, 32).to(dev)
+    o = kdkl_oracle(d["hidden"][R].cpu().double().numpy(), d["weight"].cpu().double().numpy(),
+                    d["topk_idx"][R].cpu().numpy(), d["topk_val"][R].cpu().numpy(), tau=cfg.tau, denom=cfg.T)
+    assert _fro(one.dhidden[R].float().cpu().double().numpy(), o["dH"]) <= 1e-2
+    colsum = one.dweight.double().sum(0).abs()
+    colabs = one.dweight.double().abs().sum(0)
+    assert (colsum / colabs).max().item() < 3e-3
