@@ -108,8 +108,9 @@ int kdkl_backward(const void* hidden_bf16, const void* weight_bf16, const uint8_
  * the forward sweep of a chunk can leave the unnormalised exponentials 2^(z log2e / tau - 64) in the chunk's
  * [chunk, V] bf16 buffer, and as soon as the chunk's log Z is known they are turned, in place, into
  * G = (M q - p) g / tau (Eq. "grad"). Same workspace, same peak memory, same outputs as kdkl_forward followed
- * by kdkl_backward up to one more bf16 rounding inside G (scaled logits beyond about +190 overflow the stored
- * exponential and are reported as KDKL_ERR_NONFINITE through the loss). 6 T H V flops instead of 8 T H V.
+ * by kdkl_backward up to one more bf16 rounding inside G. A scaled logit z log2e / tau beyond about +190 overflows
+ * the stored exponential: the gradients are then not finite and kdkl_status reports KDKL_ERR_NONFINITE with the
+ * row (use the two-call path for such inputs). 6 T H V flops instead of 8 T H V.
  * Arguments as the two calls; grad_loss must be known here. The workspace afterwards holds the same saved
  * state (kdkl_saved_state, kdkl_status). Not available for vocabulary shards (log Z needs the exchange first). */
 int kdkl_forward_backward(const void* hidden_bf16, const void* weight_bf16, const int32_t* topk_idx,

@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(256)
 e_to_g_kernel(__nv_bfloat16* __restrict__ G, long long ldg /* elements per row */, int n_cols /* multiple of 8 */,
               const float* __restrict__ coefA, const float* __restrict__ coefB, const float* __restrict__ lz2,
               const int* __restrict__ idx_sorted, const float* __restrict__ p_sorted, const int* __restrict__ nvalid,
-              int Ktop, float bias, int n_seg) {
+              int Ktop, float bias, int n_seg, WsHeader* hdr) {
   const long long row = blockIdx.x / n_seg;
   const int c_begin = (int)(blockIdx.x - row * n_seg) * E2G_SEG;
   const int c_end = c_begin + E2G_SEG < n_cols ? c_begin + E2G_SEG : n_cols;
@@ -228,6 +228,7 @@ e_to_g_kernel(__nv_bfloat16* __restrict__ G, long long ldg /* elements per row *
     return;
   }
   const float scale = a * exp2f(bias - lz2[row]);
+  bool bad = false;                            // an exponential that overflowed bf16 (scaled logit beyond about 190)
   uint4 buf[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -242,11 +243,14 @@ e_to_g_kernel(__nv_bfloat16* __restrict__ G, long long ldg /* elements per row *
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const float2 x = __bfloat1622float2(h2[j]);
-        h2[j] = __floats2bfloat162_rn(x.x * scale, x.y * scale);
+        const float y0 = x.x * scale, y1 = x.y * scale;
+        bad |= !(fabsf(y0) <= 3.0e38f) || !(fabsf(y1) <= 3.0e38f);
+        h2[j] = __floats2bfloat162_rn(y0, y1);
       }
       g_row[v] = buf[i];
     }
   }
+  if (bad) { atomicCAS(&hdr->status, 0, -11); atomicCAS(&hdr->where, 0, (int)row); }
   // support entries of this row that fall into the segment (sorted ascending, duplicates merged by prep)
   const int nv = nvalid[row];
   if (nv == 0) return;

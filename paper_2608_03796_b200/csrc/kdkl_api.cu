@@ -600,7 +600,7 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
     e_to_g_kernel<<<(unsigned)(rows * n_seg), 256, 0, st>>>(
         G, L.Vpad, n_cols, at<float>(ws, L.coefA) + s0, at<float>(ws, L.coefB) + s0, at<float>(ws, L.lz2) + s0,
         at<int>(ws, L.idx_sorted) + s0 * K, at<float>(ws, L.p_sorted) + s0 * K, at<int>(ws, L.nvalid) + s0, K, kExpBias,
-        n_seg);
+        n_seg, hdr);
     KDKL_LAUNCHED("e_to_g_kernel");
 
     // dH[chunk] = G W and dW (+)= G^T h, exactly as in kdkl_backward

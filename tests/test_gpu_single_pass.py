@@ -110,3 +110,24 @@ def test_single_pass_fullsize_sampled():
     colsum = one.dweight.double().sum(0).abs()
     colabs = one.dweight.double().abs().sum(0)
     assert (colsum / colabs).max().item() < 3e-3
+
+
+def test_overflowing_exponential_is_reported_not_hidden():
+    """Scaled logits far beyond the representable range of the stored exponential (about 190): the single-pass
+    call reports KDKL_ERR_NONFINITE with the row; the two-call path, which normalises by the running maximum,
+    handles the same input."""
+    dev = torch.device("cuda:0")
+    T, H, V, K = 40, 64, 512, 4
+    h, W, idx, val, _ = _case(T, H, V, K, seed=3)
+    h[7] = 4.0
+    W[11] = 4.0                                        # z[7, 11] = 4 * 4 * 64 = 1024, scaled 1477
+    one = B.FusedChunkedKL(T, H, V, K, device=dev)
+    one.forward_backward(h.to(dev), W.to(dev), idx.to(dev), val.to(dev))
+    code, detail = one.status()
+    assert code == -11 and detail[0] == 7
+    two = B.FusedChunkedKL(T, H, V, K, device=dev)
+    two.forward(h.to(dev), W.to(dev), idx.to(dev), val.to(dev))
+    two.backward(h.to(dev), W.to(dev))
+    assert two.status()[0] == 0 and torch.isfinite(two.dweight).all() and torch.isfinite(two.dhidden.float()).all()
+    o = kdkl_oracle(h.double().numpy(), W.double().numpy(), idx.numpy(), val.numpy())
+    assert abs(two.loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
