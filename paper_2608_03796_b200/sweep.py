@@ -7,8 +7,9 @@ setting runs in a fresh process so that an out-of-memory failure cannot contamin
 measurements; timing is the mean forward + backward time after warm-up; memory is the peak
 allocated CUDA memory (inputs, outputs and workspace are all torch allocations).
 
-Three methods:
-  fused     the library (kdkl_forward + kdkl_backward)
+Four methods:
+  fused     the library (kdkl_forward + kdkl_backward: the paper's schedule, four projections)
+  single    the library's single-pass step (kdkl_forward_backward: three projections, same memory)
   dense     a plain torch comparator that materialises the [T, V] logits, a dense log-softmax and the
             scattered dense teacher (section "Full Dense KL Computation"). It exists only to show what the
             fused path saves; it is expected to run out of memory at long T, which is recorded as such.
@@ -66,12 +67,15 @@ def worker(method: str, name: str, steps: int) -> dict:
         def step():
             B.kdkl_teacher_topk(d["hidden"], d["weight"], cfg.K, temperature=cfg.tau, workspace=tws)
             return torch.zeros(1)
-    elif method == "fused":
+    elif method in ("fused", "single"):
         op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev)
 
         def step():
-            op.forward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], loss_mask=d["mask"])
-            op.backward(d["hidden"], d["weight"], loss_mask=d["mask"])
+            if method == "single":
+                op.forward_backward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], loss_mask=d["mask"])
+            else:
+                op.forward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], loss_mask=d["mask"])
+                op.backward(d["hidden"], d["weight"], loss_mask=d["mask"])
             return op.loss
         out["workspace_gb"] = op.workspace.numel() / 1e9
     elif method == "fwdchunk":
@@ -143,11 +147,12 @@ def worker(method: str, name: str, steps: int) -> dict:
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / steps
         out.update(ms_per_iter=ms, it_per_s=1e3 / ms, tokens_per_s=cfg.T / (ms * 1e-3),
-                   tflops=(0.5 if method == "teacher" else 1.0) * cfg.flops / (ms * 1e-3) / 1e12,   # teacher: 2 sweeps
+                   # executed projections: fused 4 (8*T*H*V), single / dense / fwdchunk 3, teacher 2
+                   tflops={"fused": 1.0, "teacher": 0.5}.get(method, 0.75) * cfg.flops / (ms * 1e-3) / 1e12,
                    loss=float(loss.item()),
                    peak_gb=torch.cuda.max_memory_allocated() / 1e9,
                    driver_delta_gb=(free0 - torch.cuda.mem_get_info()[0]) / 1e9)
-        if method == "fused":
+        if method in ("fused", "single"):
             code, _ = op.status()
             out["status"] = code
             out["dh_norm"] = float(op.dhidden.float().norm().item())
@@ -166,6 +171,7 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--steps", type=int, default=0)
     ap.add_argument("--fused", default="c2,T8192,T16384,c3,c4a,c4b,c4c,c5")
+    ap.add_argument("--single", default="c2,c3,c4a,c4b,c4c,c5")
     ap.add_argument("--dense", default="c2,T8192,T16384,c3")
     ap.add_argument("--fwdchunk", default="c2,T8192,T16384,c3,c4a,c4b")
     ap.add_argument("--out", default="")
@@ -179,7 +185,8 @@ def main():
         return
 
     rows = []
-    for method, names in (("fused", args.fused), ("dense", args.dense), ("fwdchunk", args.fwdchunk)):
+    for method, names in (("fused", args.fused), ("single", args.single), ("dense", args.dense),
+                          ("fwdchunk", args.fwdchunk)):
         for name in [n for n in names.split(",") if n]:
             t0 = time.time()
             r = subprocess.run([sys.executable, "-m", "paper_2608_03796_b200.sweep", "--worker", method,
@@ -204,7 +211,9 @@ def main():
         lines = ["# Sequence-length sweep: iteration rate and peak memory (one B200, fresh process per setting)", "",
                  "Command: `python -m paper_2608_03796_b200.sweep --out " + args.out + "`", "",
                  f"Peaks used: bf16 burst {burst} / sustained {sust} TFLOP/s "
-                 f"({'measured' if peaks else 'fallback'}). FLOPs counted as 8*T*H*V per iteration.", "",
+                 f"({'measured' if peaks else 'fallback'}). TFLOP/s counts the projections a method executes: "
+                 "8*T*H*V per iteration for `fused` (the paper's schedule, with recompute), 6*T*H*V for `single` and for "
+                 "the two torch comparators; compare methods by ms/iter and tokens/s.", "",
                  "| method | workload | T | ms/iter | it/s | tokens/s | TFLOP/s | % burst | % sustained | peak GB | driver Δ GB | workspace GB | loss | ‖dH‖ | ‖dW‖ |",
                  "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|"]
         for r in rows:
