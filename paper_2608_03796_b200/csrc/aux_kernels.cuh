@@ -213,7 +213,8 @@ __global__ void step_coef_kernel(const float* __restrict__ Mv, const uint8_t* __
 // chunk's G: the op is bound by HBM), then the row's support entries inside the segment are patched.
 constexpr int E2G_SEG = 8192;                  // columns per block: 256 threads x 4 vectors of 8
 __global__ void __launch_bounds__(256)
-e_to_g_kernel(__nv_bfloat16* __restrict__ G, long long ldg /* elements per row */, int n_cols /* multiple of 8 */,
+e_to_g_kernel(__nv_bfloat16* __restrict__ G, long long ldg /* elements per row */, int n_cols /* V rounded up to 8 */,
+              int V /* columns the forward sweep wrote; the rest of the last vector is stale memory */,
               const float* __restrict__ coefA, const float* __restrict__ coefB, const float* __restrict__ lz2,
               const int* __restrict__ idx_sorted, const float* __restrict__ p_sorted, const int* __restrict__ nvalid,
               int Ktop, float bias, int n_seg, WsHeader* hdr) {
@@ -243,7 +244,8 @@ e_to_g_kernel(__nv_bfloat16* __restrict__ G, long long ldg /* elements per row *
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const float2 x = __bfloat1622float2(h2[j]);
-        const float y0 = x.x * scale, y1 = x.y * scale;
+        const int col = v * 8 + 2 * j;
+        const float y0 = col < V ? x.x * scale : 0.f, y1 = col + 1 < V ? x.y * scale : 0.f;
         bad |= !(fabsf(y0) <= 3.0e38f) || !(fabsf(y1) <= 3.0e38f);
         h2[j] = __floats2bfloat162_rn(y0, y1);
       }
