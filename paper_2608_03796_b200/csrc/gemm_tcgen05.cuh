@@ -443,6 +443,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         tmem_ld32(taddr + w * 32, r);
         tmem_ld_wait();
         const bool full_w = col0 + 32 <= p.N;
+        float e_fac = 0.f;                     // EPI_LSE_E: 2^(running maximum - bias) of this row and window
 
         if (kLse) {
           if (row_ok) {
@@ -464,8 +465,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
             const float m_new = fmaxf(m_run, wmax * p.scale_log2);
             float acc_s = 0.f;
+            if (EPI == EPI_LSE_E) {
+              // keep the window's exponentials (relative to the running maximum) in place of the logits:
+              // e = 2^(s - bias) = 2^(s - m_new) * 2^(m_new - bias), one multiply instead of a second ex2
 #pragma unroll
-            for (int j = 0; j < 32; ++j) acc_s += ex2_approx(fmaf(__uint_as_float(r[j]), p.scale_log2, -m_new));
+              for (int j = 0; j < 32; ++j) {
+                const float tj = ex2_approx(fmaf(__uint_as_float(r[j]), p.scale_log2, -m_new));
+                acc_s += tj;
+                r[j] = __float_as_uint(tj);
+              }
+              e_fac = ex2_approx(m_new - kExpBias);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) acc_s += ex2_approx(fmaf(__uint_as_float(r[j]), p.scale_log2, -m_new));
+            }
             s_run = s_run * ex2_approx(m_run - m_new) + acc_s;
             m_run = m_new;
           }
@@ -514,8 +527,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               // unnormalised exponentials with a fixed bias: G = A_t * e - b_t p is formed from them later
 #pragma unroll
               for (int j = 0; j < 16; ++j)
-                v[j] = pack_bf16x2(ex2_approx(fmaf(__uint_as_float(r[2 * j]), p.scale_log2, -kExpBias)),
-                                   ex2_approx(fmaf(__uint_as_float(r[2 * j + 1]), p.scale_log2, -kExpBias)));
+                v[j] = pack_bf16x2(__uint_as_float(r[2 * j]) * e_fac, __uint_as_float(r[2 * j + 1]) * e_fac);
             } else {  // EPI_DLOGITS
               // a_t * 2^(s - lz2) = 2^(s + (log2 a_t - lz2)): the row coefficient rides in the exponent
               // (a_t = 0 for ignored tokens gives -inf, hence exact zeros)
