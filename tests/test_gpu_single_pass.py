@@ -132,3 +132,41 @@ def test_overflowing_exponential_is_reported_not_hidden():
     assert two.status()[0] == 0 and torch.isfinite(two.dweight).all() and torch.isfinite(two.dhidden.float()).all()
     o = kdkl_oracle(h.double().numpy(), W.double().numpy(), idx.numpy(), val.numpy())
     assert abs(two.loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
+
+
+def test_single_pass_packed_config_sampled_rows_and_dweight():
+    """c5 (16 chunks, packing mask with a dead padding tail, tau = 2, ragged vocabulary): sampled dH rows with the
+    full run's denominator, and dW through a second run whose mask is the indicator of the sample."""
+    dev = torch.device("cuda:0")
+    cfg = I.CONFIGS["c5"]
+    d = I.make_inputs(cfg, device=dev)
+    mask = d["mask"]
+    n_counted = int(mask.sum().item())
+    op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev,
+                          want_per_token=True)
+    op.forward_backward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], loss_mask=mask)
+    assert op.status()[0] == 0
+    R = I.sample_rows(cfg, 48)
+    Rd = R.to(dev)
+    hR = d["hidden"][Rd].cpu().double().numpy()
+    W64 = d["weight"].cpu().double().numpy()
+    idxR, valR = d["topk_idx"][Rd].cpu().numpy(), d["topk_val"][Rd].cpu().numpy()
+    mR = mask[Rd].cpu().numpy()
+    with np.errstate(all="ignore"):
+        o = kdkl_oracle(hR, W64, idxR, valR, tau=cfg.tau, mask=mR, denom=n_counted)
+    np.testing.assert_allclose(op.loss_per_token[Rd].cpu().double().numpy(), o["loss_tok"], rtol=0, atol=2e-4)
+    assert _fro(op.dhidden[Rd].float().cpu().double().numpy(), o["dH"]) <= 1e-2
+    assert not op.dhidden[mask == 0].float().abs().sum().item()
+    colsum = op.dweight.double().sum(0).abs()
+    assert (colsum / op.dweight.double().abs().sum(0)).max().item() < 3e-3
+    # dW: mask = indicator of the counted sampled rows
+    mR_full = torch.zeros(cfg.T, dtype=torch.uint8, device=dev)
+    mR_full[Rd] = 1
+    mR_full &= mask
+    nR = int(mR_full.sum().item())
+    op.forward_backward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], loss_mask=mR_full)
+    assert op.status()[0] == 0
+    with np.errstate(all="ignore"):
+        oR = kdkl_oracle(hR, W64, idxR, valR, tau=cfg.tau, mask=mR, denom=nR)
+    assert abs(op.loss.item() - oR["loss"]) <= 1e-3 * abs(oR["loss"])
+    assert _fro(op.dweight.cpu().double().numpy(), oR["dW"]) <= 1e-2
