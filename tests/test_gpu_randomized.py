@@ -68,8 +68,9 @@ def _fro(a, b):
     return np.linalg.norm(a - b) / nb if nb > 0 else np.linalg.norm(a)
 
 
+@pytest.mark.parametrize("single_pass", [False, True])
 @pytest.mark.parametrize("seed", list(range(1000, 1100)))
-def test_random_configuration_matches_oracle(seed):
+def test_random_configuration_matches_oracle(seed, single_pass):
     c = _draw(seed)
     dev = torch.device("cuda:0")
     T, H, V, K = c["T"], c["H"], c["V"], c["K"]
@@ -82,8 +83,13 @@ def test_random_configuration_matches_oracle(seed):
     op.dhidden.fill_(float("nan"))
     op.dweight.copy_(base) if c["accumulate"] else op.dweight.fill_(float("nan"))
     to = lambda x: None if x is None else x.to(dev)
-    op.forward(to(c["h"]), to(c["W"]), to(c["idx"]), to(c["val"]), teacher_lse=to(c["lse"]), loss_mask=to(c["mask"]))
-    op.backward(to(c["h"]), to(c["W"]), loss_mask=to(c["mask"]), grad_loss=c["grad_loss"])
+    if single_pass:
+        op.forward_backward(to(c["h"]), to(c["W"]), to(c["idx"]), to(c["val"]), teacher_lse=to(c["lse"]),
+                            loss_mask=to(c["mask"]), grad_loss=c["grad_loss"])
+    else:
+        op.forward(to(c["h"]), to(c["W"]), to(c["idx"]), to(c["val"]), teacher_lse=to(c["lse"]),
+                   loss_mask=to(c["mask"]))
+        op.backward(to(c["h"]), to(c["W"]), loss_mask=to(c["mask"]), grad_loss=c["grad_loss"])
     code, detail = op.status()
     assert code == (-10 if c["n_bad"] else 0), (code, detail)
     if c["n_bad"]:
@@ -100,11 +106,12 @@ def test_random_configuration_matches_oracle(seed):
     np.testing.assert_allclose(lz.cpu().double().numpy()[counted], o["logZ"][counted], rtol=0, atol=TOK_ATOL)
     np.testing.assert_allclose(M.cpu().double().numpy()[counted], o["M"][counted], rtol=0, atol=1e-5)
     idx = c["idx"].numpy()
-    usable = (idx >= 0) & (idx < V) & counted[:, None]
-    gi = op.gathered_idx.cpu().numpy()
-    assert np.array_equal(gi[usable], idx[usable]) and np.all(gi[~usable] == -1)
-    gl = op.gathered_logits.cpu().double().numpy()
-    np.testing.assert_allclose(gl[usable], o["gathered_logits"][usable], rtol=0, atol=ZG_ATOL)
+    if not single_pass:                               # the single-pass call does not return the gathered logits
+        usable = (idx >= 0) & (idx < V) & counted[:, None]
+        gi = op.gathered_idx.cpu().numpy()
+        assert np.array_equal(gi[usable], idx[usable]) and np.all(gi[~usable] == -1)
+        gl = op.gathered_logits.cpu().double().numpy()
+        np.testing.assert_allclose(gl[usable], o["gathered_logits"][usable], rtol=0, atol=ZG_ATOL)
     dH = op.dhidden.float().cpu().double().numpy()
     dW = op.dweight.cpu().double().numpy()
     want_dW = o["dW"] + (base.double().numpy() if c["accumulate"] else 0.0)
