@@ -40,15 +40,17 @@ def _holder(T, H, V, K, chunk, tau, accumulate, device) -> B.FusedChunkedKL:
 class _FusedChunkedKL(torch.autograd.Function):
     @staticmethod
     def forward(ctx, hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, chunk, temperature, dweight_out,
-                weight_grad_fp32, single_pass):
+                weight_grad_fp32, single_pass, expected_grad):
         T, H = hidden.shape
         V, K = weight.shape[0], topk_idx.shape[1]
         # single pass: the gradients for an upstream gradient of 1 come out of the forward call (three projections
         # instead of four); it writes dW itself, so it is not combined with accumulation into a caller's buffer
         ctx.done = bool(single_pass) and dweight_out is None
         op = _holder(T, H, V, K, int(chunk), float(temperature), 1 if dweight_out is not None else 0, hidden.device)
+        ctx.expected = float(expected_grad)
         if ctx.done:
-            op.forward_backward(hidden, weight, topk_idx, topk_val, teacher_lse=teacher_lse, loss_mask=loss_mask)
+            op.forward_backward(hidden, weight, topk_idx, topk_val, teacher_lse=teacher_lse, loss_mask=loss_mask,
+                                grad_loss=ctx.expected)
         else:
             op.forward(hidden, weight, topk_idx, topk_val, teacher_lse=teacher_lse, loss_mask=loss_mask)
         ctx.op, ctx.mask = op, loss_mask
@@ -61,7 +63,7 @@ class _FusedChunkedKL(torch.autograd.Function):
         hidden, weight = ctx.saved_tensors
         op = ctx.op
         gl = float(grad.item())
-        if not (ctx.done and gl == 1.0):                          # any other upstream gradient: the recompute path
+        if not (ctx.done and gl == ctx.expected):                 # any other upstream gradient: the recompute path
             if ctx.dweight_out is not None:
                 saved, op.dweight = op.dweight, ctx.dweight_out   # dW += into the caller's fp32 buffer
             try:
@@ -78,17 +80,19 @@ class _FusedChunkedKL(torch.autograd.Function):
             dW = op.dweight
         else:
             dW = op.dweight.to(weight.dtype)
-        return op.dhidden.clone(), dW, None, None, None, None, None, None, None, None, None
+        return op.dhidden.clone(), dW, None, None, None, None, None, None, None, None, None, None
 
 
 def fused_chunked_kl(hidden, weight, topk_idx, topk_val, teacher_lse: Optional[torch.Tensor] = None,
                      loss_mask: Optional[torch.Tensor] = None, chunk: int = 4096, temperature: float = 1.0,
                      dweight_out: Optional[torch.Tensor] = None, weight_grad_fp32: bool = False,
-                     single_pass: bool = False) -> torch.Tensor:
+                     single_pass: bool = False, expected_grad: float = 1.0) -> torch.Tensor:
     """Mean forward KL between the cached top-K teacher and softmax(hidden @ weight.T / temperature).
-    single_pass=True computes the gradients during the forward call (kdkl_forward_backward)."""
+    single_pass=True computes the gradients during the forward call (kdkl_forward_backward) for an upstream
+    gradient of `expected_grad` (the weight this loss carries in the total); if backward then sees another
+    value, the gradients are recomputed by kdkl_backward."""
     return _FusedChunkedKL.apply(hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, chunk, temperature,
-                                 dweight_out, weight_grad_fp32, single_pass)
+                                 dweight_out, weight_grad_fp32, single_pass, expected_grad)
 
 
 class _FeatureLoss(torch.autograd.Function):

@@ -66,11 +66,11 @@ def test_single_pass_autograd_matches_oracle():
     d = I.make_inputs(cfg, device=dev)
     o = kdkl_oracle(d["hidden"].cpu().double().numpy(), d["weight"].cpu().double().numpy(),
                     d["topk_idx"].cpu().numpy(), d["topk_val"].cpu().numpy(), tau=cfg.tau)
-    for scale in (1.0, 3.0):                               # 3.0 takes the recompute path in backward
+    for scale, expected in ((1.0, 1.0), (3.0, 1.0), (0.25, 0.25)):   # (3.0, 1.0) takes the recompute path in backward
         h = d["hidden"].clone().requires_grad_(True)
         W = d["weight"].clone().requires_grad_(True)
         loss = fused_chunked_kl(h, W, d["topk_idx"], d["topk_val"], chunk=cfg.chunk, temperature=cfg.tau,
-                                single_pass=True)
+                                single_pass=True, expected_grad=expected)
         (scale * loss).backward()
         assert abs(loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
         assert _fro(h.grad.float().cpu().double().numpy(), scale * o["dH"]) <= 1e-2
