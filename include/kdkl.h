@@ -57,6 +57,12 @@ typedef struct kdkl_options {
   int32_t accumulate_dweight; /* 0: dweight is overwritten; 1: dweight += */
   int32_t dhidden_dtype;      /* 0: bf16; 1: fp32 */
   float denom_override;       /* <= 0: mean over this call's counted tokens; > 0: divide by this instead */
+  int32_t stored_exponentials;/* 1: only when one chunk covers all T tokens (chunk >= T): the forward call also
+                                 leaves the bf16 exponentials 2^(z log2e / tau - 64) in the workspace's [T, V]
+                                 buffer and kdkl_backward forms G from them instead of projecting again (three
+                                 projections for the two calls, as in kdkl_forward_backward; the vocabulary-sharded
+                                 calls included, where log Z is only known after the exchange). Otherwise
+                                 KDKL_ERR_ARG. A struct of the previous size (without this field) is accepted */
 } kdkl_options;
 
 /* Bytes of device workspace forward and backward need for this shape (chunk 0 = default 4096).

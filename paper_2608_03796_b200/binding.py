@@ -43,7 +43,7 @@ class KdklError(RuntimeError):
 class kdkl_options(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_int32), ("teacher_mode", ctypes.c_int32),
                 ("accumulate_dweight", ctypes.c_int32), ("dhidden_dtype", ctypes.c_int32),
-                ("denom_override", ctypes.c_float)]
+                ("denom_override", ctypes.c_float), ("stored_exponentials", ctypes.c_int32)]
 
 
 _lib = None
@@ -149,8 +149,10 @@ def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def make_options(teacher_mode=0, accumulate_dweight=0, dhidden_dtype=0, denom_override=0.0) -> kdkl_options:
-    return kdkl_options(ctypes.sizeof(kdkl_options), teacher_mode, accumulate_dweight, dhidden_dtype, denom_override)
+def make_options(teacher_mode=0, accumulate_dweight=0, dhidden_dtype=0, denom_override=0.0,
+                 stored_exponentials=0) -> kdkl_options:
+    return kdkl_options(ctypes.sizeof(kdkl_options), teacher_mode, accumulate_dweight, dhidden_dtype, denom_override,
+                        stored_exponentials)
 
 
 def _opt_ptr(opt: Optional[kdkl_options]):
@@ -422,11 +424,14 @@ class ShardedFusedChunkedKL:
     """
 
     def __init__(self, T, H, V_local, vocab_offset, V_total, K, n_shards, chunk=0, temperature=1.0, device="cuda",
-                 all_gather=None, all_reduce_sum=None, want_per_token=False):
+                 all_gather=None, all_reduce_sum=None, want_per_token=False, opt=None):
         self.T, self.H, self.V_local, self.K = T, H, V_local, K
         self.vocab_offset, self.V_total, self.n_shards = vocab_offset, V_total, n_shards
         self.chunk, self.temperature = chunk, temperature
-        self.opt = make_options(dhidden_dtype=1)            # fp32 partial dhidden: summed over ranks in fp32
+        # fp32 partial dhidden: summed over ranks in fp32 (an option struct passed in must ask for it too)
+        self.opt = opt if opt is not None else make_options(dhidden_dtype=1)
+        if self.opt.dhidden_dtype != 1:
+            raise ValueError("ShardedFusedChunkedKL: opt.dhidden_dtype must be 1 (fp32 partial sums)")
         self.workspace = torch.empty(kdkl_workspace_bytes(T, H, V_local, K, chunk, self.opt), dtype=torch.uint8,
                                      device=device)
         self.stats_local = torch.empty(2, T, dtype=torch.float32, device=device)

@@ -217,7 +217,8 @@ e_to_g_kernel(__nv_bfloat16* __restrict__ G, long long ldg /* elements per row *
               int V /* columns the forward sweep wrote; the rest of the last vector is stale memory */,
               const float* __restrict__ coefA, const float* __restrict__ coefB, const float* __restrict__ lz2,
               const int* __restrict__ idx_sorted, const float* __restrict__ p_sorted, const int* __restrict__ nvalid,
-              int Ktop, float bias, int n_seg, WsHeader* hdr) {
+              int Ktop, float bias, int n_seg, WsHeader* hdr, const int* go) {
+  if (go != nullptr && *go == 0) return;       // backward gate: the workspace does not hold this call's state
   const long long row = blockIdx.x / n_seg;
   const int c_begin = (int)(blockIdx.x - row * n_seg) * E2G_SEG;
   const int c_end = c_begin + E2G_SEG < n_cols ? c_begin + E2G_SEG : n_cols;

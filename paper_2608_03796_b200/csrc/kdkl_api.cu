@@ -220,6 +220,18 @@ static WsLayout ws_layout(long long T, long long H, long long V, int K, long lon
   return L;
 }
 
+// Options of this or of the previous struct size (without stored_exponentials) are accepted.
+static int copy_options(const kdkl_options* opt, kdkl_options* eff) {
+  memset(eff, 0, sizeof(*eff));
+  if (!opt) return KDKL_OK;
+  constexpr int32_t kOldSize = (int32_t)offsetof(kdkl_options, stored_exponentials);
+  if (opt->struct_size != (int32_t)sizeof(kdkl_options) && opt->struct_size != kOldSize) return KDKL_ERR_ARG;
+  memcpy(eff, opt, (size_t)opt->struct_size);
+  eff->struct_size = (int32_t)sizeof(kdkl_options);
+  if (eff->stored_exponentials < 0 || eff->stored_exponentials > 1) return KDKL_ERR_ARG;
+  return KDKL_OK;
+}
+
 static int check_common(const void* hidden, const void* weight, long long T, long long H, long long V, int K,
                         long long chunk, float tau, const kdkl_options* opt, const void* ws, size_t ws_bytes,
                         kdkl_options* eff, WsLayout* L) {
@@ -227,16 +239,13 @@ static int check_common(const void* hidden, const void* weight, long long T, lon
   if (T < 1 || H < 1 || V < 1 || K < 1 || K > KDKL_MAX_K || (H % 8) != 0 || V >= (1ll << 31) || T >= (1ll << 31))
     return KDKL_ERR_SHAPE;
   if (!(tau > 0.f) || chunk < 0) return KDKL_ERR_ARG;
-  memset(eff, 0, sizeof(*eff));
-  if (opt) {
-    if (opt->struct_size != (int32_t)sizeof(kdkl_options)) return KDKL_ERR_ARG;
-    *eff = *opt;
-  }
+  if (copy_options(opt, eff) != KDKL_OK) return KDKL_ERR_ARG;
   if (eff->teacher_mode < 0 || eff->teacher_mode > 1) return KDKL_ERR_ARG;
   if (eff->teacher_mode == 1 && tau != 1.0f) return KDKL_ERR_ARG;
   if (eff->dhidden_dtype < 0 || eff->dhidden_dtype > 1) return KDKL_ERR_ARG;
   if (((uintptr_t)hidden & 15) || ((uintptr_t)weight & 15) || ((uintptr_t)ws & 15)) return KDKL_ERR_ALIGN;
   *L = ws_layout(T, H, V, K, chunk);
+  if (eff->stored_exponentials && T > L->C) return KDKL_ERR_ARG;   // needs one chunk over all tokens
   if (ws_bytes < L->total) return KDKL_ERR_WORKSPACE;
   DeviceInfo di;
   int rc = device_info(&di);
@@ -327,7 +336,15 @@ static int forward_impl(const void* hidden, const void* weight, const int32_t* t
     p.colread = at<int>(ws, L.colread) + s0 * K;
     p.m_live = (live && p.m_tiles <= MAX_LIVE_M) ? live + fci * L.tiles_per_chunk : nullptr;
     stage_mark(ST_F1, st);
-    if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA /*no output map*/, p, di.sm_count, st))) return rc;
+    if (o.stored_exponentials) {
+      // one chunk covers all tokens: leave the exponentials in the G buffer for a backward without recompute
+      CUtensorMap tmE;
+      if ((rc = make_tmap_out_bf16(&tmE, at<__nv_bfloat16>(ws, L.G), (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad)))
+        return rc;
+      if ((rc = launch_gemm<EPI_LSE_E, false, false>(tmA, tmW, tmE, p, di.sm_count, st))) return rc;
+    } else {
+      if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA /*no output map*/, p, di.sm_count, st))) return rc;
+    }
     stage_mark(ST_COMBINE, st);
 
     combine_kernel<<<(unsigned)((rows + 31) / 32), COMBINE_WARPS * 32, 0, st>>>(
@@ -375,7 +392,7 @@ int kdkl_forward_finish(const float* all_stats, int32_t n_shards, const uint8_t*
   if (n_shards < 1 || T < 1 || H < 1 || V_local < 1 || K < 1) return KDKL_ERR_SHAPE;
   kdkl_options o;
   memset(&o, 0, sizeof(o));
-  if (opt) { if (opt->struct_size != (int32_t)sizeof(kdkl_options)) return KDKL_ERR_ARG; o = *opt; }
+  if (copy_options(opt, &o) != KDKL_OK) return KDKL_ERR_ARG;
   WsLayout L = ws_layout(T, H, V_local, K, chunk);
   if (ws_bytes < L.total) return KDKL_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
@@ -453,7 +470,18 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     CUtensorMap tmGout;
     if ((rc = make_tmap_out_bf16(&tmGout, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad))) return rc;
     stage_mark(ST_B1, st);
-    if ((rc = launch_gemm<EPI_DLOGITS, false, false>(tmA, tmW, tmGout, p, di.sm_count, st))) return rc;
+    if (o.stored_exponentials) {
+      // the forward call left the exponentials of this (only) chunk in G: no second projection
+      const int n_cols = (int)(((V + 7) / 8) * 8);
+      const int n_seg = (n_cols + E2G_SEG - 1) / E2G_SEG;
+      e_to_g_kernel<<<(unsigned)(rows * n_seg), 256, 0, st>>>(
+          G, L.Vpad, n_cols, (int)V, at<float>(ws, L.coefA) + s0, at<float>(ws, L.coefB) + s0,
+          at<float>(ws, L.lz2) + s0, at<int>(ws, L.idx_sorted) + s0 * K, at<float>(ws, L.p_sorted) + s0 * K,
+          at<int>(ws, L.nvalid) + s0, K, kExpBias, n_seg, hdr, go);
+      KDKL_LAUNCHED("e_to_g_kernel");
+    } else {
+      if ((rc = launch_gemm<EPI_DLOGITS, false, false>(tmA, tmW, tmGout, p, di.sm_count, st))) return rc;
+    }
     stage_mark(ST_B2, st);
 
     // B2: dH[chunk] = G W   (M = rows, N = H, K = V)
@@ -600,7 +628,7 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
     e_to_g_kernel<<<(unsigned)(rows * n_seg), 256, 0, st>>>(
         G, L.Vpad, n_cols, (int)V, at<float>(ws, L.coefA) + s0, at<float>(ws, L.coefB) + s0, at<float>(ws, L.lz2) + s0,
         at<int>(ws, L.idx_sorted) + s0 * K, at<float>(ws, L.p_sorted) + s0 * K, at<int>(ws, L.nvalid) + s0, K, kExpBias,
-        n_seg, hdr);
+        n_seg, hdr, nullptr);
     KDKL_LAUNCHED("e_to_g_kernel");
 
     // dH[chunk] = G W and dW (+)= G^T h, exactly as in kdkl_backward

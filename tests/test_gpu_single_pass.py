@@ -170,3 +170,29 @@ def test_single_pass_packed_config_sampled_rows_and_dweight():
         oR = kdkl_oracle(hR, W64, idxR, valR, tau=cfg.tau, mask=mR, denom=nR)
     assert abs(op.loss.item() - oR["loss"]) <= 1e-3 * abs(oR["loss"])
     assert _fro(op.dweight.cpu().double().numpy(), oR["dW"]) <= 1e-2
+
+
+def test_two_calls_with_stored_exponentials_one_chunk():
+    """Option stored_exponentials: forward leaves the exponentials, backward forms G from them (no second
+    projection), valid when one chunk covers all tokens. Same checks as the single-pass call."""
+    dev = torch.device("cuda:0")
+    T, H, V, K, tau = 700, 136, 3001, 12, 1.3
+    h, W, idx, val, mask = _case(T, H, V, K, seed=77, mask_mode=2)
+    opt = B.make_options(stored_exponentials=1)
+    op = B.FusedChunkedKL(T, H, V, K, chunk=0, temperature=tau, opt=opt, device=dev, want_per_token=True)
+    op.workspace.view(torch.int16).fill_(0x7fc0)
+    to = lambda x: None if x is None else x.to(dev)
+    op.forward(to(h), to(W), to(idx), to(val), loss_mask=to(mask))
+    op.backward(to(h), to(W), loss_mask=to(mask), grad_loss=0.5)
+    assert op.status()[0] == 0
+    with np.errstate(all="ignore"):
+        o = kdkl_oracle(h.double().numpy(), W.double().numpy(), idx.numpy(), val.numpy(), tau=tau, mask=mask.numpy(),
+                        grad_loss=0.5)
+    assert abs(op.loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
+    assert _fro(op.dhidden.float().cpu().double().numpy(), o["dH"]) <= 1e-2
+    assert _fro(op.dweight.cpu().double().numpy(), o["dW"]) <= 1e-2
+    # more than one chunk is refused on the host
+    with pytest.raises(B.KdklError) as e:
+        B.FusedChunkedKL(T, H, V, K, chunk=256, temperature=tau, opt=opt, device=dev).forward(
+            to(h), to(W), to(idx), to(val), loss_mask=to(mask))
+    assert e.value.code == -5

@@ -19,7 +19,7 @@ def _fro(a, b):
     return np.linalg.norm(a - b) / np.linalg.norm(b)
 
 
-def _run_sharded(d, T, H, V, K, bounds, chunk, tau, lse=None, grad_loss=1.0):
+def _run_sharded(d, T, H, V, K, bounds, chunk, tau, lse=None, grad_loss=1.0, opt=None):
     dev = torch.device("cuda:0")
     g = {k: (v.to(dev) if v is not None else None) for k, v in d.items()}
     lse_d = None if lse is None else lse.to(dev)
@@ -28,7 +28,7 @@ def _run_sharded(d, T, H, V, K, bounds, chunk, tau, lse=None, grad_loss=1.0):
     for r in range(R):
         v0, v1 = bounds[r], bounds[r + 1]
         ranks.append(B.ShardedFusedChunkedKL(T, H, v1 - v0, v0, V, K, R, chunk=chunk, temperature=tau, device=dev,
-                                             want_per_token=True))
+                                             want_per_token=True, opt=opt))
     W = [g["weight"][bounds[r]:bounds[r + 1]].contiguous() for r in range(R)]
     for r, op in enumerate(ranks):
         op.forward_local(g["hidden"], W[r], g["topk_idx"], g["topk_val"], teacher_lse=lse_d, loss_mask=g["mask"])
@@ -161,3 +161,23 @@ def test_random_shardings_match_oracle(seed):
     assert _fro(dW.cpu().double().numpy(), o["dW"]) <= 1e-2
     if mask is not None:
         assert not dH[mask == 0].abs().sum().item()
+
+
+def test_sharded_without_recompute_when_one_chunk_covers_the_tokens():
+    """stored_exponentials with vocabulary shards: log Z is known only after the exchange, the exponentials wait in
+    each rank's buffer, and the backward of every rank forms its G slice from them (three projections)."""
+    T, H, V, K, tau = 300, 264, 4120, 9, 1.0
+    g = torch.Generator().manual_seed(5)
+    d = {"hidden": torch.randn(T, H, generator=g).to(torch.bfloat16),
+         "weight": (torch.randn(V, H, generator=g) / H ** 0.5).to(torch.bfloat16),
+         "topk_idx": torch.stack([torch.randperm(V, generator=g)[:K] for _ in range(T)]).to(torch.int32),
+         "topk_val": (torch.randn(T, K, generator=g) * 3 ** 0.5).float(),
+         "mask": (torch.rand(T, generator=g) >= 0.1).to(torch.uint8)}
+    ranks, dH, dW = _run_sharded(d, T, H, V, K, [0, 1000, 2500, 4120], 0, tau,
+                                 opt=B.make_options(stored_exponentials=1, dhidden_dtype=1))
+    o = kdkl_oracle(d["hidden"].double().numpy(), d["weight"].double().numpy(), d["topk_idx"].numpy(),
+                    d["topk_val"].numpy(), tau=tau, mask=d["mask"].numpy())
+    for op in ranks:
+        assert abs(op.loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
+    assert _fro(dH.cpu().double().numpy(), o["dH"]) <= 1e-2
+    assert _fro(dW.cpu().double().numpy(), o["dW"]) <= 1e-2

@@ -40,7 +40,7 @@ def test_sizes_without_a_gpu():
 
 def test_options_struct_layout():
     o = binding.make_options(teacher_mode=1, denom_override=3.0)
-    assert o.struct_size == 20 and o.teacher_mode == 1 and o.denom_override == 3.0
+    assert o.struct_size == 24 and o.teacher_mode == 1 and o.denom_override == 3.0 and o.stored_exponentials == 0
 
 
 def test_host_side_argument_checks_without_a_gpu():
@@ -64,6 +64,12 @@ def test_host_side_argument_checks_without_a_gpu():
     bad_opt.struct_size = 7
     assert fwd(opt=binding._opt_ptr(bad_opt)) == -5
     assert fwd(opt=binding._opt_ptr(binding.make_options(teacher_mode=1)), tau=2.0) == -5
+    old_size = binding.make_options()
+    old_size.struct_size = 20                     # the struct before stored_exponentials was added is still accepted
+    assert fwd(opt=binding._opt_ptr(old_size), wsb=ws - 1) == -4
+    # stored exponentials need one chunk over all tokens
+    assert fwd(opt=binding._opt_ptr(binding.make_options(stored_exponentials=1)), chunk=32) == -5
+    assert fwd(opt=binding._opt_ptr(binding.make_options(stored_exponentials=2))) == -5
     # backward: same checks plus its own outputs
     def bwd(dh=P, dw=P, **kw):
         a = dict(hidden=P, weight=P, T=T, H=H, V=V, K=K, chunk=0, tau=1.0, wsp=Q, wsb=ws)
