@@ -526,5 +526,20 @@ class TokenShardedFusedKL:
         self._all_reduce_sum(self.dweight)                     # the data-parallel gradient reduction
         return self.dhidden, self.dweight
 
+    def forward_backward_local(self, hidden, weight, topk_idx, topk_val, n_global, teacher_lse=None, loss_mask=None,
+                               grad_loss=1.0):
+        """Single-pass step of this rank (three projections) with the global divisor."""
+        self.opt = make_options(denom_override=n_global)
+        kdkl_forward_backward(hidden, weight, topk_idx, topk_val, self.workspace, self.loss, self.dhidden,
+                              self.dweight, teacher_lse=teacher_lse, loss_mask=loss_mask, chunk=self.chunk,
+                              temperature=self.temperature, opt=self.opt, grad_loss=grad_loss)
+
+    def forward_backward(self, hidden, weight, topk_idx, topk_val, teacher_lse=None, loss_mask=None, grad_loss=1.0):
+        self.forward_backward_local(hidden, weight, topk_idx, topk_val, self.count_tokens(loss_mask), teacher_lse,
+                                    loss_mask, grad_loss)
+        self._all_reduce_sum(self.loss)
+        self._all_reduce_sum(self.dweight)
+        return self.loss, self.dhidden, self.dweight
+
     def status(self):
         return kdkl_status(self.workspace)

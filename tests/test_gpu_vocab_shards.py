@@ -86,7 +86,8 @@ def test_sharded_c1_two_halves_equals_unsharded_loss():
     assert _fro(dH.cpu().double().numpy(), full.dhidden.cpu().double().numpy()) < 2e-3
 
 
-def test_token_shards_match_oracle():
+@pytest.mark.parametrize("single_pass", [False, True])
+def test_token_shards_match_oracle(single_pass):
     """Data-parallel form: uneven token slices, the global denominator on every rank, dW and loss summed."""
     T, H, V, K, tau = 300, 136, 2100, 7, 1.0
     g = torch.Generator().manual_seed(51)
@@ -104,8 +105,12 @@ def test_token_shards_match_oracle():
         a, b = bounds[r], bounds[r + 1]
         op = B.TokenShardedFusedKL(b - a, H, V, K, chunk=64, temperature=tau, device=dev, all_reduce_sum=lambda t: t)
         sl = {k: (v[a:b].contiguous() if k != "weight" else v) for k, v in gd.items()}
-        op.forward_local(sl["hidden"], sl["weight"], sl["topk_idx"], sl["topk_val"], n_global, loss_mask=sl["mask"])
-        op.backward_local(sl["hidden"], sl["weight"], loss_mask=sl["mask"])
+        if single_pass:
+            op.forward_backward_local(sl["hidden"], sl["weight"], sl["topk_idx"], sl["topk_val"], n_global,
+                                      loss_mask=sl["mask"])
+        else:
+            op.forward_local(sl["hidden"], sl["weight"], sl["topk_idx"], sl["topk_val"], n_global, loss_mask=sl["mask"])
+            op.backward_local(sl["hidden"], sl["weight"], loss_mask=sl["mask"])
         assert op.status()[0] == 0
         ranks.append(op)
     loss = sum(op.loss.item() for op in ranks)                       # what the all-reduces deliver
