@@ -295,3 +295,30 @@ def test_device_side_status_codes():
     op3 = _run(d2, T, H, V, K, 0, 1.0)
     assert op3.status()[0] == 0
     assert torch.equal(op2.loss_per_token, op3.loss_per_token) and torch.equal(op2.dweight, op3.dweight)
+
+
+def test_invariances_offset_and_slot_permutation():
+    """Two invariances the definition has, checked on the GPU path itself: (i) with no teacher_lse the teacher
+    is a softmax over the K values, so a per-token constant added to them changes nothing; (ii) the order of
+    the K slots of a row is irrelevant (the kernel sorts them): losses agree to fp32 rounding, and the
+    gathered logits follow their slots."""
+    T, H, V, K, tau = 150, 72, 1001, 13, 1.3
+    d = _small_case(T, H, V, K, seed=31)
+    base = _run(d, T, H, V, K, 64, tau)
+    g = torch.Generator().manual_seed(2)
+    shifted = dict(d)
+    shifted["topk_val"] = d["topk_val"] + torch.randn(T, 1, generator=g) * 5.0
+    a = _run(shifted, T, H, V, K, 64, tau)
+    assert (a.loss_per_token - base.loss_per_token).abs().max().item() < 5e-5
+    assert ((a.dweight - base.dweight).norm() / base.dweight.norm()).item() < 2e-3
+    perm = torch.stack([torch.randperm(K, generator=g) for _ in range(T)])
+    shuffled = dict(d)
+    shuffled["topk_idx"] = torch.gather(d["topk_idx"], 1, perm).contiguous()
+    shuffled["topk_val"] = torch.gather(d["topk_val"], 1, perm).contiguous()
+    b = _run(shuffled, T, H, V, K, 64, tau)
+    assert (b.loss_per_token - base.loss_per_token).abs().max().item() < 5e-6
+    assert torch.equal(b.gathered_idx.cpu(), shuffled["topk_idx"])
+    assert torch.equal(b.gathered_logits.cpu(), torch.gather(base.gathered_logits.cpu(), 1, perm))
+    # the teacher's normaliser is summed in slot order, so p moves in its last bits and single bf16 roundings of G flip
+    assert ((b.dweight - base.dweight).norm() / base.dweight.norm()).item() < 2e-3
+    assert ((b.dhidden.float() - base.dhidden.float()).norm() / base.dhidden.float().norm()).item() < 2e-3
