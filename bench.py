@@ -295,7 +295,19 @@ def main():
     barrier()
     sp_ms = max_over_ranks(sp0.elapsed_time(sp1), world, dev) / args.steps
     assert op.status()[0] == 0 and abs(float(op.loss.item()) - loss_val) <= 1e-6 * abs(loss_val)
-    single_pass = {"ms_per_step": sp_ms, "tokens_per_s": whole_job_tokens_per_s(T, world, sp_ms),
+    sp_acc = {}
+    n_sp_prof = 1 if args.capture else 3
+    for _ in range(n_sp_prof):
+        for k, (ms, n) in B.kdkl_profile_single_pass(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"],
+                                                      op.workspace, op.loss, op.dhidden, op.dweight,
+                                                      loss_mask=d["mask"], chunk=cfg.chunk,
+                                                      temperature=cfg.tau).items():
+            a = sp_acc.setdefault(k, [0.0, 0])
+            a[0] += ms
+            a[1] += n
+    sp_stages = {k: {"ms_per_step": v[0] / n_sp_prof, "launches_per_step": v[1] // n_sp_prof,
+                     "ms_per_launch": v[0] / v[1]} for k, v in sp_acc.items()}
+    single_pass = {"ms_per_step": sp_ms, "stages": sp_stages, "tokens_per_s": whole_job_tokens_per_s(T, world, sp_ms),
                    "flops_executed": 0.75 * cfg.flops, "tflops_executed_per_gpu": 0.75 * cfg.flops / (sp_ms * 1e-3) / 1e12,
                    "launches_per_step": op.launches,
                    "what": "forward + backward in one call without the second projection (6*T*H*V flops)"}

@@ -250,6 +250,15 @@ int kdkl_teacher_topk(const void* hidden_bf16, const void* weight_bf16, int64_t 
                       float temperature, void* workspace, size_t workspace_bytes, int32_t* topk_idx,
                       float* topk_val, float* lse, void* cuda_stream);
 
+/* The same per-stage measurement for kdkl_forward_backward. Stage 5 is then the in-place conversion of the stored
+ * exponentials into G (the place of the recompute GEMM); the other stages as above. */
+int kdkl_profile_single_pass(const void* hidden_bf16, const void* weight_bf16, const int32_t* topk_idx,
+                             const float* topk_val, const float* teacher_lse, const uint8_t* loss_mask, int64_t T,
+                             int64_t H, int64_t V, int32_t K, int64_t chunk, float temperature,
+                             const kdkl_options* opt, float grad_loss, void* workspace, size_t workspace_bytes,
+                             float* loss_out, void* dhidden, float* dweight, void* cuda_stream, float* stage_ms,
+                             int32_t* stage_launches);
+
 #define KDKL_FEATURE_MSE 0
 #define KDKL_FEATURE_COSINE 1
 

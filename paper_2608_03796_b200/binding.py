@@ -28,7 +28,7 @@ EXPORTS = [
     "kdkl_last_launch_count", "kdkl_logz_noalloc", "kdkl_forward_shard", "kdkl_forward_finish",
     "kdkl_wait_selftest", "kdkl_teacher_topk", "kdkl_teacher_topk_workspace_bytes",
     "kdkl_feature_loss", "kdkl_feature_loss_workspace_bytes", "kdkl_step_host_record", "kdkl_record_staging_bytes",
-    "kdkl_forward_backward",
+    "kdkl_forward_backward", "kdkl_profile_single_pass",
 ]
 
 FEATURE_MSE, FEATURE_COSINE = 0, 1
@@ -89,6 +89,10 @@ def lib() -> ctypes.CDLL:
     L.kdkl_profile_stages.restype = ctypes.c_int
     L.kdkl_profile_stages.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, f32, vp, sz,
                                       vp, vp, vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
+    L.kdkl_profile_single_pass.restype = ctypes.c_int
+    L.kdkl_profile_single_pass.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, f32, vp, sz,
+                                           vp, vp, vp, vp, ctypes.POINTER(ctypes.c_float),
+                                           ctypes.POINTER(ctypes.c_int32)]
     L.kdkl_gemm_bf16.restype = ctypes.c_int
     L.kdkl_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, vp, vp]
     L.kdkl_logz_noalloc.restype = ctypes.c_int
@@ -311,6 +315,25 @@ def kdkl_profile_stages(hidden, weight, topk_idx, topk_val, workspace, loss_out,
                                      _dptr(workspace), workspace.numel() * workspace.element_size(), _dptr(loss_out),
                                      _dptr(dhidden), _dptr(dweight), _stream(), ms, nl))
     return {STAGES[i]: (float(ms[i]), int(nl[i])) for i in range(8)}
+
+
+STAGES_SINGLE = ["prep", "fwd_gemm_lse_exp", "combine", "loss_reduce", "bwd_coef", "exp_to_dlogits", "dhidden_gemm",
+                 "dweight_gemm"]
+
+
+def kdkl_profile_single_pass(hidden, weight, topk_idx, topk_val, workspace, loss_out, dhidden, dweight, *,
+                             teacher_lse=None, loss_mask=None, chunk=0, temperature=1.0, opt=None, grad_loss=1.0):
+    """The single-pass step with an event between kernels: {stage: (ms, launches)}. Synchronises."""
+    T, H = hidden.shape
+    V = weight.shape[0]
+    K = topk_idx.shape[1]
+    ms = (ctypes.c_float * 8)()
+    nl = (ctypes.c_int32 * 8)()
+    _check(lib().kdkl_profile_single_pass(_dptr(hidden), _dptr(weight), _dptr(topk_idx), _dptr(topk_val),
+                                          _dptr(teacher_lse), _dptr(loss_mask), T, H, V, K, chunk, temperature,
+                                          _opt_ptr(opt), grad_loss, _dptr(workspace), workspace.numel(),
+                                          _dptr(loss_out), _dptr(dhidden), _dptr(dweight), _stream(), ms, nl))
+    return {STAGES_SINGLE[i]: (float(ms[i]), int(nl[i])) for i in range(8) if nl[i] > 0}
 
 
 def kdkl_gemm_bf16(A, B, C, M, N, K, a_mn=0, b_mn=0, status=None) -> None:

@@ -854,6 +854,38 @@ int kdkl_profile_stages(const void* hidden, const void* weight, const int32_t* t
   return rc;
 }
 
+// Same measurement for the single-pass step. Stage 5 is the in-place conversion of the stored exponentials
+// (the place the recompute GEMM has in the two-call step).
+int kdkl_profile_single_pass(const void* hidden, const void* weight, const int32_t* topk_idx, const float* topk_val,
+                             const float* teacher_lse, const uint8_t* loss_mask, int64_t T, int64_t H, int64_t V,
+                             int32_t K, int64_t chunk, float tau, const kdkl_options* opt, float grad_loss, void* ws,
+                             size_t ws_bytes, float* loss_out, void* dhidden, float* dweight, void* cuda_stream,
+                             float* stage_ms, int32_t* stage_launches) {
+  if (!stage_ms || !stage_launches) return KDKL_ERR_NULL;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  g_timer.on = true;
+  g_timer.ev.clear();
+  g_timer.stage.clear();
+  int rc = kdkl_forward_backward(hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, T, H, V, K, chunk, tau,
+                                 opt, grad_loss, ws, ws_bytes, loss_out, nullptr, dhidden, dweight, cuda_stream);
+  stage_mark(ST_END, st);
+  g_timer.on = false;
+  cudaError_t e = cudaStreamSynchronize(st);
+  for (int i = 0; i < ST_COUNT; ++i) { stage_ms[i] = 0.f; stage_launches[i] = 0; }
+  for (size_t i = 0; e == cudaSuccess && i + 1 < g_timer.ev.size(); ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, g_timer.ev[i], g_timer.ev[i + 1]) == cudaSuccess) {
+      stage_ms[g_timer.stage[i]] += ms;
+      stage_launches[g_timer.stage[i]] += 1;
+    }
+  }
+  for (cudaEvent_t ev : g_timer.ev) cudaEventDestroy(ev);
+  g_timer.ev.clear();
+  g_timer.stage.clear();
+  if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
+  return rc;
+}
+
 // ------------------------------------------------------------------ teacher top-K cache record
 constexpr long long kTopkTakeAllMaxV = 8192;
 struct TopkLayout { long long C, Cpad, n_tiles; int npad, cap, cpad; size_t hdr, zeros, part_m, part_s, thr, cnt, cidx, cval, total; };
