@@ -211,7 +211,8 @@ __global__ void step_coef_kernel(const float* __restrict__ Mv, const uint8_t* __
 //   G = a_t * 2^(s - lz2_t) - b_t p = (a_t * 2^(bias - lz2_t)) * e - b_t p at the support      (Eq. "grad")
 // One block per (row, 8192-column segment): the dense scaling is a streaming pass (read + write of the
 // chunk's G: the op is bound by HBM), then the row's support entries inside the segment are patched.
-constexpr int E2G_SEG = 8192;                  // columns per block: 256 threads x 4 vectors of 8
+constexpr int E2G_VEC = 8;                     // 16-byte vectors per thread
+constexpr int E2G_SEG = 256 * E2G_VEC * 8;     // columns per block: 256 threads x E2G_VEC vectors of 8
 __global__ void __launch_bounds__(256)
 e_to_g_kernel(__nv_bfloat16* __restrict__ G, long long ldg /* elements per row */, int n_cols /* V rounded up to 8 */,
               int V /* columns the forward sweep wrote; the rest of the last vector is stale memory */,
@@ -231,14 +232,14 @@ e_to_g_kernel(__nv_bfloat16* __restrict__ G, long long ldg /* elements per row *
   }
   const float scale = a * exp2f(bias - lz2[row]);
   bool bad = false;                            // an exponential that overflowed bf16 (scaled logit beyond about 190)
-  uint4 buf[4];
+  uint4 buf[E2G_VEC];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < E2G_VEC; ++i) {
     const int v = v_begin + threadIdx.x + i * 256;
     if (v < v_end) buf[i] = g_row[v];
   }
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < E2G_VEC; ++i) {
     const int v = v_begin + threadIdx.x + i * 256;
     if (v < v_end) {
       __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&buf[i]);
