@@ -43,6 +43,10 @@ def _case(T, H, V, K, seed, mask_mode=0, dup=False):
     (700, 72, 1001, 7, 256, 0.5, 2, True, {"grad_loss": -2.0}),
     (1300, 128, 3000, 33, 0, 2.0, 2, False, {"dh32": 1, "accumulate": 1}),
     (5, 8, 9, 9, 1, 1.0, 0, False, {}),
+    (20, 64, 1500, 1024, 0, 1.0, 0, False, {}),            # the largest supported K
+    (40, 64, 255, 5, 0, 2.0, 1, False, {}),                # vocabulary smaller than one tile
+    (257, 4104, 520, 3, 256, 1.0, 0, False, {}),           # ragged last k-block, rows one past a pair tile
+    (130, 72, 8200, 17, 37, 1.0, 1, True, {}),             # vocabulary just past one conversion segment, odd chunk
 ])
 def test_single_pass_matches_oracle_and_two_call_path(T, H, V, K, chunk, tau, mask_mode, dup, opts):
     dev = torch.device("cuda:0")
