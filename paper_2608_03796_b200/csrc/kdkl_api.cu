@@ -474,6 +474,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
       // the forward call left the exponentials of this (only) chunk in G: no second projection
       const int n_cols = (int)(((V + 7) / 8) * 8);
       const int n_seg = (n_cols + E2G_SEG - 1) / E2G_SEG;
+      if ((long long)rows * n_seg > 2147483647ll) return KDKL_ERR_SHAPE;   // one block per (row, segment)
       e_to_g_kernel<<<(unsigned)(rows * n_seg), 256, 0, st>>>(
           G, L.Vpad, n_cols, (int)V, at<float>(ws, L.coefA) + s0, at<float>(ws, L.coefB) + s0,
           at<float>(ws, L.lz2) + s0, at<int>(ws, L.idx_sorted) + s0 * K, at<float>(ws, L.p_sorted) + s0 * K,
@@ -625,6 +626,7 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
     stage_mark(ST_B1, st);
     const int n_cols = (int)(((V + 7) / 8) * 8);
     const int n_seg = (n_cols + E2G_SEG - 1) / E2G_SEG;
+      if ((long long)rows * n_seg > 2147483647ll) return KDKL_ERR_SHAPE;   // one block per (row, segment)
     e_to_g_kernel<<<(unsigned)(rows * n_seg), 256, 0, st>>>(
         G, L.Vpad, n_cols, (int)V, at<float>(ws, L.coefA) + s0, at<float>(ws, L.coefB) + s0, at<float>(ws, L.lz2) + s0,
         at<int>(ws, L.idx_sorted) + s0 * K, at<float>(ws, L.p_sorted) + s0 * K, at<int>(ws, L.nvalid) + s0, K, kExpBias,
