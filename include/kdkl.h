@@ -285,6 +285,14 @@ int kdkl_feature_loss(const void* student_bf16, const void* teacher_bf16, const 
                       int32_t accumulate, void* workspace, size_t workspace_bytes, float* loss_out,
                       float* loss_per_token, void* dstudent_bf16, void* cuda_stream);
 
+/* The same record with one projection instead of two: the first sweep also stores the fp32 logits of the pass
+ * (4096 tokens at a time) and the candidates are collected from them instead of being recomputed. Costs
+ * 4096 x V x 4 bytes more workspace (2 GiB at V = 131072); same results, same limits, same errors. */
+size_t kdkl_teacher_topk_stored_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K);
+int kdkl_teacher_topk_stored(const void* hidden_bf16, const void* weight_bf16, int64_t T, int64_t H, int64_t V,
+                             int32_t K, float temperature, void* workspace, size_t workspace_bytes,
+                             int32_t* topk_idx, float* topk_val, float* lse, void* cuda_stream);
+
 /* Exercises the bounded wait every kernel of this library uses on its mbarriers: one thread waits on
  * a barrier that nothing completes, gives up after limit_ns (1 .. 1e9) and the kernel returns normally.
  * status: device int32[2], zeroed by the caller; afterwards {KDKL_ERR_TIMEOUT, 99}. The context stays

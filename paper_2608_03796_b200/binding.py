@@ -28,7 +28,8 @@ EXPORTS = [
     "kdkl_last_launch_count", "kdkl_logz_noalloc", "kdkl_forward_shard", "kdkl_forward_finish",
     "kdkl_wait_selftest", "kdkl_teacher_topk", "kdkl_teacher_topk_workspace_bytes",
     "kdkl_feature_loss", "kdkl_feature_loss_workspace_bytes", "kdkl_step_host_record", "kdkl_record_staging_bytes",
-    "kdkl_forward_backward", "kdkl_profile_single_pass",
+    "kdkl_forward_backward", "kdkl_profile_single_pass", "kdkl_teacher_topk_stored",
+    "kdkl_teacher_topk_stored_workspace_bytes",
 ]
 
 FEATURE_MSE, FEATURE_COSINE = 0, 1
@@ -99,6 +100,10 @@ def lib() -> ctypes.CDLL:
     L.kdkl_logz_noalloc.argtypes = [vp, vp, i64, i64, i64, f32, vp, vp]
     L.kdkl_teacher_topk_workspace_bytes.restype = sz
     L.kdkl_teacher_topk_workspace_bytes.argtypes = [i64, i64, i64, i32]
+    L.kdkl_teacher_topk_stored_workspace_bytes.restype = sz
+    L.kdkl_teacher_topk_stored_workspace_bytes.argtypes = [i64, i64, i64, i32]
+    L.kdkl_teacher_topk_stored.restype = ctypes.c_int
+    L.kdkl_teacher_topk_stored.argtypes = [vp, vp, i64, i64, i64, i32, f32, vp, sz, vp, vp, vp, vp]
     L.kdkl_teacher_topk.restype = ctypes.c_int
     L.kdkl_teacher_topk.argtypes = [vp, vp, i64, i64, i64, i32, f32, vp, sz, vp, vp, vp, vp]
     L.kdkl_feature_loss_workspace_bytes.restype = sz
@@ -349,18 +354,20 @@ def kdkl_logz_noalloc(hidden, weight, logz_out, temperature=1.0) -> None:
     _check(lib().kdkl_logz_noalloc(_dptr(hidden), _dptr(weight), T, H, V, temperature, _dptr(logz_out), _stream()))
 
 
-def kdkl_teacher_topk(hidden, weight, K, temperature=1.0, workspace=None):
-    """The teacher cache record: (topk_idx int32 [T,K], topk_val fp32 [T,K] descending, lse fp32 [T], workspace)."""
+def kdkl_teacher_topk(hidden, weight, K, temperature=1.0, workspace=None, stored=False):
+    """The teacher cache record: (topk_idx int32 [T,K], topk_val fp32 [T,K] descending, lse fp32 [T], workspace).
+    stored=True keeps the fp32 logits of each 4096-token pass in the workspace (one projection instead of two)."""
     T, H = hidden.shape
     V = weight.shape[0]
+    size_fn = lib().kdkl_teacher_topk_stored_workspace_bytes if stored else lib().kdkl_teacher_topk_workspace_bytes
+    call = lib().kdkl_teacher_topk_stored if stored else lib().kdkl_teacher_topk
     if workspace is None:
-        workspace = torch.empty(lib().kdkl_teacher_topk_workspace_bytes(T, H, V, K), dtype=torch.uint8,
-                                device=hidden.device)
+        workspace = torch.empty(size_fn(T, H, V, K), dtype=torch.uint8, device=hidden.device)
     idx = torch.empty(T, K, dtype=torch.int32, device=hidden.device)
     val = torch.empty(T, K, dtype=torch.float32, device=hidden.device)
     lse = torch.empty(T, dtype=torch.float32, device=hidden.device)
-    _check(lib().kdkl_teacher_topk(_dptr(hidden), _dptr(weight), T, H, V, K, temperature, _dptr(workspace),
-                                   workspace.numel(), _dptr(idx), _dptr(val), _dptr(lse), _stream()))
+    _check(call(_dptr(hidden), _dptr(weight), T, H, V, K, temperature, _dptr(workspace), workspace.numel(),
+                _dptr(idx), _dptr(val), _dptr(lse), _stream()))
     return idx, val, lse, workspace
 
 

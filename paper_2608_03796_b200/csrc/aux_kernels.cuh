@@ -544,6 +544,42 @@ topk_threshold_kernel(const float* __restrict__ part_m, const float* __restrict_
   }
 }
 
+// Teacher cache with stored logits: the candidates of a row are collected from the fp32 logits the first
+// sweep stored, by the same test the recompute epilogue applies (z * scale >= the row's threshold, the
+// same fp32 product). One block per (row, 8192-column segment); a streaming read of the logits.
+constexpr int COLLECT_SEG = 8192;
+__global__ void __launch_bounds__(256)
+topk_collect_kernel(const float* __restrict__ z, long long ldz, int V, float scale_log2, const float* __restrict__ thr,
+                    int* __restrict__ cand_cnt, int* __restrict__ cand_idx, float* __restrict__ cand_val, int cap,
+                    int n_seg) {
+  const long long row = blockIdx.x / n_seg;
+  const int c_begin = (int)(blockIdx.x - row * n_seg) * COLLECT_SEG;
+  const float t = thr[row];
+  const float4* zr = reinterpret_cast<const float4*>(z + row * ldz);
+  float4 buf[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int c = c_begin + (threadIdx.x + i * 256) * 4;
+    if (c < V) buf[i] = zr[c >> 2];                     // ldz is a multiple of 4: the last vector may hold stale columns
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int c = c_begin + (threadIdx.x + i * 256) * 4;
+    if (c >= V) continue;
+    const float v[4] = {buf[i].x, buf[i].y, buf[i].z, buf[i].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (c + j < V && v[j] * scale_log2 >= t) {
+        const int slot = atomicAdd(cand_cnt + row, 1);
+        if (slot < cap) {
+          cand_idx[row * cap + slot] = c + j;
+          cand_val[row * cap + slot] = v[j];
+        }
+      }
+    }
+  }
+}
+
 // Sweep 2 -> record. One warp (block) per row: sort the emitted candidates by (logit descending, index
 // ascending) and keep the first K. More candidates than the list holds is reported, not hidden.
 __global__ void __launch_bounds__(32)

@@ -22,6 +22,8 @@
 //   EPI_DLOGITS     backward: G = a_t * exp(z/tau - logZ) - b_t * p at the support, cast to
 //                   bf16 (Eq. "grad", Algorithm 1 backward)
 //   EPI_TOPK        teacher cache: emits the (column, logit) pairs above a per-row threshold
+//   EPI_LSE_Z       EPI_LSE that also stores the fp32 logits (teacher cache with one projection: the selection then
+//                   reads them back instead of projecting again)
 //   EPI_LSE_E       EPI_LSE that also stores the unnormalised exponentials 2^(z log2e / tau - 64) in bf16, for the
 //                   single-pass forward + backward (no second projection: G is made from them once log Z is known)
 #pragma once
@@ -56,7 +58,7 @@ struct GemmCfg {
                                     2 * MAX_LIVE_KB /*live k-block list*/ + 2 * MAX_LIVE_M /*live row-tile list*/;
 };
 
-enum { EPI_STORE_F32 = 0, EPI_STORE_BF16 = 1, EPI_LSE = 2, EPI_DLOGITS = 3, EPI_TOPK = 4, EPI_LSE_E = 5 };
+enum { EPI_STORE_F32 = 0, EPI_STORE_BF16 = 1, EPI_LSE = 2, EPI_DLOGITS = 3, EPI_TOPK = 4, EPI_LSE_E = 5, EPI_LSE_Z = 6 };
 
 // EPI_LSE_E stores e = 2^(z log2e / tau - kExpBias) in bf16: representable for scaled logits in about
 // [-62, 190] (bf16 has fp32's exponent range), i.e. far below any weight that matters and far above any sane logit.
@@ -360,8 +362,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int lg = warp & 3;                   // TMEM lane group this warp may read
     const int row_in_tile = lg * 32 + lane;
     constexpr bool kBf16Out = (EPI == EPI_STORE_BF16 || EPI == EPI_DLOGITS || EPI == EPI_LSE_E);
-    constexpr bool kLse = (EPI == EPI_LSE || EPI == EPI_LSE_E);
-    constexpr bool kStore = (EPI == EPI_STORE_F32 || kBf16Out);
+    constexpr bool kLse = (EPI == EPI_LSE || EPI == EPI_LSE_E || EPI == EPI_LSE_Z);
+    constexpr bool kStore = (EPI == EPI_STORE_F32 || EPI == EPI_LSE_Z || kBf16Out);
     uint32_t lt = 0, nbox = 0;
     bool ok = true;
     // Dead row tiles (every token ignored) belong to no work unit. LSE / TOPK have nothing to write for
@@ -370,7 +372,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (mskip && kStore && !(EPI == EPI_STORE_F32 && p.accumulate)) {
       const int n_dead = p.m_tiles - m_count;
       const int zero_units = n_dead * p.n_tiles * p.k_splits;
-      constexpr int BOX_COLS = (EPI == EPI_STORE_F32) ? 32 : 64;
+      constexpr int BOX_COLS = kBf16Out ? 64 : 32;
       for (int zu = worker; zu < zero_units; zu += num_workers) {
         const int split = zu / (n_dead * p.n_tiles);
         const int rem = zu - split * (n_dead * p.n_tiles);
@@ -514,7 +516,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (lane == 0) bulk_wait_read<1>();   // the store issued two boxes ago has read this box
             __syncwarp();
           }
-          if (EPI == EPI_STORE_F32) {
+          if (!kBf16Out) {                     // fp32 boxes: EPI_STORE_F32, EPI_LSE_Z
 #pragma unroll
             for (int c = 0; c < 8; ++c)
               st_shared_v4(srow + ((c ^ (lane & 7)) << 4), r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);

@@ -890,9 +890,13 @@ int kdkl_profile_single_pass(const void* hidden, const void* weight, const int32
 
 // ------------------------------------------------------------------ teacher top-K cache record
 constexpr long long kTopkTakeAllMaxV = 8192;
-struct TopkLayout { long long C, Cpad, n_tiles; int npad, cap, cpad; size_t hdr, zeros, part_m, part_s, thr, cnt, cidx, cval, total; };
+struct TopkLayout {
+  long long C, Cpad, n_tiles, ldz;
+  int npad, cap, cpad;
+  size_t hdr, zeros, part_m, part_s, thr, cnt, cidx, cval, z, total;
+};
 static int pow2_at_least(long long x) { int p = 32; while (p < x) p <<= 1; return p; }
-static TopkLayout topk_layout(long long T, long long V, int K) {
+static TopkLayout topk_layout(long long T, long long V, int K, bool stored = false) {
   TopkLayout L;
   L.C = T < 4096 ? T : 4096;
   L.Cpad = (long long)up((size_t)L.C, 128);
@@ -916,6 +920,8 @@ static TopkLayout topk_layout(long long T, long long V, int K) {
   L.cnt = take((size_t)L.Cpad * 4);
   L.cidx = take((size_t)L.Cpad * L.cap * 4);
   L.cval = take((size_t)L.Cpad * L.cap * 4);
+  L.ldz = (long long)up((size_t)V, 32);                    // fp32 logits of one pass, when they are stored
+  L.z = take(stored ? (size_t)L.Cpad * L.ldz * 4 : 0);
   L.total = o;
   return L;
 }
@@ -925,8 +931,14 @@ size_t kdkl_teacher_topk_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_
   return topk_layout(T, V, K).total;
 }
 
-int kdkl_teacher_topk(const void* hidden, const void* weight, int64_t T, int64_t H, int64_t V, int32_t K, float tau,
-                      void* ws, size_t ws_bytes, int32_t* topk_idx, float* topk_val, float* lse, void* cuda_stream) {
+size_t kdkl_teacher_topk_stored_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K) {
+  if (T < 1 || H < 1 || V < 1 || K < 1) return 0;
+  return topk_layout(T, V, K, true).total;
+}
+
+static int teacher_topk_impl(const void* hidden, const void* weight, int64_t T, int64_t H, int64_t V, int32_t K,
+                             float tau, void* ws, size_t ws_bytes, int32_t* topk_idx, float* topk_val, float* lse,
+                             void* cuda_stream, bool stored) {
   g_launches = 0;
   if (!hidden || !weight || !ws || !topk_idx || !topk_val || !lse) return KDKL_ERR_NULL;
   if (T < 1 || H < 1 || V < 1 || K < 1 || K > 256 || K > V || (H % 8) != 0 || V > (1ll << 20) || T >= (1ll << 31))
@@ -934,7 +946,7 @@ int kdkl_teacher_topk(const void* hidden, const void* weight, int64_t T, int64_t
   if ((V + BN - 1) / BN < K && V > kTopkTakeAllMaxV) return KDKL_ERR_SHAPE;   // needs V >= 256 K or V <= 8192
   if (!(tau > 0.f)) return KDKL_ERR_ARG;
   if (((uintptr_t)hidden & 15) || ((uintptr_t)weight & 15) || ((uintptr_t)ws & 15)) return KDKL_ERR_ALIGN;
-  const TopkLayout L = topk_layout(T, V, K);
+  const TopkLayout L = topk_layout(T, V, K, stored);
   if (ws_bytes < L.total) return KDKL_ERR_WORKSPACE;
   DeviceInfo di;
   int rc = device_info(&di);
@@ -959,16 +971,31 @@ int kdkl_teacher_topk(const void* hidden, const void* weight, int64_t T, int64_t
     p.scale_log2 = kLog2e / tau; p.Ktop = 1;
     p.nvalid = at<int>(ws, L.zeros); p.idx_sorted = at<int>(ws, L.zeros);     // no teacher entries to gather
     p.part_m = at<float>(ws, L.part_m); p.part_s = at<float>(ws, L.part_s); p.part_stride = L.Cpad;
-    // sweep 1: per-tile maxima and sum-exp
-    if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA, p, di.sm_count, st))) return rc;
+    // sweep 1: per-tile maxima and sum-exp (and, in the stored form, the fp32 logits themselves)
+    if (stored) {
+      CUtensorMap tmZ;
+      if ((rc = make_tmap_out_f32(&tmZ, at<float>(ws, L.z), (uint64_t)V, (uint64_t)rows, (uint64_t)L.ldz))) return rc;
+      if ((rc = launch_gemm<EPI_LSE_Z, false, false>(tmA, tmW, tmZ, p, di.sm_count, st))) return rc;
+    } else {
+      if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA, p, di.sm_count, st))) return rc;
+    }
     topk_threshold_kernel<<<(unsigned)rows, 32, (size_t)L.npad * 4, st>>>(
         at<float>(ws, L.part_m), at<float>(ws, L.part_s), L.Cpad, (int)L.n_tiles, L.npad, K, at<float>(ws, L.thr),
         at<int>(ws, L.cnt), lse + s0);
     KDKL_LAUNCHED("topk_threshold_kernel");
-    // sweep 2: recompute, emit everything at or above the row's threshold
-    p.thr = at<float>(ws, L.thr); p.cand_cnt = at<int>(ws, L.cnt);
-    p.cand_idx = at<int>(ws, L.cidx); p.cand_val = at<float>(ws, L.cval); p.cand_cap = L.cap;
-    if ((rc = launch_gemm<EPI_TOPK, false, false>(tmA, tmW, tmA, p, di.sm_count, st))) return rc;
+    if (stored) {
+      // collect everything at or above the row's threshold from the stored logits
+      const int n_seg = (int)((V + COLLECT_SEG - 1) / COLLECT_SEG);
+      topk_collect_kernel<<<(unsigned)(rows * n_seg), 256, 0, st>>>(
+          at<float>(ws, L.z), L.ldz, (int)V, p.scale_log2, at<float>(ws, L.thr), at<int>(ws, L.cnt),
+          at<int>(ws, L.cidx), at<float>(ws, L.cval), L.cap, n_seg);
+      KDKL_LAUNCHED("topk_collect_kernel");
+    } else {
+      // sweep 2: recompute, emit everything at or above the row's threshold
+      p.thr = at<float>(ws, L.thr); p.cand_cnt = at<int>(ws, L.cnt);
+      p.cand_idx = at<int>(ws, L.cidx); p.cand_val = at<float>(ws, L.cval); p.cand_cap = L.cap;
+      if ((rc = launch_gemm<EPI_TOPK, false, false>(tmA, tmW, tmA, p, di.sm_count, st))) return rc;
+    }
     KDKL_CUDA(cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.cpad * 8));
     topk_select_kernel<<<(unsigned)rows, 32, (size_t)L.cpad * 8, st>>>(
         at<int>(ws, L.cnt), at<int>(ws, L.cidx), at<float>(ws, L.cval), L.cap, L.cpad, K, topk_idx, topk_val, s0,
@@ -976,6 +1003,17 @@ int kdkl_teacher_topk(const void* hidden, const void* weight, int64_t T, int64_t
     KDKL_LAUNCHED("topk_select_kernel");
   }
   return KDKL_OK;
+}
+
+int kdkl_teacher_topk(const void* hidden, const void* weight, int64_t T, int64_t H, int64_t V, int32_t K, float tau,
+                      void* ws, size_t ws_bytes, int32_t* topk_idx, float* topk_val, float* lse, void* cuda_stream) {
+  return teacher_topk_impl(hidden, weight, T, H, V, K, tau, ws, ws_bytes, topk_idx, topk_val, lse, cuda_stream, false);
+}
+
+int kdkl_teacher_topk_stored(const void* hidden, const void* weight, int64_t T, int64_t H, int64_t V, int32_t K,
+                             float tau, void* ws, size_t ws_bytes, int32_t* topk_idx, float* topk_val, float* lse,
+                             void* cuda_stream) {
+  return teacher_topk_impl(hidden, weight, T, H, V, K, tau, ws, ws_bytes, topk_idx, topk_val, lse, cuda_stream, true);
 }
 
 // ------------------------------------------------------------------ hidden-state feature loss

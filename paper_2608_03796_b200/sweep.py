@@ -59,13 +59,14 @@ def worker(method: str, name: str, steps: int) -> dict:
     torch.cuda.reset_peak_memory_stats()
     out = {"method": method, "workload": name, "T": cfg.T, "H": cfg.H, "V": cfg.V, "K": cfg.K, "chunk": cfg.chunk,
            "input_gb": torch.cuda.memory_allocated() / 1e9}
-    if method == "teacher":
+    if method in ("teacher", "teacher_stored"):
         # the teacher cache kernel on the same shape: hidden / weight play the teacher's role
-        _, _, _, tws = B.kdkl_teacher_topk(d["hidden"], d["weight"], cfg.K, temperature=cfg.tau)
+        st = method == "teacher_stored"
+        _, _, _, tws = B.kdkl_teacher_topk(d["hidden"], d["weight"], cfg.K, temperature=cfg.tau, stored=st)
         out["workspace_gb"] = tws.numel() / 1e9
 
         def step():
-            B.kdkl_teacher_topk(d["hidden"], d["weight"], cfg.K, temperature=cfg.tau, workspace=tws)
+            B.kdkl_teacher_topk(d["hidden"], d["weight"], cfg.K, temperature=cfg.tau, workspace=tws, stored=st)
             return torch.zeros(1)
     elif method in ("fused", "single"):
         op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev)
@@ -147,8 +148,8 @@ def worker(method: str, name: str, steps: int) -> dict:
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / steps
         out.update(ms_per_iter=ms, it_per_s=1e3 / ms, tokens_per_s=cfg.T / (ms * 1e-3),
-                   # executed projections: fused 4 (8*T*H*V), single / dense / fwdchunk 3, teacher 2
-                   tflops={"fused": 1.0, "teacher": 0.5}.get(method, 0.75) * cfg.flops / (ms * 1e-3) / 1e12,
+                   # executed projections: fused 4 (8*T*H*V), single / dense / fwdchunk 3, teacher 2, teacher_stored 1
+                   tflops={"fused": 1.0, "teacher": 0.5, "teacher_stored": 0.25}.get(method, 0.75) * cfg.flops / (ms * 1e-3) / 1e12,
                    loss=float(loss.item()),
                    peak_gb=torch.cuda.max_memory_allocated() / 1e9,
                    driver_delta_gb=(free0 - torch.cuda.mem_get_info()[0]) / 1e9)

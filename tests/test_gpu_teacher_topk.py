@@ -24,9 +24,9 @@ def _case(T, H, V, seed):
     return h, W
 
 
-def _check(h, W, K, tau):
+def _check(h, W, K, tau, stored=False):
     dev = torch.device("cuda:0")
-    idx, val, lse, ws = B.kdkl_teacher_topk(h.to(dev), W.to(dev), K, temperature=tau)
+    idx, val, lse, ws = B.kdkl_teacher_topk(h.to(dev), W.to(dev), K, temperature=tau, stored=stored)
     code, _ = B.kdkl_status(ws)
     assert code == 0
     idx, val, lse = idx.cpu().numpy(), val.cpu().double().numpy(), lse.cpu().double().numpy()
@@ -48,11 +48,24 @@ def _check(h, W, K, tau):
     return idx, val, lse, o
 
 
+@pytest.mark.parametrize("stored", [False, True])
 @pytest.mark.parametrize("T,H,V,K,tau", [(300, 264, 4120, 16, 1.0), (70, 64, 300, 100, 2.0), (5, 8, 9, 9, 1.0),
-                                         (1100, 128, 70000, 100, 1.0)])
-def test_teacher_topk_matches_oracle(T, H, V, K, tau):
+                                         (1100, 128, 70000, 100, 1.0), (4200, 64, 4099, 8, 1.0)])
+def test_teacher_topk_matches_oracle(T, H, V, K, tau, stored):
+    """Both forms: two projections, and one projection with the fp32 logits of each pass kept in the workspace.
+    The last shape spans two 4096-token passes with a vocabulary that is not a multiple of 4."""
     h, W = _case(T, H, V, seed=T + V)
-    _check(h, W, K, tau)
+    _check(h, W, K, tau, stored)
+
+
+def test_stored_form_gives_the_same_record_bit_for_bit():
+    """Same logits, same threshold, same selection: the two forms must agree exactly."""
+    dev = torch.device("cuda:0")
+    h, W = _case(700, 136, 9000, seed=11)
+    a = B.kdkl_teacher_topk(h.to(dev), W.to(dev), 32, temperature=1.3)
+    b = B.kdkl_teacher_topk(h.to(dev), W.to(dev), 32, temperature=1.3, stored=True)
+    assert B.kdkl_status(a[3])[0] == 0 and B.kdkl_status(b[3])[0] == 0
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])
 
 
 def test_ties_break_by_smaller_index_and_overflow_is_reported():
@@ -103,6 +116,11 @@ def test_fullsize_sampled_rows():
     W = I.weight(cfg, device=dev)
     idx, val, lse, ws = B.kdkl_teacher_topk(h, W, cfg.K, temperature=1.0)
     assert B.kdkl_status(ws)[0] == 0
+    del ws
+    sidx, sval, slse, sws = B.kdkl_teacher_topk(h, W, cfg.K, temperature=1.0, stored=True)   # one projection
+    assert B.kdkl_status(sws)[0] == 0
+    assert torch.equal(sidx, idx) and torch.equal(sval, val) and torch.equal(slse, lse)
+    del sws, sidx, sval, slse
     R = I.sample_rows(cfg, 24).to(dev)
     o = teacher_topk_oracle(h[R].cpu().double().numpy(), W.cpu().double().numpy(), cfg.K, tau=1.0)
     gi, gv = idx[R].cpu().numpy(), val[R].cpu().double().numpy()
