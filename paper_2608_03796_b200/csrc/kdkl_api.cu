@@ -259,6 +259,71 @@ static Tp* at(void* ws, size_t off) { return reinterpret_cast<Tp*>(reinterpret_c
 
 static int next_pow2(int x) { int p = 2; while (p < x) p <<= 1; return p; }
 
+// The two output GEMMs of one chunk, shared by kdkl_backward and kdkl_forward_backward: G holds the chunk's
+// dlogits (bf16 [rows, Vpad]).
+//   dH[chunk] = G W        (M = rows, N = H, K = V; split-K with a fixed-order fix-up when the tiles are few)
+//   dW (+)= G^T h[chunk]   (M = V, N = H, K = rows; both operands MN-major: G is [t, v] with v contiguous,
+//                           h is [t, h] with h contiguous)
+struct ChunkOut {
+  const __nv_bfloat16* G; const __nv_bfloat16* hA; void* dhidden; long long s0, rows, H, V;
+  const WsLayout* L; const kdkl_options* o; WsHeader* hdr; void* ws; const int* go;
+  const uint8_t* live_m;   // row-tile flags for the dH GEMM (nullptr: none)
+  const uint8_t* live_c;   // the chunk's row-tile flags for the dW contraction (nullptr: none)
+  int accumulate_dw;
+};
+static int launch_chunk_outputs(const ChunkOut& c, const CUtensorMap& tmWmn, const CUtensorMap& tmdW, int sm_count,
+                                cudaStream_t st) {
+  const WsLayout& L = *c.L;
+  const long long rows = c.rows, H = c.H, V = c.V, s0 = c.s0;
+  int rc;
+  CUtensorMap tmG, tmGmn, tmhmn, tmdH;
+  stage_mark(ST_B2, st);
+  if ((rc = make_tmap_bf16(&tmG, c.G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, BK, BM))) return rc;
+  GemmParams p2;
+  memset(&p2, 0, sizeof(p2));
+  p2.M = (int)rows; p2.N = (int)H; p2.K = (int)V;
+  p2.m_tiles = (int)((rows + kTileM - 1) / kTileM); p2.n_tiles = (int)((H + BN - 1) / BN); p2.m_inner = 0;
+  p2.status = &c.hdr->status; p2.go = c.go;
+  p2.m_live = c.live_m;              // dead row tiles: their dH rows are written as zeros
+  // a short last chunk may want a different split; never more than the workspace was sized for
+  int sp = choose_k_splits((long long)p2.m_tiles * p2.n_tiles, (V + BK - 1) / BK);
+  if (sp > L.dh_splits) sp = L.dh_splits;
+  p2.k_splits = sp;
+  __nv_bfloat16* dh16 = c.o->dhidden_dtype == 0 ? reinterpret_cast<__nv_bfloat16*>(c.dhidden) + s0 * H : nullptr;
+  float* dh32 = c.o->dhidden_dtype == 1 ? reinterpret_cast<float*>(c.dhidden) + s0 * H : nullptr;
+  if (sp > 1) {
+    // partial sums of each split go to fp32 slabs [split][Cpad, H]; a fixed-order fix-up adds them
+    float* part = at<float>(c.ws, L.dh_part);
+    p2.split_rows = (int)L.Cpad;
+    if ((rc = make_tmap_out_f32(&tmdH, part, (uint64_t)H, (uint64_t)sp * L.Cpad, (uint64_t)H))) return rc;
+    if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, sm_count, st))) return rc;
+    const long long n4 = rows * H / 4;
+    splitk_fixup_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(part, (long long)L.Cpad * H, sp, n4, dh16, dh32,
+                                                                     c.go);
+    KDKL_LAUNCHED("splitk_fixup_kernel");
+  } else if (dh16 != nullptr) {
+    if ((rc = make_tmap_out_bf16(&tmdH, dh16, (uint64_t)H, (uint64_t)rows, (uint64_t)H))) return rc;
+    if ((rc = launch_gemm<EPI_STORE_BF16, false, true>(tmG, tmWmn, tmdH, p2, sm_count, st))) return rc;
+  } else {
+    if ((rc = make_tmap_out_f32(&tmdH, dh32, (uint64_t)H, (uint64_t)rows, (uint64_t)H))) return rc;
+    if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, sm_count, st))) return rc;
+  }
+
+  if ((rc = make_tmap_bf16(&tmGmn, c.G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, 64, BK))) return rc;
+  if ((rc = make_tmap_bf16(&tmhmn, c.hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, 64, BK))) return rc;
+  GemmParams p3;
+  memset(&p3, 0, sizeof(p3));
+  p3.M = (int)V; p3.N = (int)H; p3.K = (int)rows;
+  p3.m_tiles = (int)((V + kTileM - 1) / kTileM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0; p3.k_splits = 1;
+  p3.status = &c.hdr->status; p3.go = c.go;
+  p3.accumulate = c.accumulate_dw;
+  // dead row tiles of G are zeros: they are left out of the contraction over tokens (the kernel takes up to 32 flags)
+  p3.k_live = (rows <= 32ll * kTileM && (rows + BK - 1) / BK <= MAX_LIVE_KB) ? c.live_c : nullptr;
+  stage_mark(ST_B3, st);
+  return launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, tmdW, p3, sm_count, st);
+}
+
+
 }  // namespace kdkl
 
 using namespace kdkl;
@@ -447,7 +512,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
     const uint8_t* live_c = live ? live + ci * L.tiles_per_chunk : nullptr;
     const __nv_bfloat16* hA = reinterpret_cast<const __nv_bfloat16*>(hidden) + s0 * H;
-    CUtensorMap tmA, tmG, tmGmn, tmhmn;
+    CUtensorMap tmA;
     if ((rc = make_tmap_bf16(&tmA, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, BK, BM))) return rc;
 
     // B1: recompute logits, G = coefA * q - coefB * p
@@ -483,57 +548,10 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     } else {
       if ((rc = launch_gemm<EPI_DLOGITS, false, false>(tmA, tmW, tmGout, p, di.sm_count, st))) return rc;
     }
-    stage_mark(ST_B2, st);
 
-    // B2: dH[chunk] = G W   (M = rows, N = H, K = V)
-    if ((rc = make_tmap_bf16(&tmG, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, BK, BM))) return rc;
-    GemmParams p2;
-    memset(&p2, 0, sizeof(p2));
-    p2.M = (int)rows; p2.N = (int)H; p2.K = (int)V;
-    p2.m_tiles = (int)((rows + kTileM - 1) / kTileM); p2.n_tiles = (int)((H + BN - 1) / BN); p2.m_inner = 0;
-    p2.status = &hdr->status; p2.go = go;
-    p2.accumulate = 0;
-    p2.m_live = live_m;                // their dH rows are zeros
-    // a short last chunk may want a different split; never more than the workspace was sized for
-    int sp = choose_k_splits((long long)p2.m_tiles * p2.n_tiles, (V + BK - 1) / BK);
-    if (sp > L.dh_splits) sp = L.dh_splits;
-    p2.k_splits = sp;
-    CUtensorMap tmdH;
-    if (sp > 1) {
-      // partial sums of each split go to fp32 slabs [split][Cpad, H]; a fixed-order fix-up adds them
-      float* part = at<float>(ws, L.dh_part);
-      p2.split_rows = (int)L.Cpad;
-      if ((rc = make_tmap_out_f32(&tmdH, part, (uint64_t)H, (uint64_t)sp * L.Cpad, (uint64_t)H))) return rc;
-      if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
-      const long long n4 = rows * H / 4;
-      splitk_fixup_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(
-          part, (long long)L.Cpad * H, sp, n4, o.dhidden_dtype == 0 ? reinterpret_cast<__nv_bfloat16*>(dhidden) + s0 * H : nullptr,
-          o.dhidden_dtype == 1 ? reinterpret_cast<float*>(dhidden) + s0 * H : nullptr, go);
-      KDKL_LAUNCHED("splitk_fixup_kernel");
-    } else if (o.dhidden_dtype == 0) {
-      if ((rc = make_tmap_out_bf16(&tmdH, reinterpret_cast<__nv_bfloat16*>(dhidden) + s0 * H, (uint64_t)H,
-                                   (uint64_t)rows, (uint64_t)H))) return rc;
-      if ((rc = launch_gemm<EPI_STORE_BF16, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
-    } else {
-      if ((rc = make_tmap_out_f32(&tmdH, reinterpret_cast<float*>(dhidden) + s0 * H, (uint64_t)H, (uint64_t)rows,
-                                  (uint64_t)H))) return rc;
-      if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
-    }
-
-    // B3: dW (+)= G^T h   (M = V, N = H, K = rows)
-    // both operands MN-major: G is [t, v] with v (= M) contiguous, h is [t, h] with h (= N) contiguous
-    if ((rc = make_tmap_bf16(&tmGmn, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, 64, BK))) return rc;
-    if ((rc = make_tmap_bf16(&tmhmn, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, 64, BK))) return rc;
-    GemmParams p3;
-    memset(&p3, 0, sizeof(p3));
-    p3.M = (int)V; p3.N = (int)H; p3.K = (int)rows;
-    p3.m_tiles = (int)((V + kTileM - 1) / kTileM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0; p3.k_splits = 1;
-    p3.status = &hdr->status; p3.go = go;
-    p3.accumulate = (ci > 0 || o.accumulate_dweight) ? 1 : 0;
-    // and their zero rows of G are left out of the contraction over tokens (the kernel takes up to 32 flags)
-    p3.k_live = (rows <= 32ll * kTileM && (rows + BK - 1) / BK <= MAX_LIVE_KB) ? live_c : nullptr;
-    stage_mark(ST_B3, st);
-    if ((rc = launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, tmdW, p3, di.sm_count, st))) return rc;
+    ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, go, live_m, live_c,
+                (ci > 0 || o.accumulate_dweight) ? 1 : 0};
+    if ((rc = launch_chunk_outputs(co, tmWmn, tmdW, di.sm_count, st))) return rc;
   }
   return KDKL_OK;
 }
@@ -594,7 +612,7 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
     const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
     const uint8_t* live_c = live ? live + ci * L.tiles_per_chunk : nullptr;
     const __nv_bfloat16* hA = reinterpret_cast<const __nv_bfloat16*>(hidden) + s0 * H;
-    CUtensorMap tmA, tmGout, tmG, tmGmn, tmhmn, tmdH;
+    CUtensorMap tmA, tmGout;
     if ((rc = make_tmap_bf16(&tmA, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, BK, BM))) return rc;
     if ((rc = make_tmap_out_bf16(&tmGout, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad))) return rc;
 
@@ -634,48 +652,9 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
     KDKL_LAUNCHED("e_to_g_kernel");
 
     // dH[chunk] = G W and dW (+)= G^T h, exactly as in kdkl_backward
-    stage_mark(ST_B2, st);
-    if ((rc = make_tmap_bf16(&tmG, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, BK, BM))) return rc;
-    GemmParams p2;
-    memset(&p2, 0, sizeof(p2));
-    p2.M = (int)rows; p2.N = (int)H; p2.K = (int)V;
-    p2.m_tiles = (int)((rows + kTileM - 1) / kTileM); p2.n_tiles = (int)((H + BN - 1) / BN); p2.m_inner = 0;
-    p2.status = &hdr->status; p2.go = nullptr;
-    p2.m_live = live_m;
-    int sp = choose_k_splits((long long)p2.m_tiles * p2.n_tiles, (V + BK - 1) / BK);
-    if (sp > L.dh_splits) sp = L.dh_splits;
-    p2.k_splits = sp;
-    if (sp > 1) {
-      float* part = at<float>(ws, L.dh_part);
-      p2.split_rows = (int)L.Cpad;
-      if ((rc = make_tmap_out_f32(&tmdH, part, (uint64_t)H, (uint64_t)sp * L.Cpad, (uint64_t)H))) return rc;
-      if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
-      const long long n4 = rows * H / 4;
-      splitk_fixup_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(
-          part, (long long)L.Cpad * H, sp, n4,
-          o.dhidden_dtype == 0 ? reinterpret_cast<__nv_bfloat16*>(dhidden) + s0 * H : nullptr,
-          o.dhidden_dtype == 1 ? reinterpret_cast<float*>(dhidden) + s0 * H : nullptr, nullptr);
-      KDKL_LAUNCHED("splitk_fixup_kernel");
-    } else if (o.dhidden_dtype == 0) {
-      if ((rc = make_tmap_out_bf16(&tmdH, reinterpret_cast<__nv_bfloat16*>(dhidden) + s0 * H, (uint64_t)H,
-                                   (uint64_t)rows, (uint64_t)H))) return rc;
-      if ((rc = launch_gemm<EPI_STORE_BF16, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
-    } else {
-      if ((rc = make_tmap_out_f32(&tmdH, reinterpret_cast<float*>(dhidden) + s0 * H, (uint64_t)H, (uint64_t)rows,
-                                  (uint64_t)H))) return rc;
-      if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, di.sm_count, st))) return rc;
-    }
-    if ((rc = make_tmap_bf16(&tmGmn, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, 64, BK))) return rc;
-    if ((rc = make_tmap_bf16(&tmhmn, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, 64, BK))) return rc;
-    GemmParams p3;
-    memset(&p3, 0, sizeof(p3));
-    p3.M = (int)V; p3.N = (int)H; p3.K = (int)rows;
-    p3.m_tiles = (int)((V + kTileM - 1) / kTileM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0; p3.k_splits = 1;
-    p3.status = &hdr->status; p3.go = nullptr;
-    p3.accumulate = (ci > 0 || o.accumulate_dweight) ? 1 : 0;
-    p3.k_live = (rows <= 32ll * kTileM && (rows + BK - 1) / BK <= MAX_LIVE_KB) ? live_c : nullptr;
-    stage_mark(ST_B3, st);
-    if ((rc = launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, tmdW, p3, di.sm_count, st))) return rc;
+    ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, nullptr, live_m, live_c,
+                (ci > 0 || o.accumulate_dweight) ? 1 : 0};
+    if ((rc = launch_chunk_outputs(co, tmWmn, tmdW, di.sm_count, st))) return rc;
   }
   stage_mark(ST_REDUCE, st);
   loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, tau, H, V, K,
