@@ -259,6 +259,52 @@ static Tp* at(void* ws, size_t off) { return reinterpret_cast<Tp*>(reinterpret_c
 
 static int next_pow2(int x) { int p = 2; while (p < x) p <<= 1; return p; }
 
+// Header reset, teacher preparation and (with a mask) the live-row-tile flags: the common start of every forward.
+// Returns the flags (nullptr without a mask) through *live.
+static int launch_prep(const WsLayout& L, const kdkl_options& o, void* ws, const int32_t* topk_idx,
+                       const float* topk_val, const float* teacher_lse, const uint8_t* loss_mask, long long T,
+                       long long V, long long v0, long long V_total, int K, float inv_tau, const uint8_t** live,
+                       cudaStream_t st) {
+  WsHeader* hdr = at<WsHeader>(ws, L.hdr);
+  stage_mark(ST_PREP, st);
+  header_reset_kernel<<<1, 32, 0, st>>>(hdr);
+  KDKL_LAUNCHED("header_reset_kernel");
+  const int Kpad = next_pow2(K);
+  const size_t prep_smem = (size_t)PREP_WARPS * Kpad * (4 + 4 + 2);
+  prep_kernel<<<(unsigned)((T + PREP_WARPS - 1) / PREP_WARPS), PREP_WARPS * 32, prep_smem, st>>>(
+      topk_idx, topk_val, teacher_lse, loss_mask, T, (int)V, (int)v0, (int)V_total, K, Kpad, inv_tau, o.teacher_mode,
+      at<int>(ws, L.idx_sorted), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<int>(ws, L.nvalid),
+      at<float>(ws, L.M), at<float>(ws, L.Hent), hdr);
+  KDKL_LAUNCHED("prep_kernel");
+  // with a mask: which row tiles hold at least one counted token (the others are skipped by every GEMM,
+  // forward and backward; the flags stay in the workspace for kdkl_backward)
+  *live = nullptr;
+  if (loss_mask != nullptr) {
+    tile_live_kernel<<<(unsigned)((L.n_live + 7) / 8), 256, 0, st>>>(loss_mask, T, L.C, kTileM, (int)L.tiles_per_chunk,
+                                                                    L.n_live, at<uint8_t>(ws, L.live));
+    KDKL_LAUNCHED("tile_live_kernel");
+    *live = at<uint8_t>(ws, L.live);
+  }
+  return KDKL_OK;
+}
+
+// Parameters of the forward sweep of the chunk that starts at token s0 (EPI_LSE and its storing variants).
+static void fill_forward_params(GemmParams* p, const WsLayout& L, void* ws, long long s0, long long rows, long long H,
+                                long long V, int K, float inv_tau, const uint8_t* live_c) {
+  WsHeader* hdr = at<WsHeader>(ws, L.hdr);
+  memset(p, 0, sizeof(*p));
+  p->M = (int)rows; p->N = (int)V; p->K = (int)H;
+  p->m_tiles = (int)((rows + kTileM - 1) / kTileM); p->n_tiles = (int)L.n_tiles_v; p->m_inner = 1; p->k_splits = 1;
+  p->status = &hdr->status; p->go = nullptr;
+  p->scale_log2 = kLog2e * inv_tau; p->Ktop = K;
+  p->idx_sorted = at<int>(ws, L.idx_sorted) + s0 * K;
+  p->nvalid = at<int>(ws, L.nvalid) + s0;
+  p->part_m = at<float>(ws, L.part_m); p->part_s = at<float>(ws, L.part_s); p->part_stride = L.Cpad;
+  p->zg = at<float>(ws, L.zg) + s0 * K;
+  p->colread = at<int>(ws, L.colread) + s0 * K;
+  p->m_live = (live_c && p->m_tiles <= MAX_LIVE_M) ? live_c : nullptr;
+}
+
 // The two output GEMMs of one chunk, shared by kdkl_backward and kdkl_forward_backward: G holds the chunk's
 // dlogits (bf16 [rows, Vpad]).
 //   dH[chunk] = G W        (M = rows, N = H, K = V; split-K with a fixed-order fix-up when the tiles are few)
@@ -358,26 +404,9 @@ static int forward_impl(const void* hidden, const void* weight, const int32_t* t
   WsHeader* hdr = at<WsHeader>(ws, L.hdr);
   const float inv_tau = 1.0f / tau;
 
-  stage_mark(ST_PREP, st);
-  header_reset_kernel<<<1, 32, 0, st>>>(hdr);
-  KDKL_LAUNCHED("header_reset_kernel");
-
-  const int Kpad = next_pow2(K);
-  const size_t prep_smem = (size_t)PREP_WARPS * Kpad * (4 + 4 + 2);
-  prep_kernel<<<(unsigned)((T + PREP_WARPS - 1) / PREP_WARPS), PREP_WARPS * 32, prep_smem, st>>>(
-      topk_idx, topk_val, teacher_lse, loss_mask, T, (int)V, (int)v0, (int)V_total, K, Kpad, inv_tau, o.teacher_mode,
-      at<int>(ws, L.idx_sorted), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<int>(ws, L.nvalid),
-      at<float>(ws, L.M), at<float>(ws, L.Hent), hdr);
-  KDKL_LAUNCHED("prep_kernel");
-  // with a mask: which row tiles hold at least one counted token (the others are skipped by every GEMM,
-  // forward and backward; the flags stay in the workspace for kdkl_backward)
   const uint8_t* live = nullptr;
-  if (loss_mask != nullptr) {
-    tile_live_kernel<<<(unsigned)((L.n_live + 7) / 8), 256, 0, st>>>(loss_mask, T, L.C, kTileM, (int)L.tiles_per_chunk,
-                                                                    L.n_live, at<uint8_t>(ws, L.live));
-    KDKL_LAUNCHED("tile_live_kernel");
-    live = at<uint8_t>(ws, L.live);
-  }
+  if ((rc = launch_prep(L, o, ws, topk_idx, topk_val, teacher_lse, loss_mask, T, V, v0, V_total, K, inv_tau, &live, st)))
+    return rc;
 
   CUtensorMap tmW;
   if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, kBRows))) return rc;
@@ -389,17 +418,7 @@ static int forward_impl(const void* hidden, const void* weight, const int32_t* t
     const __nv_bfloat16* hA = reinterpret_cast<const __nv_bfloat16*>(hidden) + s0 * H;
     if ((rc = make_tmap_bf16(&tmA, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, BK, BM))) return rc;
     GemmParams p;
-    memset(&p, 0, sizeof(p));
-    p.M = (int)rows; p.N = (int)V; p.K = (int)H;
-    p.m_tiles = (int)((rows + kTileM - 1) / kTileM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1; p.k_splits = 1;
-    p.status = &hdr->status; p.go = nullptr;
-    p.scale_log2 = kLog2e * inv_tau; p.Ktop = K;
-    p.idx_sorted = at<int>(ws, L.idx_sorted) + s0 * K;
-    p.nvalid = at<int>(ws, L.nvalid) + s0;
-    p.part_m = at<float>(ws, L.part_m); p.part_s = at<float>(ws, L.part_s); p.part_stride = L.Cpad;
-    p.zg = at<float>(ws, L.zg) + s0 * K;
-    p.colread = at<int>(ws, L.colread) + s0 * K;
-    p.m_live = (live && p.m_tiles <= MAX_LIVE_M) ? live + fci * L.tiles_per_chunk : nullptr;
+    fill_forward_params(&p, L, ws, s0, rows, H, V, K, inv_tau, live ? live + fci * L.tiles_per_chunk : nullptr);
     stage_mark(ST_F1, st);
     if (o.stored_exponentials) {
       // one chunk covers all tokens: leave the exponentials in the G buffer for a backward without recompute
@@ -577,23 +596,9 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
   WsHeader* hdr = at<WsHeader>(ws, L.hdr);
   const float inv_tau = 1.0f / tau;
 
-  stage_mark(ST_PREP, st);
-  header_reset_kernel<<<1, 32, 0, st>>>(hdr);
-  KDKL_LAUNCHED("header_reset_kernel");
-  const int Kpad = next_pow2(K);
-  const size_t prep_smem = (size_t)PREP_WARPS * Kpad * (4 + 4 + 2);
-  prep_kernel<<<(unsigned)((T + PREP_WARPS - 1) / PREP_WARPS), PREP_WARPS * 32, prep_smem, st>>>(
-      topk_idx, topk_val, teacher_lse, loss_mask, T, (int)V, 0, (int)V, K, Kpad, inv_tau, o.teacher_mode,
-      at<int>(ws, L.idx_sorted), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<int>(ws, L.nvalid),
-      at<float>(ws, L.M), at<float>(ws, L.Hent), hdr);
-  KDKL_LAUNCHED("prep_kernel");
   const uint8_t* live = nullptr;
-  if (loss_mask != nullptr) {
-    tile_live_kernel<<<(unsigned)((L.n_live + 7) / 8), 256, 0, st>>>(loss_mask, T, L.C, kTileM, (int)L.tiles_per_chunk,
-                                                                    L.n_live, at<uint8_t>(ws, L.live));
-    KDKL_LAUNCHED("tile_live_kernel");
-    live = at<uint8_t>(ws, L.live);
-  }
+  if ((rc = launch_prep(L, o, ws, topk_idx, topk_val, teacher_lse, loss_mask, T, V, 0, V, K, inv_tau, &live, st)))
+    return rc;
   // the divisor of the mean and the per-token gradient coefficients are needed before the first chunk here
   count_tokens_kernel<<<1, 1024, 0, st>>>(loss_mask, T, o.denom_override, hdr);
   KDKL_LAUNCHED("count_tokens_kernel");
@@ -618,18 +623,8 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
 
     // F1': logits tile by tile -> online log-sum-exp partials, gathered teacher logits, and e = 2^(s - bias) into G
     GemmParams p;
-    memset(&p, 0, sizeof(p));
-    p.M = (int)rows; p.N = (int)V; p.K = (int)H;
-    p.m_tiles = (int)((rows + kTileM - 1) / kTileM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1; p.k_splits = 1;
-    p.status = &hdr->status; p.go = nullptr;
-    p.scale_log2 = kLog2e * inv_tau; p.Ktop = K;
-    p.idx_sorted = at<int>(ws, L.idx_sorted) + s0 * K;
-    p.nvalid = at<int>(ws, L.nvalid) + s0;
-    p.part_m = at<float>(ws, L.part_m); p.part_s = at<float>(ws, L.part_s); p.part_stride = L.Cpad;
-    p.zg = at<float>(ws, L.zg) + s0 * K;
-    p.colread = at<int>(ws, L.colread) + s0 * K;
-    const uint8_t* live_m = (live_c && p.m_tiles <= MAX_LIVE_M) ? live_c : nullptr;
-    p.m_live = live_m;
+    fill_forward_params(&p, L, ws, s0, rows, H, V, K, inv_tau, live_c);
+    const uint8_t* live_m = p.m_live;
     stage_mark(ST_F1, st);
     if ((rc = launch_gemm<EPI_LSE_E, false, false>(tmA, tmW, tmGout, p, di.sm_count, st))) return rc;
     stage_mark(ST_COMBINE, st);
