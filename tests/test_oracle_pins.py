@@ -269,3 +269,29 @@ def test_statistical_sanity_on_config_generators():
                     d["topk_idx"].numpy(), d["topk_val"].numpy(), tau=cfg.tau, want_grads=False)
     assert abs(o["logZ"].mean() - (math.log(cfg.V) + 0.5)) < 0.1
     assert 5.0 < o["loss"] < 9.0
+
+
+@pytest.mark.parametrize("seed", list(range(40)))
+def test_random_configurations_match_torch_autograd(seed):
+    """Seeded random shapes and options (temperature, masks, duplicates, partial mass, upstream gradient) against the
+    torch float64 library expression with autograd: any dropped term, wrong sign or transposed operand that only
+    shows for some combination of options fails here."""
+    r = np.random.default_rng(1000 + seed)
+    T, H, V = int(r.integers(1, 40)), int(r.integers(1, 30)), int(r.integers(2, 150))
+    K = int(r.integers(1, min(V, 12) + 1))
+    tau = float(r.choice([0.5, 1.0, 1.0, 2.5]))
+    h, W, idx, val = _rand_case(T, H, V, K, seed=seed, distinct=bool(r.random() < 0.6))
+    mask = (r.random(T) > 0.3).astype(np.uint8) if r.random() < 0.6 else None
+    if mask is not None and mask.sum() == 0:
+        mask[0] = 1
+    lse = None
+    if r.random() < 0.5:
+        l = val / tau
+        lse = np.log(np.exp(l - l.max(1, keepdims=True)).sum(1)) + l.max(1) + r.random(T) * 0.7      # mass < 1
+    gl = float(r.choice([1.0, -0.5, 2.0]))
+    o = kdkl_oracle(h, W, idx, val, tau=tau, mask=mask, teacher_lse=lse, grad_loss=gl)
+    loss, per_tok, dH, dW = _torch_ref(h, W, idx, val, tau, mask, lse=lse, grad_loss=gl)
+    assert abs(o["loss"] - loss) <= 1e-11 * max(1.0, abs(loss))
+    np.testing.assert_allclose(o["loss_tok"], per_tok, rtol=1e-9, atol=1e-11)
+    np.testing.assert_allclose(o["dH"], dH, rtol=1e-8, atol=1e-12)
+    np.testing.assert_allclose(o["dW"], dW, rtol=1e-8, atol=1e-12)
