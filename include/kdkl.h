@@ -71,6 +71,13 @@ typedef struct kdkl_options {
 size_t kdkl_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk,
                             const kdkl_options* opt);
 
+/* Debug aid for tests (no counterpart in the paper): the table of the workspace's slabs, in layout order, as byte
+ * offsets and used lengths; returns the number of slabs (fills at most `capacity` entries). With the environment
+ * variable KDKL_WS_GUARD_BYTES = n (read at every call) the layout leaves n untouched bytes after every slab, so a
+ * test can pre-fill the workspace, run, and check that nothing wrote past the end of a slab. */
+int kdkl_workspace_layout(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options* opt,
+                          int64_t* offsets, int64_t* lengths, int32_t capacity);
+
 /* Forward (Algorithm 1, "Forward"; Eq. "decomp"). One tensor-core sweep per chunk computes the
  * online max / sum-exp over the vocabulary and gathers z at the teacher's indices.
  *   hidden_bf16   [T, H]  bf16   student final hidden states

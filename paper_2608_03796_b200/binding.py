@@ -29,7 +29,7 @@ EXPORTS = [
     "kdkl_wait_selftest", "kdkl_teacher_topk", "kdkl_teacher_topk_workspace_bytes",
     "kdkl_feature_loss", "kdkl_feature_loss_workspace_bytes", "kdkl_step_host_record", "kdkl_record_staging_bytes",
     "kdkl_forward_backward", "kdkl_profile_single_pass", "kdkl_teacher_topk_stored",
-    "kdkl_teacher_topk_stored_workspace_bytes",
+    "kdkl_teacher_topk_stored_workspace_bytes", "kdkl_workspace_layout",
 ]
 
 FEATURE_MSE, FEATURE_COSINE = 0, 1
@@ -61,6 +61,9 @@ def lib() -> ctypes.CDLL:
     vp, i64, i32, f32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_float, ctypes.c_size_t
     L.kdkl_workspace_bytes.restype = sz
     L.kdkl_workspace_bytes.argtypes = [i64, i64, i64, i32, i64, vp]
+    L.kdkl_workspace_layout.restype = ctypes.c_int
+    L.kdkl_workspace_layout.argtypes = [i64, i64, i64, i32, i64, vp, ctypes.POINTER(ctypes.c_int64),
+                                        ctypes.POINTER(ctypes.c_int64), i32]
     L.kdkl_forward.restype = ctypes.c_int
     L.kdkl_forward.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, vp, sz, vp, vp, vp, vp, vp]
     L.kdkl_forward_shard.restype = ctypes.c_int
@@ -170,6 +173,14 @@ def _opt_ptr(opt: Optional[kdkl_options]):
 
 def kdkl_workspace_bytes(T, H, V, K, chunk=0, opt=None) -> int:
     return lib().kdkl_workspace_bytes(T, H, V, K, chunk, _opt_ptr(opt))
+
+
+def kdkl_workspace_layout(T, H, V, K, chunk=0, opt=None):
+    """[(offset, used length)] of every workspace slab, in layout order (debug aid; see include/kdkl.h)."""
+    off = (ctypes.c_int64 * 32)()
+    ln = (ctypes.c_int64 * 32)()
+    n = lib().kdkl_workspace_layout(T, H, V, K, chunk, _opt_ptr(opt), off, ln, 32)
+    return [(int(off[i]), int(ln[i])) for i in range(n)]
 
 
 def kdkl_forward(hidden, weight, topk_idx, topk_val, workspace, loss_out, *, teacher_lse=None, loss_mask=None,

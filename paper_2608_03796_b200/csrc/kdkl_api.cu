@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <vector>
@@ -182,8 +183,21 @@ struct WsLayout {
   int dh_splits;             // split-K factor of the dH GEMM at full chunks
   size_t hdr, idx_sorted, p_sorted, perm, zg, colread, nvalid, M, Hent, lz2, logZ, loss_tok, coefA, coefB;
   size_t part_m, part_s, G, dh_part, live, total;
+  static constexpr int kMaxSlabs = 24;
+  int n_slabs;
+  size_t slab_off[kMaxSlabs], slab_len[kMaxSlabs];   // every slab in layout order (for kdkl_workspace_layout)
   long long tiles_per_chunk, n_live;   // live-row-tile flags: one per kTileM rows of every chunk
 };
+
+// Debug aid: KDKL_WS_GUARD_BYTES=n in the environment puts n untouched bytes after every workspace slab (and makes
+// the workspace that much larger), so that a test can pre-fill the workspace, run, and see whether any kernel
+// wrote past the end of a slab (kdkl_workspace_layout gives the slab table). Unset or 0: the compact layout.
+static size_t ws_guard_bytes() {
+  const char* e = getenv("KDKL_WS_GUARD_BYTES");
+  if (e == nullptr) return 0;
+  const long long v = atoll(e);
+  return v > 0 && v <= (1ll << 20) ? up((size_t)v, 256) : 0;
+}
 
 static WsLayout ws_layout(long long T, long long H, long long V, int K, long long chunk) {
   WsLayout L;
@@ -193,7 +207,14 @@ static WsLayout ws_layout(long long T, long long H, long long V, int K, long lon
   L.Vpad = (long long)up((size_t)V, 64);
   L.n_tiles_v = (V + BN - 1) / BN;
   size_t o = 0;
-  auto take = [&](size_t bytes) { size_t at = o; o = up(o + bytes, 256); return at; };
+  const size_t guard = ws_guard_bytes();
+  L.n_slabs = 0;
+  auto take = [&](size_t bytes) {
+    size_t at = o;
+    if (L.n_slabs < WsLayout::kMaxSlabs) { L.slab_off[L.n_slabs] = at; L.slab_len[L.n_slabs] = bytes; ++L.n_slabs; }
+    o = up(o + bytes, 256) + guard;
+    return at;
+  };
   L.hdr = take(256);
   L.idx_sorted = take((size_t)T * K * 4);
   L.p_sorted = take((size_t)T * K * 4);
@@ -378,6 +399,15 @@ extern "C" {
 
 const char* kdkl_last_error(void) { return g_err; }
 int64_t kdkl_last_launch_count(void) { return g_launches; }
+
+int kdkl_workspace_layout(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options*,
+                          int64_t* offsets, int64_t* lengths, int32_t capacity) {
+  if (T < 1 || H < 1 || V < 1 || K < 1 || !offsets || !lengths) return 0;
+  const WsLayout L = ws_layout(T, H, V, K, chunk);
+  const int n = L.n_slabs < capacity ? L.n_slabs : capacity;
+  for (int i = 0; i < n; ++i) { offsets[i] = (int64_t)L.slab_off[i]; lengths[i] = (int64_t)L.slab_len[i]; }
+  return L.n_slabs;
+}
 
 size_t kdkl_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options*) {
   if (T < 1 || H < 1 || V < 1 || K < 1) return 0;
