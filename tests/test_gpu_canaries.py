@@ -84,3 +84,38 @@ def test_no_kernel_writes_outside_its_buffers(monkeypatch, T, H, V, K, chunk, ma
         assert nxt - (o + n) >= 4096
         assert bool((ws[o + n:nxt] == PATTERN).all()), f"write past the slab at offset {o} (+{n})"
     assert out.guards_intact()
+
+
+@pytest.mark.parametrize("T,H,kind", [(37, 72, 0), (257, 4096, 1), (19, 20000, 1), (130, 1032, 0)])
+def test_feature_loss_stays_inside_its_buffers(T, H, kind):
+    dev = torch.device("cuda:0")
+    g = torch.Generator().manual_seed(T + H)
+    s = torch.randn(T, H, generator=g).to(torch.bfloat16).to(dev)
+    r = torch.randn(T, H, generator=g).to(torch.bfloat16).to(dev)
+    mask = (torch.arange(T) % 3 != 0).to(torch.uint8).to(dev)
+    wsb = B.kdkl_feature_loss_workspace_bytes(T)
+    out = Carver(wsb + T * H * 2 + T * 4 + 16 * 1024, dev)
+    ws = out.take((wsb,), torch.uint8)
+    d = out.take((T, H), torch.bfloat16)
+    tok = out.take((T,), torch.float32)
+    loss = out.take((1,), torch.float32)
+    B.kdkl_feature_loss(s, r, ws, loss, kind=kind, loss_mask=mask, loss_per_token=tok, dstudent=d)
+    torch.cuda.synchronize()
+    assert torch.isfinite(loss).all() and out.guards_intact()
+
+
+@pytest.mark.parametrize("stored", [False, True])
+def test_teacher_topk_stays_inside_its_buffers(stored):
+    dev = torch.device("cuda:0")
+    T, H, V, K = 300, 264, 4120, 16
+    g = torch.Generator().manual_seed(3)
+    h = torch.randn(T, H, generator=g).to(torch.bfloat16).to(dev)
+    W = (torch.randn(V, H, generator=g) / H ** 0.5).to(torch.bfloat16).to(dev)
+    size_fn = B.lib().kdkl_teacher_topk_stored_workspace_bytes if stored else B.lib().kdkl_teacher_topk_workspace_bytes
+    wsb = size_fn(T, H, V, K)
+    out = Carver(wsb + 64 * 1024, dev)
+    ws = out.take((wsb,), torch.uint8)
+    idx, val, lse, _ = B.kdkl_teacher_topk(h, W, K, workspace=ws, stored=stored)
+    torch.cuda.synchronize()
+    assert B.kdkl_status(ws)[0] == 0 and int(idx.min()) >= 0 and int(idx.max()) < V
+    assert out.guards_intact()
