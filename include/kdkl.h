@@ -125,7 +125,8 @@ int kdkl_backward(const void* hidden_bf16, const void* weight_bf16, const uint8_
  * the stored exponential: the gradients are then not finite and kdkl_status reports KDKL_ERR_NONFINITE with the
  * row (use the two-call path for such inputs). 6 T H V flops instead of 8 T H V.
  * Arguments as the two calls; grad_loss must be known here. The workspace afterwards holds the same saved
- * state (kdkl_saved_state, kdkl_status). Not available for vocabulary shards (log Z needs the exchange first). */
+ * state (kdkl_saved_state, kdkl_status). Vocabulary shards need the cross-shard exchange before log Z is known:
+ * there the same saving is available through option stored_exponentials when one chunk covers all tokens. */
 int kdkl_forward_backward(const void* hidden_bf16, const void* weight_bf16, const int32_t* topk_idx,
                           const float* topk_val, const float* teacher_lse, const uint8_t* loss_mask, int64_t T,
                           int64_t H, int64_t V, int32_t K, int64_t chunk, float temperature, const kdkl_options* opt,
