@@ -83,3 +83,21 @@ def test_profile_stages_accounts_for_every_launch_and_changes_nothing():
     assert st["prep"][1] == 1 and st["loss_reduce"][1] == 1 and st["bwd_coef"][1] == 1
     assert all(ms > 0 for ms, n in st.values())
     assert torch.equal(op.loss, ref_loss) and torch.equal(op.dweight, ref_dw)
+
+
+def test_profile_single_pass_accounts_for_every_stage_and_changes_nothing():
+    cfg = I.CONFIGS["c1"]
+    d = I.make_inputs(cfg)
+    dev = torch.device("cuda:0")
+    g = {k: (v.to(dev) if v is not None else None) for k, v in d.items()}
+    op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev)
+    op.forward_backward(g["hidden"], g["weight"], g["topk_idx"], g["topk_val"])
+    ref = (op.loss.clone(), op.dhidden.clone(), op.dweight.clone())
+    st = B.kdkl_profile_single_pass(g["hidden"], g["weight"], g["topk_idx"], g["topk_val"], op.workspace, op.loss,
+                                    op.dhidden, op.dweight, chunk=cfg.chunk, temperature=cfg.tau)
+    chunks = cfg.T // cfg.chunk
+    assert st["fwd_gemm_lse_exp"][1] == chunks and st["exp_to_dlogits"][1] == chunks and st["combine"][1] == chunks
+    assert st["dhidden_gemm"][1] == chunks and st["dweight_gemm"][1] == chunks
+    assert st["prep"][1] == 1 and st["loss_reduce"][1] == 1 and "bwd_coef" not in st
+    assert all(ms > 0 for ms, n in st.values())
+    assert torch.equal(op.loss, ref[0]) and torch.equal(op.dhidden, ref[1]) and torch.equal(op.dweight, ref[2])
