@@ -1,0 +1,87 @@
+"""Gradient comparison beyond one global norm (a helper for the GPU parity tests; not a test itself).
+
+The CUDA path's only rounding of consequence is G (the chunk's dlogits), rounded once to bf16 before the two
+output contractions; everything else is fp32 accumulation of exact bf16 products. bf16 keeps 8 significand
+bits, so a rounding moves a value by at most u = 2^-8 of itself. For an output element
+
+    out[r, c] = sum_j G[j] * x[j]        (dH: j = vocabulary, x = W[:, c];  dW: j = token, x = h[:, c])
+
+the error is sum_j delta_j G[j] x[j] with |delta_j| <= u and no preferred sign. Two regimes:
+  * one term dominates (a support entry with a large teacher probability): |error| <= u |out|;
+  * many comparable terms: the error is a sum of independent zero-mean terms, standard deviation at most
+    u / sqrt(3) times the root-mean-square of the row (x is N(0, s^2) along c, so the row's rms is
+    s * |G|_2 and the error's deviation is (u / sqrt 3) * s * |G|_2).
+Hence, element by element,
+
+    |cuda - oracle| <= u_out |oracle| + u |oracle| + C_SIGMA * n^(1/2) * (u / sqrt 3) * rms(oracle row)
+
+with u_out = 2^-8 when the output itself is stored in bf16 (dH by default) and 0 for fp32 outputs, n the number
+of bf16 roundings inside G (1; 2 for the single-pass step, whose stored exponential is rounded as well), and
+C_SIGMA = 8 standard deviations (5e8 elements of a full-size dW never reach it by chance). Row by row, the
+relative Frobenius error must stay below the tolerance stated for the whole matrix (1e-2): about three times
+what the model predicts (u / sqrt 3 = 2.3e-3, plus the output rounding), so a row whose sparse teacher term
+or tail columns went missing fails although it vanishes inside the whole-matrix norm.
+"""
+import numpy as np
+
+U_BF16 = 2.0 ** -8
+C_SIGMA = 8.0
+ROW_FRO = 1e-2
+
+
+def elementwise_tolerance(ref_block, out_bf16=False, roundings=1):
+    """The bound above for a block of whole rows of the oracle's matrix (float64 [rows, cols])."""
+    rms = np.sqrt(np.mean(ref_block * ref_block, axis=1, keepdims=True))
+    rel = U_BF16 * (2.0 if out_bf16 else 1.0)
+    return rel * np.abs(ref_block) + C_SIGMA * np.sqrt(float(roundings)) * (U_BF16 / np.sqrt(3.0)) * rms
+
+
+def check_grad_matrix(got, ref, name, out_bf16=False, roundings=1, row_fro=ROW_FRO, block=4096, extra_tol=None):
+    """got, ref: [rows, cols] (anything np.asarray takes; compared in float64, row block by row block so that a
+    full-size dW does not need several float64 copies). extra_tol (scalar or [rows, cols]) is added to every
+    element's bound: the fp32 rounding of `dW +=` onto existing contents. Raises AssertionError naming the worst
+    row / element.
+    Returns (largest per-row relative error, largest elementwise error / tolerance)."""
+    rows = ref.shape[0]
+    assert got.shape == ref.shape, (name, got.shape, ref.shape)
+    norms = np.empty(rows)
+    errs = np.empty(rows)
+    worst_ratio, worst_at = 0.0, None
+    for r0 in range(0, rows, block):
+        b = np.asarray(ref[r0:r0 + block], dtype=np.float64)
+        a = np.asarray(got[r0:r0 + block], dtype=np.float64)
+        assert np.isfinite(a).all(), f"{name}: non-finite values in rows {r0}..{r0 + len(a) - 1}"
+        diff = np.abs(a - b)
+        norms[r0:r0 + len(b)] = np.sqrt((b * b).sum(axis=1))
+        errs[r0:r0 + len(b)] = np.sqrt((diff * diff).sum(axis=1))
+        tol = elementwise_tolerance(b, out_bf16, roundings)
+        if extra_tol is not None:
+            tol = tol + (extra_tol if np.ndim(extra_tol) == 0 else np.asarray(extra_tol)[r0:r0 + block])
+        # rows the oracle holds as exact zeros (ignored tokens) must be exact zeros
+        ratio = np.where(tol > 0, diff / np.where(tol > 0, tol, 1.0), np.where(diff > 0, np.inf, 0.0))
+        k = int(np.argmax(ratio))
+        if ratio.flat[k] > worst_ratio:
+            worst_ratio = float(ratio.flat[k])
+            rr, cc = np.unravel_index(k, ratio.shape)
+            worst_at = (r0 + int(rr), int(cc), float(a[rr, cc]), float(b[rr, cc]), float(tol[rr, cc]))
+    assert worst_ratio <= 1.0, (f"{name}: element (row, col, got, oracle, tolerance) = {worst_at} is "
+                                f"{worst_ratio:.2f} x its tolerance")
+    # per-row relative Frobenius error, on every row whose norm is not negligible next to the largest
+    live = norms > 1e-6 * norms.max() if rows and norms.max() > 0 else np.zeros(rows, bool)
+    rel = np.where(live, errs / np.where(live, norms, 1.0), 0.0)
+    r = int(np.argmax(rel)) if rows else 0
+    assert not rows or rel[r] <= row_fro, f"{name}: row {r} relative error {rel[r]:.3e} > {row_fro:.0e}"
+    return (float(rel[r]) if rows else 0.0), worst_ratio
+
+
+def check_support_rows(got_dw, ref_dw, topk_idx, tokens, name, roundings=1):
+    """The rows of dW at the teacher indices of the given tokens: the place where the sparse -p term of
+    Eq. "grad" lands. Compared like any other rows, but named, so that a missing support correction is
+    reported as such."""
+    V = ref_dw.shape[0]
+    rows = sorted({int(v) for t in tokens for v in np.asarray(topk_idx[t]).tolist() if 0 <= v < V})
+    if not rows:
+        return
+    sel = np.asarray(rows)
+    check_grad_matrix(np.asarray(got_dw)[sel], np.asarray(ref_dw)[sel], f"{name} (support rows)", False, roundings,
+                      block=len(sel))

@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+from gradcheck import check_grad_matrix, check_support_rows
 from oracle.kdkl_oracle import kdkl_oracle
 from paper_2608_03796_b200 import binding as B
 from paper_2608_03796_b200 import inputs as I
@@ -74,6 +75,7 @@ def test_fullsize_sampled_parity(name, n_rows, partial_mass):
     dH = full.dhidden[Rd].float().cpu().double().numpy()
     assert _fro(dH, o["dH"]) <= GRAD_FRO
     assert not dH[~counted].any()
+    check_grad_matrix(dH, o["dH"], "dH (sampled rows of the full run)", out_bf16=True)
 
     # ---- whole-run properties
     tok = full.loss_per_token.double()
@@ -105,6 +107,10 @@ def test_fullsize_sampled_parity(name, n_rows, partial_mass):
     assert abs(sub.loss.item() - oR["loss"]) <= LOSS_RTOL * abs(oR["loss"])
     dW_sub = sub.dweight.cpu().double().numpy()
     assert _fro(dW_sub, oR["dW"]) <= GRAD_FRO
+    # every vocabulary row and every element of the sampled tokens' dW, and by name the rows at the teacher
+    # indices of a few sampled tokens, where the sparse -p term of Eq. "grad" lives
+    check_grad_matrix(dW_sub, oR["dW"], "dW (tokens of the sample)")
+    check_support_rows(dW_sub, oR["dW"], idxR, list(np.flatnonzero(counted)[:4]), "dW (tokens of the sample)")
     del oR, dW_sub
 
     # ---- additivity over a disjoint split of the mask: N dW = |R| dW_R + (N - |R|) dW_rest

@@ -7,6 +7,7 @@ import numpy as np
 import pytest
 import torch
 
+from gradcheck import check_grad_matrix, check_support_rows
 from oracle.kdkl_oracle import kdkl_oracle
 from paper_2608_03796_b200 import binding as B
 
@@ -119,5 +120,11 @@ def test_random_configuration_matches_oracle(seed, single_pass):
     assert not dH[~counted].any()
     if counted.any():
         assert _fro(dH, o["dH"]) <= GRAD_FRO and _fro(dW, want_dW) <= GRAD_FRO
+        # every row and every element (the single-pass step rounds its stored exponential as well: two roundings)
+        nr = 2 if single_pass else 1
+        b64 = base.double().numpy() if c["accumulate"] else 0.0
+        check_grad_matrix(dH, o["dH"], "dH", out_bf16=not c["dh32"], roundings=nr)
+        check_grad_matrix(dW - b64, o["dW"], "dW", roundings=nr, extra_tol=2.0 ** -22 * np.abs(b64))
+        check_support_rows(dW - b64, o["dW"], idx, list(np.flatnonzero(counted)[:3]), "dW", roundings=nr)
     else:
         assert not dH.any() and np.array_equal(dW, want_dW)

@@ -8,6 +8,7 @@ import numpy as np
 import pytest
 import torch
 
+from gradcheck import check_grad_matrix, check_support_rows
 from oracle.kdkl_oracle import kdkl_oracle
 from paper_2608_03796_b200 import binding as B
 from paper_2608_03796_b200 import inputs as I
@@ -84,6 +85,12 @@ def test_single_pass_matches_oracle_and_two_call_path(T, H, V, K, chunk, tau, ma
     assert _fro(dH, o["dH"]) <= 1e-2 and _fro(dW, want_dW) <= 1e-2
     if mask is not None:
         assert not dH[mask_np == 0].any()
+    # row by row and element by element; G carries two bf16 roundings here (the stored exponential, then G)
+    b64 = base.double().numpy() if opts.get("accumulate") else 0.0
+    check_grad_matrix(dH, o["dH"], "dH", out_bf16=one.dhidden.dtype == torch.bfloat16, roundings=2)
+    check_grad_matrix(dW - b64, o["dW"], "dW", roundings=2, extra_tol=2.0 ** -22 * np.abs(b64))
+    cnt = np.ones(T, bool) if mask is None else mask_np != 0
+    check_support_rows(dW - b64, o["dW"], idx.numpy(), list(np.flatnonzero(cnt)[:3]), "dW", roundings=2)
     # and close to the two-call gradients (two independent roundings of G against one)
     assert _fro(dH, two.dhidden.float().cpu().double().numpy()) <= 6e-3
     assert _fro(dW, two.dweight.cpu().double().numpy()) <= 6e-3
@@ -112,6 +119,8 @@ def test_single_pass_fullsize_sampled():
     o = kdkl_oracle(d["hidden"][R].cpu().double().numpy(), d["weight"].cpu().double().numpy(),
                     d["topk_idx"][R].cpu().numpy(), d["topk_val"][R].cpu().numpy(), tau=cfg.tau, denom=cfg.T)
     assert _fro(one.dhidden[R].float().cpu().double().numpy(), o["dH"]) <= 1e-2
+    check_grad_matrix(one.dhidden[R].float().cpu().double().numpy(), o["dH"], "dH (sampled rows)", out_bf16=True,
+                      roundings=2)
     colsum = one.dweight.double().sum(0).abs()
     colabs = one.dweight.double().abs().sum(0)
     assert (colsum / colabs).max().item() < 3e-3
@@ -174,6 +183,9 @@ def test_single_pass_packed_config_sampled_rows_and_dweight():
         oR = kdkl_oracle(hR, W64, idxR, valR, tau=cfg.tau, mask=mR, denom=nR)
     assert abs(op.loss.item() - oR["loss"]) <= 1e-3 * abs(oR["loss"])
     assert _fro(op.dweight.cpu().double().numpy(), oR["dW"]) <= 1e-2
+    check_grad_matrix(op.dweight.cpu().numpy(), oR["dW"], "dW (tokens of the sample)", roundings=2)
+    check_support_rows(op.dweight.cpu().numpy(), oR["dW"], idxR, list(np.flatnonzero(mR != 0)[:4]),
+                       "dW (tokens of the sample)", roundings=2)
 
 
 def test_two_calls_with_stored_exponentials_one_chunk():
@@ -195,6 +207,8 @@ def test_two_calls_with_stored_exponentials_one_chunk():
     assert abs(op.loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
     assert _fro(op.dhidden.float().cpu().double().numpy(), o["dH"]) <= 1e-2
     assert _fro(op.dweight.cpu().double().numpy(), o["dW"]) <= 1e-2
+    check_grad_matrix(op.dhidden.float().cpu().numpy(), o["dH"], "dH", out_bf16=True, roundings=2)
+    check_grad_matrix(op.dweight.cpu().numpy(), o["dW"], "dW", roundings=2)
     # more than one chunk is refused on the host
     with pytest.raises(B.KdklError) as e:
         B.FusedChunkedKL(T, H, V, K, chunk=256, temperature=tau, opt=opt, device=dev).forward(

@@ -1,0 +1,74 @@
+"""The gradient comparison helper must (a) accept what the CUDA path's arithmetic produces - fp32 contractions of a
+G that was rounded once to bf16 - and (b) reject a defect confined to one row although the whole-matrix norm
+does not see it. Checked here on synthetic matrices with the structure of Eq. "grad" (a dense softmax part plus
+K large sparse teacher entries per token), on the CPU."""
+import numpy as np
+import pytest
+import torch
+
+from gradcheck import check_grad_matrix, check_support_rows
+
+
+def _dlogits(T, V, K, seed):
+    g = torch.Generator().manual_seed(seed)
+    q = torch.softmax(torch.randn(T, V, generator=g, dtype=torch.float64), dim=-1)
+    idx = torch.stack([torch.randperm(V, generator=g)[:K] for _ in range(T)])
+    p = torch.softmax(torch.randn(T, K, generator=g, dtype=torch.float64) * 3 ** 0.5, dim=-1)
+    sparse = torch.zeros(T, V, dtype=torch.float64).scatter_add_(1, idx, p)
+    return q / T, sparse / T, idx
+
+
+def _bf16(x):
+    return x.to(torch.float32).to(torch.bfloat16).to(torch.float64)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_accepts_one_bf16_rounding_and_rejects_a_row_without_its_teacher_term(seed):
+    T, V, H, K = 1300, 2000, 64, 8
+    dense, sparse, idx = _dlogits(T, V, K, seed)
+    g = torch.Generator().manual_seed(100 + seed)
+    h = _bf16(torch.randn(T, H, generator=g))
+    W = _bf16(torch.randn(V, H, generator=g) / H ** 0.5)
+    G = dense - sparse
+    ref_dW, ref_dH = (G.T @ h).numpy(), (G @ W).numpy()
+    Gr = _bf16(G)
+    got_dW, got_dH = (Gr.T @ h).numpy(), _bf16(Gr @ W).numpy()
+    rel_w, ratio_w = check_grad_matrix(got_dW, ref_dW, "dW")
+    rel_h, ratio_h = check_grad_matrix(got_dH, ref_dH, "dH", out_bf16=True)
+    assert rel_w < 5e-3 and rel_h < 6e-3 and ratio_w < 0.8 and ratio_h < 0.8     # with room to spare
+    check_support_rows(got_dW, ref_dW, idx.numpy(), [0, 7, T - 1], "dW")
+
+    # the defect: token 7 loses its sparse teacher term (a missed support correction in one row of 1300)
+    bad = G.clone()
+    bad[7] = dense[7]
+    bad_r = _bf16(bad)
+    bad_dW, bad_dH = (bad_r.T @ h).numpy(), _bf16(bad_r @ W).numpy()
+    fro = lambda a, b: np.linalg.norm(a - b) / np.linalg.norm(b)
+    assert fro(bad_dW, ref_dW) > fro(got_dW, ref_dW)
+    with pytest.raises(AssertionError):
+        check_grad_matrix(bad_dH, ref_dH, "dH", out_bf16=True)
+    with pytest.raises(AssertionError):
+        check_support_rows(bad_dW, ref_dW, idx.numpy(), [7], "dW")
+    with pytest.raises(AssertionError):
+        check_grad_matrix(bad_dW, ref_dW, "dW")
+
+
+def test_a_defect_hidden_from_the_global_norm_is_caught():
+    """One wrong run of 64 elements in a 20000 x 256 dW: 1e-2 relative Frobenius over the whole matrix stays
+    green, the per-row and per-element bounds do not."""
+    g = torch.Generator().manual_seed(5)
+    ref = torch.randn(20000, 256, generator=g, dtype=torch.float64).numpy()
+    got = ref * (1 + 1e-3)
+    got[12345, 64:128] = 0.0
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) < 1e-2
+    with pytest.raises(AssertionError):
+        check_grad_matrix(got, ref, "dW")
+
+
+def test_zero_rows_must_be_exact_zeros():
+    ref = np.zeros((4, 8)); ref[1] = 1.0
+    got = ref.copy()
+    check_grad_matrix(got, ref, "dH", out_bf16=True)
+    got[2, 3] = 1e-9
+    with pytest.raises(AssertionError):
+        check_grad_matrix(got, ref, "dH", out_bf16=True)

@@ -3,11 +3,13 @@
 kdkl_logz_noalloc is for callers that cannot allocate device memory at all (for instance a plugin
 inside a server whose pool already owns the GPU): its scratch is a fixed array inside the library.
 It must give the same log Z as kdkl_forward, which uses a caller-allocated workspace, on two calls
-in a row that share that array.
+in a row that share that array - and both must agree with the fp64 oracle's log Z.
 """
+import numpy as np
 import pytest
 import torch
 
+from oracle.kdkl_oracle import kdkl_oracle
 from paper_2608_03796_b200 import binding as B
 
 pytestmark = pytest.mark.gpu
@@ -38,6 +40,9 @@ def test_logz_noalloc_matches_forward_twice_in_a_row():
         assert torch.cuda.memory_allocated() == before
         assert torch.isfinite(out).all()
         assert (out - ref).abs().max().item() <= 2e-4
+        o = kdkl_oracle(h.cpu().double().numpy(), W.cpu().double().numpy(), idx.cpu().numpy(), val.cpu().numpy(),
+                        tau=tau, want_grads=False)
+        np.testing.assert_allclose(out.cpu().double().numpy(), o["logZ"], rtol=0, atol=2e-4)
 
 
 def test_logz_noalloc_rejects_oversized_vocabulary():
