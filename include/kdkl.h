@@ -14,8 +14,11 @@
  *
  * Conventions for every entry point unless stated otherwise
  *   - all data pointers are DEVICE pointers owned by the caller; the library allocates no
- *     device memory, keeps no global state, and only enqueues work on the given stream
- *     (no host synchronisation);
+ *     device memory and only enqueues work on the given stream (no host synchronisation).
+ *     Between calls it keeps nothing of a call's data: its only state is, per thread, the text of
+ *     the last error and the last launch count, and, per process, what it has learnt about each
+ *     device (SM count, compute capability, kernel attributes already set) plus the test hook
+ *     kdkl_debug_guard_bytes;
  *   - matrices are row-major and contiguous; hidden, weight and the workspace must be
  *     16-byte aligned; H must be a multiple of 8;
  *   - return value: KDKL_OK or a negative KDKL_ERR_* detected on the host before anything
@@ -42,9 +45,13 @@ extern "C" {
 #define KDKL_ERR_CUDA (-7)      /* a CUDA call failed; kdkl_last_error() has the text */
 /* device-detected, reported by kdkl_status(): */
 #define KDKL_ERR_TIMEOUT (-8)   /* a bounded wait inside a kernel expired */
-#define KDKL_ERR_STATE (-9)     /* backward called on a workspace forward did not fill for this shape */
+#define KDKL_ERR_STATE (-9)     /* backward called on a workspace forward did not fill for this shape, chunk size and
+                                   temperature (or, with stored_exponentials, whose exponentials are gone) */
 #define KDKL_ERR_INDEX (-10)    /* a teacher index >= V was seen (the entry was ignored) */
 #define KDKL_ERR_NONFINITE (-11)/* a counted token's loss is not finite */
+#define KDKL_ERR_RANGE (-13)    /* stored exponentials only (kdkl_forward_backward, option stored_exponentials): a
+                                   counted token's scaled logits all lie below the range the bf16 exponentials
+                                   keep (log2 of its normaliser < -40); use kdkl_forward + kdkl_backward there */
 
 #define KDKL_MAX_K 1024
 
@@ -62,8 +69,20 @@ typedef struct kdkl_options {
                                  buffer and kdkl_backward forms G from them instead of projecting again (three
                                  projections for the two calls, as in kdkl_forward_backward; the vocabulary-sharded
                                  calls included, where log Z is only known after the exchange). Otherwise
-                                 KDKL_ERR_ARG. A struct of the previous size (without this field) is accepted */
+                                 KDKL_ERR_ARG. The conversion is in place, so kdkl_backward can run ONCE per
+                                 forward call in this mode: a second one reports KDKL_ERR_STATE and writes nothing.
+                                 A struct of the previous size (without this field) is accepted */
+  const double* denom_device; /* NULL, or a DEVICE pointer to one double read when the kernels run: the divisor of
+                                 the mean (takes precedence over denom_override). For data-parallel callers that
+                                 sum kdkl_count_tokens over their ranks on the device: no host read of the count.
+                                 A struct of a previous size (without this field) is accepted */
 } kdkl_options;
+
+/* Number of counted tokens of a batch (mask = 1; T when loss_mask is NULL), written as one double to
+ * count_out (DEVICE). One small kernel on the stream. The divisor of the mean for a caller whose tokens
+ * are spread over several ranks is the sum of these counts (text under Eq. "kl": the mean runs over all
+ * loss-masked positions); pass that sum back through kdkl_options.denom_device. */
+int kdkl_count_tokens(const uint8_t* loss_mask, int64_t T, double* count_out, void* cuda_stream);
 
 /* Bytes of device workspace forward and backward need for this shape (chunk 0 = default 4096).
  * The same workspace must be passed to forward and then to backward: it carries the saved
@@ -71,12 +90,14 @@ typedef struct kdkl_options {
 size_t kdkl_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk,
                             const kdkl_options* opt);
 
-/* Debug aid for tests (no counterpart in the paper): the table of the workspace's slabs, in layout order, as byte
- * offsets and used lengths; returns the number of slabs (fills at most `capacity` entries). With the environment
- * variable KDKL_WS_GUARD_BYTES = n (read at every call) the layout leaves n untouched bytes after every slab, so a
- * test can pre-fill the workspace, run, and check that nothing wrote past the end of a slab. */
+/* Debug aids for tests (no counterpart in the paper). kdkl_workspace_layout: the table of the workspace's slabs, in
+ * layout order, as byte offsets and used lengths; returns the number of slabs (fills at most `capacity` entries).
+ * kdkl_debug_guard_bytes(n): from now on (process-wide, until changed; n = 0 restores the compact layout, n is
+ * rounded up to 256 and capped at 1 MiB) every layout leaves n untouched bytes after every slab, so a test can
+ * pre-fill the workspace, run, and check that nothing wrote past the end of a slab; returns the previous value. */
 int kdkl_workspace_layout(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options* opt,
                           int64_t* offsets, int64_t* lengths, int32_t capacity);
+int64_t kdkl_debug_guard_bytes(int64_t n);
 
 /* Forward (Algorithm 1, "Forward"; Eq. "decomp"). One tensor-core sweep per chunk computes the
  * online max / sum-exp over the vocabulary and gathers z at the teacher's indices.

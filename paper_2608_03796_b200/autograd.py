@@ -7,9 +7,13 @@
 Marshalling only: forward runs kdkl_forward, backward runs kdkl_backward with the upstream gradient
 as `grad_loss`; nothing of the loss arithmetic happens in torch ops. The upstream gradient of a scalar
 loss is read to the host once (`grad.item()`), since the C entry point takes it as a plain float.
-Workspace and gradient buffers are cached per shape on the function object, so repeated steps allocate
-nothing. `weight_grad_fp32=True` hands back the fp32 dW buffer itself (Megatron-style main_grad use)
-instead of a bf16 copy; with `dweight_out` given, dW is accumulated into that fp32 tensor in place.
+Workspace and gradient buffers are pooled per shape, so repeated steps allocate nothing. A forward call takes a
+buffer set out of the pool and owns it until its backward has run: two losses of one shape that are both alive
+(loss1 + loss2, pipelined micro-batches, activation checkpointing) therefore never share the saved state of
+Algorithm 1, and a backward whose buffer set has been reused in the meantime (a second backward through a freed
+graph) raises instead of returning gradients of another batch. `weight_grad_fp32=True` hands the fp32 dW
+buffer over to the caller (the pool allocates a new one next time) instead of a bf16 copy; with `dweight_out`
+given, dW is accumulated into that fp32 tensor in place.
 """
 from __future__ import annotations
 
@@ -19,22 +23,32 @@ import torch
 
 from . import binding as B
 
-_cache: dict = {}
+_free: dict = {}          # key -> buffer sets (FusedChunkedKL holders) no live loss is using
 
 
 def clear_cache() -> None:
-    """Drops the cached workspaces and gradient buffers (one set per shape seen so far)."""
-    _cache.clear()
+    """Drops the pooled workspaces and gradient buffers (sets in use by a live loss are unaffected)."""
+    _free.clear()
 
 
-def _holder(T, H, V, K, chunk, tau, accumulate, device) -> B.FusedChunkedKL:
+def _acquire(T, H, V, K, chunk, tau, accumulate, device):
+    """A buffer set for this shape that nothing else is using: out of the pool, or a new one."""
     key = (T, H, V, K, chunk, tau, accumulate, str(device))
-    op = _cache.get(key)
-    if op is None:
+    pool = _free.setdefault(key, [])
+    if pool:
+        op = pool.pop()
+        if op.dweight is None:                                    # handed over to a caller last time
+            op.dweight = torch.empty(V, H, dtype=torch.float32, device=device)
+    else:
         op = B.FusedChunkedKL(T, H, V, K, chunk=chunk, temperature=tau,
                               opt=B.make_options(accumulate_dweight=accumulate), device=device)
-        _cache[key] = op
-    return op
+        op.generation = 0
+    op.generation += 1
+    return key, op
+
+
+def _release(key, op) -> None:
+    _free.setdefault(key, []).append(op)
 
 
 class _FusedChunkedKL(torch.autograd.Function):
@@ -46,22 +60,30 @@ class _FusedChunkedKL(torch.autograd.Function):
         # single pass: the gradients for an upstream gradient of 1 come out of the forward call (three projections
         # instead of four); it writes dW itself, so it is not combined with accumulation into a caller's buffer
         ctx.done = bool(single_pass) and dweight_out is None
-        op = _holder(T, H, V, K, int(chunk), float(temperature), 1 if dweight_out is not None else 0, hidden.device)
+        key, op = _acquire(T, H, V, K, int(chunk), float(temperature), 1 if dweight_out is not None else 0,
+                           hidden.device)
         ctx.expected = float(expected_grad)
         if ctx.done:
             op.forward_backward(hidden, weight, topk_idx, topk_val, teacher_lse=teacher_lse, loss_mask=loss_mask,
                                 grad_loss=ctx.expected)
         else:
             op.forward(hidden, weight, topk_idx, topk_val, teacher_lse=teacher_lse, loss_mask=loss_mask)
-        ctx.op, ctx.mask = op, loss_mask
+        loss = op.loss.clone().squeeze(0)
+        if not (ctx.needs_input_grad[0] or ctx.needs_input_grad[1]):
+            _release(key, op)                                     # no backward will come: the set is free again
+            return loss
+        ctx.op, ctx.key, ctx.generation, ctx.mask = op, key, op.generation, loss_mask
         ctx.dweight_out, ctx.weight_grad_fp32 = dweight_out, weight_grad_fp32
         ctx.save_for_backward(hidden, weight)
-        return op.loss.clone().squeeze(0)
+        return loss
 
     @staticmethod
     def backward(ctx, grad):
         hidden, weight = ctx.saved_tensors
         op = ctx.op
+        if op.generation != ctx.generation:
+            raise RuntimeError("fused_chunked_kl: this loss's saved state has been reused by a later forward call "
+                               "(backward ran twice without retain_graph semantics the buffers can honour)")
         gl = float(grad.item())
         if not (ctx.done and gl == ctx.expected):                 # any other upstream gradient: the recompute path
             if ctx.dweight_out is not None:
@@ -77,10 +99,12 @@ class _FusedChunkedKL(torch.autograd.Function):
         if ctx.dweight_out is not None:
             dW = None
         elif ctx.weight_grad_fp32:
-            dW = op.dweight
+            dW, op.dweight = op.dweight, None                     # ownership passes to the caller
         else:
             dW = op.dweight.to(weight.dtype)
-        return op.dhidden.clone(), dW, None, None, None, None, None, None, None, None, None, None
+        dH = op.dhidden.clone()
+        _release(ctx.key, op)          # free for the next forward; a second backward of this graph before that
+        return dH, dW, None, None, None, None, None, None, None, None, None, None   # still finds its state intact
 
 
 def fused_chunked_kl(hidden, weight, topk_idx, topk_val, teacher_lse: Optional[torch.Tensor] = None,

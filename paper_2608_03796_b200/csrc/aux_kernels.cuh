@@ -28,7 +28,11 @@ struct WsHeader {
   float denom;       // divisor of the mean actually used
   float tau;
   double loss_sum;   // sum of counted per-token losses
+  long long chunk;   // tokens per chunk of the forward call that filled the workspace
+  int g_state;       // what the [chunk, V] buffer holds after forward: G_NONE, G_EXPONENTIALS (option
+                     // stored_exponentials: backward converts them once), G_CONSUMED (they have been converted)
 };
+enum { G_NONE = 0, G_EXPONENTIALS = 1, G_CONSUMED = 2 };
 
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
@@ -45,6 +49,7 @@ __global__ void header_reset_kernel(WsHeader* hdr) {
   if (threadIdx.x == 0 && blockIdx.x == 0) {
     hdr->status = 0; hdr->where = 0; hdr->magic = 0; hdr->go = 0;
     hdr->n_bad_idx = 0; hdr->n_tokens = 0; hdr->denom = 0.f; hdr->loss_sum = 0.0;
+    hdr->chunk = 0; hdr->g_state = G_NONE;
   }
 }
 
@@ -176,9 +181,11 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
 
 // ------------------------------------------------------------------------------------ single-pass step
 // The single-pass forward + backward needs the divisor of the mean before the first chunk (the
-// two-call path learns it at the end of forward): N = number of counted tokens, or the override.
+// two-call path learns it at the end of forward): N = number of counted tokens, or the override (a host
+// value, or a device value the caller reduced over its ranks: denom_dev).
 __global__ void __launch_bounds__(1024)
-count_tokens_kernel(const uint8_t* __restrict__ mask, long long T, float denom_override, WsHeader* hdr) {
+count_tokens_kernel(const uint8_t* __restrict__ mask, long long T, float denom_override,
+                    const double* __restrict__ denom_dev, WsHeader* hdr, double* __restrict__ count_out) {
   __shared__ long long part[32];
   long long c = 0;
   if (mask) { for (long long t = threadIdx.x; t < T; t += 1024) c += mask[t] != 0; }
@@ -189,8 +196,9 @@ count_tokens_kernel(const uint8_t* __restrict__ mask, long long T, float denom_o
   if (threadIdx.x == 0) {
     long long n = 0;
     for (int i = 0; i < 32; ++i) n += part[i];
+    if (count_out != nullptr) { *count_out = (double)n; return; }   // the stand-alone count (kdkl_count_tokens)
     hdr->n_tokens = n;
-    hdr->denom = denom_override > 0.f ? denom_override : (float)n;
+    hdr->denom = denom_dev != nullptr ? (float)*denom_dev : (denom_override > 0.f ? denom_override : (float)n);
   }
 }
 
@@ -220,6 +228,9 @@ e_to_g_kernel(__nv_bfloat16* __restrict__ G, long long ldg /* elements per row *
               const int* __restrict__ idx_sorted, const float* __restrict__ p_sorted, const int* __restrict__ nvalid,
               int Ktop, float bias, int n_seg, WsHeader* hdr, const int* go) {
   if (go != nullptr && *go == 0) return;       // backward gate: the workspace does not hold this call's state
+  // called from kdkl_backward (go given): the conversion is in place, so a second backward on this state must
+  // not convert again - the header says so from here on (bwd_coef_kernel of that later call reads it)
+  if (go != nullptr && blockIdx.x == 0 && threadIdx.x == 0) hdr->g_state = G_CONSUMED;
   const long long row = blockIdx.x / n_seg;
   const int c_begin = (int)(blockIdx.x - row * n_seg) * E2G_SEG;
   const int c_end = c_begin + E2G_SEG < n_cols ? c_begin + E2G_SEG : n_cols;
@@ -302,6 +313,10 @@ tile_live_kernel(const uint8_t* __restrict__ mask, long long T, long long chunk,
 // coalesce. 32 lanes per row (1024 threads) keep 32 x 32 partial pairs in flight per block: the kernel
 // reads chunk x n_tiles x 8 bytes (16 MiB at chunk 4096, V = 131072) and is bound by memory latency.
 constexpr int COMBINE_WARPS = 32;
+// With stored exponentials e = 2^(s - 64) in bf16, entries below s = -62 flush to zero. A row's entries that matter
+// lie within about 20 of its log2-normaliser, so rows with lz2 >= -40 lose nothing; below that the call reports
+// KDKL_ERR_RANGE (the two-call path has no such limit).
+constexpr float kExpStoreMinLz2 = -40.f;
 __global__ void __launch_bounds__(COMBINE_WARPS * 32)
 combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_s, long long part_stride,
                int n_tiles, int rows, long long row0, int K, float inv_tau, const int* __restrict__ nvalid,
@@ -309,7 +324,8 @@ combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_
                const int* __restrict__ colread, const float* __restrict__ Mv, const float* __restrict__ Hent,
                const uint8_t* __restrict__ mask, float* __restrict__ lz2, float* __restrict__ logZ_nat,
                float* __restrict__ loss_tok, float* __restrict__ loss_tok_user, float* __restrict__ g_logits,
-               int* __restrict__ g_idx, int v0, float* __restrict__ shard_stats, long long T_total, WsHeader* hdr) {
+               int* __restrict__ g_idx, int v0, float* __restrict__ shard_stats, long long T_total, WsHeader* hdr,
+               int exp_stored) {
   __shared__ float sm_m[COMBINE_WARPS][32], sm_s[COMBINE_WARPS][32];
   __shared__ float sm_lz[32];
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
@@ -339,6 +355,11 @@ combine_kernel(const float* __restrict__ part_m, const float* __restrict__ part_
       mm = mn;
     }
     const float l2 = row_counted ? mm + log2f(ss) : 0.f;
+    // stored exponentials carry a fixed bias instead of the row maximum: a row whose scaled logits all sit
+    // far below zero would flush to zero there (its softmax term would vanish from G unnoticed)
+    if (exp_stored && row_counted && l2 < kExpStoreMinLz2) {
+      atomicCAS(&hdr->status, 0, -13); atomicCAS(&hdr->where, 0, (int)(row0 + r));
+    }
     sm_lz[tx] = l2;
     lz2[row0 + r] = l2;
     logZ_nat[row0 + r] = l2 * kLn2;
@@ -420,8 +441,8 @@ __global__ void shard_finish_kernel(const float* __restrict__ all_stats, int R, 
 // workspace as complete for backward.
 __global__ void __launch_bounds__(1024)
 loss_reduce_kernel(const float* __restrict__ loss_tok, const uint8_t* __restrict__ mask, long long T,
-                   float denom_override, float tau, long long H, long long V, int K, float* loss_out,
-                   WsHeader* hdr) {
+                   float denom_override, const double* __restrict__ denom_dev, float tau, long long H, long long V,
+                   int K, long long chunk, int g_state, float* loss_out, WsHeader* hdr) {
   __shared__ double sm_sum[1024];
   __shared__ long long sm_cnt[1024];
   double acc = 0.0;
@@ -438,9 +459,9 @@ loss_reduce_kernel(const float* __restrict__ loss_tok, const uint8_t* __restrict
   }
   if (threadIdx.x == 0) {
     const long long n = sm_cnt[0];
-    const float denom = denom_override > 0.f ? denom_override : (float)n;
+    const float denom = denom_dev != nullptr ? (float)*denom_dev : (denom_override > 0.f ? denom_override : (float)n);
     hdr->n_tokens = n; hdr->denom = denom; hdr->loss_sum = sm_sum[0]; hdr->tau = tau;
-    hdr->T = T; hdr->H = H; hdr->V = V; hdr->K = K;
+    hdr->T = T; hdr->H = H; hdr->V = V; hdr->K = K; hdr->chunk = chunk; hdr->g_state = g_state;
     *loss_out = denom > 0.f ? (float)(sm_sum[0] / (double)denom) : 0.f;
     __threadfence();
     hdr->magic = KDKL_MAGIC;
@@ -450,11 +471,24 @@ loss_reduce_kernel(const float* __restrict__ loss_tok, const uint8_t* __restrict
 // ------------------------------------------------------------------------------------ backward prep
 // coefA_t = g_t M_t / tau, coefB_t = g_t / tau with g_t = grad_loss * mask_t / denom
 // (Algorithm 1 backward: G = (M g) q, G -= p g; the 1/tau is the chain rule through z/tau).
-// Also checks that the workspace was filled by a forward call of the same shape.
+// Also checks that the workspace was filled by a forward call of the same shape, chunk size and temperature,
+// and - when backward is to convert stored exponentials instead of projecting again - that forward left
+// them and no earlier backward has converted them already (the conversion is in place: it can run once;
+// e_to_g_kernel marks them consumed). Block 0 records the verdict in `go` for the kernels that follow;
+// nothing the verdict depends on is written by this grid.
 __global__ void bwd_coef_kernel(const float* __restrict__ Mv, const uint8_t* __restrict__ mask, long long T,
-                                long long H, long long V, int K, float grad_loss, float inv_tau,
-                                float* __restrict__ coefA, float* __restrict__ coefB, WsHeader* hdr) {
-  const bool state_ok = hdr->magic == KDKL_MAGIC && hdr->T == T && hdr->H == H && hdr->V == V && hdr->K == K;
+                                long long H, long long V, int K, long long chunk, float tau, int want_exponentials,
+                                float grad_loss, float inv_tau, float* __restrict__ coefA,
+                                float* __restrict__ coefB, WsHeader* hdr) {
+  __shared__ int sm_ok;
+  if (threadIdx.x == 0) {
+    bool ok = hdr->magic == KDKL_MAGIC && hdr->T == T && hdr->H == H && hdr->V == V && hdr->K == K &&
+              hdr->chunk == chunk && hdr->tau == tau;
+    if (want_exponentials) ok = ok && hdr->g_state == G_EXPONENTIALS;
+    sm_ok = ok ? 1 : 0;
+  }
+  __syncthreads();
+  const bool state_ok = sm_ok != 0;
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     hdr->go = state_ok ? 1 : 0;
     if (!state_ok) atomicCAS(&hdr->status, 0, -9);

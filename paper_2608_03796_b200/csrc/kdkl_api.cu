@@ -117,23 +117,51 @@ static int make_tmap_out_bf16(CUtensorMap* m, void* base, uint64_t cols, uint64_
 constexpr int kNCTA = KDKL_NCTA;
 constexpr int kTileM = GemmCfg<kNCTA>::TILE_M;
 constexpr int kBRows = GemmCfg<kNCTA>::B_ROWS;
-struct DeviceInfo { int sm_count; int cc_major; bool ok; };
+// What the library has learnt about each device, asked once per device and process (a benign race: two
+// threads asking at the same time store the same values).
+constexpr int kMaxDevices = 64;
+struct DeviceInfo { int dev; int sm_count; int cc_major; };
+struct DeviceCache { bool known; int sm_count; int cc_major; };
+static DeviceCache g_devices[kMaxDevices];
 static int device_info(DeviceInfo* di) {
   int dev = 0;
   KDKL_CUDA(cudaGetDevice(&dev));
+  di->dev = dev;
+  if (dev >= 0 && dev < kMaxDevices && g_devices[dev].known) {
+    di->sm_count = g_devices[dev].sm_count; di->cc_major = g_devices[dev].cc_major;
+    return KDKL_OK;
+  }
   KDKL_CUDA(cudaDeviceGetAttribute(&di->sm_count, cudaDevAttrMultiProcessorCount, dev));
   KDKL_CUDA(cudaDeviceGetAttribute(&di->cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+  if (dev >= 0 && dev < kMaxDevices) {
+    g_devices[dev].sm_count = di->sm_count; g_devices[dev].cc_major = di->cc_major; g_devices[dev].known = true;
+  }
   return KDKL_OK;
+}
+// SM count of the current device for sizing decisions that are also taken where there may be no device
+// (kdkl_workspace_bytes on a build machine): a B200's 148 then.
+static int sm_count_or_default() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 148; }
+  if (dev >= 0 && dev < kMaxDevices && g_devices[dev].known) return g_devices[dev].sm_count;
+  DeviceInfo di;
+  if (device_info(&di) != KDKL_OK || di.sm_count < 2) { cudaGetLastError(); return 148; }
+  return di.sm_count;
 }
 
 template <int EPI, bool A_MN, bool B_MN>
 static int launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const GemmParams& p,
-                       int sm_count, cudaStream_t st) {
+                       const DeviceInfo& di, cudaStream_t st) {
   auto kern = gemm_tcgen05_kernel<EPI, A_MN, B_MN, kNCTA>;
   constexpr int smem = GemmCfg<kNCTA>::SMEM_BYTES;
-  // set on every launch: the attribute belongs to the current device's copy of the kernel, and a
-  // process may drive several devices
-  KDKL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  // The shared-memory limit belongs to the current device's copy of this instantiation: set once per device
+  // (a process may drive several), not per launch.
+  static bool attr_set[kMaxDevices];
+  const int sm_count = di.sm_count;
+  if (di.dev < 0 || di.dev >= kMaxDevices || !attr_set[di.dev]) {
+    KDKL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    if (di.dev >= 0 && di.dev < kMaxDevices) attr_set[di.dev] = true;
+  }
   // persistent: one worker (a CTA, or a pair of CTAs on neighbouring SMs) per SM (pair), each walking
   // the work units with a stride of the worker count
   const int units = p.m_tiles * p.n_tiles * p.k_splits;
@@ -163,9 +191,9 @@ static inline size_t up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // How many work units to cut each output tile's contraction into so that the units fill whole
 // waves of SMs: the smallest count (<= 4, each unit keeping >= 32 k-blocks) that reaches 95 %
-// wave efficiency, else the most efficient one. Sized for the 148 SMs of a B200.
-static int choose_k_splits(long long tiles, long long kblocks) {
-  const long long sms = 148 / kNCTA;
+// wave efficiency, else the most efficient one, for the device's count of workers (SMs / CTAs per tile).
+static int choose_k_splits(long long tiles, long long kblocks, int sm_count) {
+  const long long sms = (sm_count < kNCTA ? kNCTA : sm_count) / kNCTA;
   int best = 1;
   double best_eff = 0.0;
   for (int sp = 1; sp <= 4; ++sp) {
@@ -189,15 +217,11 @@ struct WsLayout {
   long long tiles_per_chunk, n_live;   // live-row-tile flags: one per kTileM rows of every chunk
 };
 
-// Debug aid: KDKL_WS_GUARD_BYTES=n in the environment puts n untouched bytes after every workspace slab (and makes
-// the workspace that much larger), so that a test can pre-fill the workspace, run, and see whether any kernel
-// wrote past the end of a slab (kdkl_workspace_layout gives the slab table). Unset or 0: the compact layout.
-static size_t ws_guard_bytes() {
-  const char* e = getenv("KDKL_WS_GUARD_BYTES");
-  if (e == nullptr) return 0;
-  const long long v = atoll(e);
-  return v > 0 && v <= (1ll << 20) ? up((size_t)v, 256) : 0;
-}
+// Debug aid: kdkl_debug_guard_bytes(n) puts n untouched bytes after every workspace slab (and makes the
+// workspace that much larger), so that a test can pre-fill the workspace, run, and see whether any kernel
+// wrote past the end of a slab (kdkl_workspace_layout gives the slab table). 0: the compact layout.
+static size_t g_guard_bytes = 0;
+static size_t ws_guard_bytes() { return g_guard_bytes; }
 
 static WsLayout ws_layout(long long T, long long H, long long V, int K, long long chunk) {
   WsLayout L;
@@ -232,7 +256,8 @@ static WsLayout ws_layout(long long T, long long H, long long V, int K, long lon
   L.part_m = take((size_t)L.n_tiles_v * L.Cpad * 4);
   L.part_s = take((size_t)L.n_tiles_v * L.Cpad * 4);
   L.G = take((size_t)L.Cpad * L.Vpad * 2);
-  L.dh_splits = choose_k_splits(((L.C + kTileM - 1) / kTileM) * ((H + BN - 1) / BN), (V + BK - 1) / BK);
+  L.dh_splits = choose_k_splits(((L.C + kTileM - 1) / kTileM) * ((H + BN - 1) / BN), (V + BK - 1) / BK,
+                                sm_count_or_default());
   L.dh_part = take(L.dh_splits > 1 ? (size_t)L.dh_splits * L.Cpad * H * 4 : 0);
   L.tiles_per_chunk = (L.C + kTileM - 1) / kTileM;
   L.n_live = ((T + L.C - 1) / L.C) * L.tiles_per_chunk;
@@ -241,12 +266,14 @@ static WsLayout ws_layout(long long T, long long H, long long V, int K, long lon
   return L;
 }
 
-// Options of this or of the previous struct size (without stored_exponentials) are accepted.
+// Options of this or of an earlier struct size (without denom_device; without stored_exponentials) are accepted.
 static int copy_options(const kdkl_options* opt, kdkl_options* eff) {
   memset(eff, 0, sizeof(*eff));
   if (!opt) return KDKL_OK;
-  constexpr int32_t kOldSize = (int32_t)offsetof(kdkl_options, stored_exponentials);
-  if (opt->struct_size != (int32_t)sizeof(kdkl_options) && opt->struct_size != kOldSize) return KDKL_ERR_ARG;
+  constexpr int32_t kSize1 = (int32_t)offsetof(kdkl_options, stored_exponentials);
+  constexpr int32_t kSize2 = (int32_t)(offsetof(kdkl_options, stored_exponentials) + sizeof(int32_t));
+  if (opt->struct_size != (int32_t)sizeof(kdkl_options) && opt->struct_size != kSize1 && opt->struct_size != kSize2)
+    return KDKL_ERR_ARG;
   memcpy(eff, opt, (size_t)opt->struct_size);
   eff->struct_size = (int32_t)sizeof(kdkl_options);
   if (eff->stored_exponentials < 0 || eff->stored_exponentials > 1) return KDKL_ERR_ARG;
@@ -255,7 +282,7 @@ static int copy_options(const kdkl_options* opt, kdkl_options* eff) {
 
 static int check_common(const void* hidden, const void* weight, long long T, long long H, long long V, int K,
                         long long chunk, float tau, const kdkl_options* opt, const void* ws, size_t ws_bytes,
-                        kdkl_options* eff, WsLayout* L) {
+                        kdkl_options* eff, WsLayout* L, DeviceInfo* di) {
   if (!hidden || !weight || !ws) return KDKL_ERR_NULL;
   if (T < 1 || H < 1 || V < 1 || K < 1 || K > KDKL_MAX_K || (H % 8) != 0 || V >= (1ll << 31) || T >= (1ll << 31))
     return KDKL_ERR_SHAPE;
@@ -268,10 +295,9 @@ static int check_common(const void* hidden, const void* weight, long long T, lon
   *L = ws_layout(T, H, V, K, chunk);
   if (eff->stored_exponentials && T > L->C) return KDKL_ERR_ARG;   // needs one chunk over all tokens
   if (ws_bytes < L->total) return KDKL_ERR_WORKSPACE;
-  DeviceInfo di;
-  int rc = device_info(&di);
+  int rc = device_info(di);
   if (rc) return rc;
-  if (di.cc_major != 10) return KDKL_ERR_ARCH;
+  if (di->cc_major != 10) return KDKL_ERR_ARCH;
   return KDKL_OK;
 }
 
@@ -338,8 +364,8 @@ struct ChunkOut {
   const uint8_t* live_c;   // the chunk's row-tile flags for the dW contraction (nullptr: none)
   int accumulate_dw;
 };
-static int launch_chunk_outputs(const ChunkOut& c, const CUtensorMap& tmWmn, const CUtensorMap& tmdW, int sm_count,
-                                cudaStream_t st) {
+static int launch_chunk_outputs(const ChunkOut& c, const CUtensorMap& tmWmn, const CUtensorMap& tmdW,
+                                const DeviceInfo& di, cudaStream_t st) {
   const WsLayout& L = *c.L;
   const long long rows = c.rows, H = c.H, V = c.V, s0 = c.s0;
   int rc;
@@ -353,7 +379,7 @@ static int launch_chunk_outputs(const ChunkOut& c, const CUtensorMap& tmWmn, con
   p2.status = &c.hdr->status; p2.go = c.go;
   p2.m_live = c.live_m;              // dead row tiles: their dH rows are written as zeros
   // a short last chunk may want a different split; never more than the workspace was sized for
-  int sp = choose_k_splits((long long)p2.m_tiles * p2.n_tiles, (V + BK - 1) / BK);
+  int sp = choose_k_splits((long long)p2.m_tiles * p2.n_tiles, (V + BK - 1) / BK, di.sm_count);
   if (sp > L.dh_splits) sp = L.dh_splits;
   p2.k_splits = sp;
   __nv_bfloat16* dh16 = c.o->dhidden_dtype == 0 ? reinterpret_cast<__nv_bfloat16*>(c.dhidden) + s0 * H : nullptr;
@@ -363,17 +389,17 @@ static int launch_chunk_outputs(const ChunkOut& c, const CUtensorMap& tmWmn, con
     float* part = at<float>(c.ws, L.dh_part);
     p2.split_rows = (int)L.Cpad;
     if ((rc = make_tmap_out_f32(&tmdH, part, (uint64_t)H, (uint64_t)sp * L.Cpad, (uint64_t)H))) return rc;
-    if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, sm_count, st))) return rc;
+    if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, di, st))) return rc;
     const long long n4 = rows * H / 4;
     splitk_fixup_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(part, (long long)L.Cpad * H, sp, n4, dh16, dh32,
                                                                      c.go);
     KDKL_LAUNCHED("splitk_fixup_kernel");
   } else if (dh16 != nullptr) {
     if ((rc = make_tmap_out_bf16(&tmdH, dh16, (uint64_t)H, (uint64_t)rows, (uint64_t)H))) return rc;
-    if ((rc = launch_gemm<EPI_STORE_BF16, false, true>(tmG, tmWmn, tmdH, p2, sm_count, st))) return rc;
+    if ((rc = launch_gemm<EPI_STORE_BF16, false, true>(tmG, tmWmn, tmdH, p2, di, st))) return rc;
   } else {
     if ((rc = make_tmap_out_f32(&tmdH, dh32, (uint64_t)H, (uint64_t)rows, (uint64_t)H))) return rc;
-    if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, sm_count, st))) return rc;
+    if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, di, st))) return rc;
   }
 
   if ((rc = make_tmap_bf16(&tmGmn, c.G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, 64, BK))) return rc;
@@ -387,7 +413,7 @@ static int launch_chunk_outputs(const ChunkOut& c, const CUtensorMap& tmWmn, con
   // dead row tiles of G are zeros: they are left out of the contraction over tokens (the kernel takes up to 32 flags)
   p3.k_live = (rows <= 32ll * kTileM && (rows + BK - 1) / BK <= MAX_LIVE_KB) ? c.live_c : nullptr;
   stage_mark(ST_B3, st);
-  return launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, tmdW, p3, sm_count, st);
+  return launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, tmdW, p3, di, st);
 }
 
 
@@ -426,10 +452,9 @@ static int forward_impl(const void* hidden, const void* weight, const int32_t* t
   if (!topk_idx || !topk_val || (!loss_out && !shard_stats)) return KDKL_ERR_NULL;
   kdkl_options o;
   WsLayout L;
-  int rc = check_common(hidden, weight, T, H, V, K, chunk, tau, opt, ws, ws_bytes, &o, &L);
-  if (rc) return rc;
   DeviceInfo di;
-  if ((rc = device_info(&di))) return rc;
+  int rc = check_common(hidden, weight, T, H, V, K, chunk, tau, opt, ws, ws_bytes, &o, &L, &di);
+  if (rc) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   WsHeader* hdr = at<WsHeader>(ws, L.hdr);
   const float inv_tau = 1.0f / tau;
@@ -455,9 +480,9 @@ static int forward_impl(const void* hidden, const void* weight, const int32_t* t
       CUtensorMap tmE;
       if ((rc = make_tmap_out_bf16(&tmE, at<__nv_bfloat16>(ws, L.G), (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad)))
         return rc;
-      if ((rc = launch_gemm<EPI_LSE_E, false, false>(tmA, tmW, tmE, p, di.sm_count, st))) return rc;
+      if ((rc = launch_gemm<EPI_LSE_E, false, false>(tmA, tmW, tmE, p, di, st))) return rc;
     } else {
-      if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA /*no output map*/, p, di.sm_count, st))) return rc;
+      if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA /*no output map*/, p, di, st))) return rc;
     }
     stage_mark(ST_COMBINE, st);
 
@@ -530,10 +555,9 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
   if (((uintptr_t)dhidden & 15) || ((uintptr_t)dweight & 15)) return KDKL_ERR_ALIGN;
   kdkl_options o;
   WsLayout L;
-  int rc = check_common(hidden, weight, T, H, V, K, chunk, tau, opt, ws, ws_bytes, &o, &L);
-  if (rc) return rc;
   DeviceInfo di;
-  if ((rc = device_info(&di))) return rc;
+  int rc = check_common(hidden, weight, T, H, V, K, chunk, tau, opt, ws, ws_bytes, &o, &L, &di);
+  if (rc) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   WsHeader* hdr = at<WsHeader>(ws, L.hdr);
   const int* go = &hdr->go;
@@ -595,12 +619,12 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
           at<int>(ws, L.nvalid) + s0, K, kExpBias, n_seg, hdr, go);
       KDKL_LAUNCHED("e_to_g_kernel");
     } else {
-      if ((rc = launch_gemm<EPI_DLOGITS, false, false>(tmA, tmW, tmGout, p, di.sm_count, st))) return rc;
+      if ((rc = launch_gemm<EPI_DLOGITS, false, false>(tmA, tmW, tmGout, p, di, st))) return rc;
     }
 
     ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, go, live_m, live_c,
                 (ci > 0 || o.accumulate_dweight) ? 1 : 0};
-    if ((rc = launch_chunk_outputs(co, tmWmn, tmdW, di.sm_count, st))) return rc;
+    if ((rc = launch_chunk_outputs(co, tmWmn, tmdW, di, st))) return rc;
   }
   return KDKL_OK;
 }
@@ -618,10 +642,9 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
   if (((uintptr_t)dhidden & 15) || ((uintptr_t)dweight & 15)) return KDKL_ERR_ALIGN;
   kdkl_options o;
   WsLayout L;
-  int rc = check_common(hidden, weight, T, H, V, K, chunk, tau, opt, ws, ws_bytes, &o, &L);
-  if (rc) return rc;
   DeviceInfo di;
-  if ((rc = device_info(&di))) return rc;
+  int rc = check_common(hidden, weight, T, H, V, K, chunk, tau, opt, ws, ws_bytes, &o, &L, &di);
+  if (rc) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   WsHeader* hdr = at<WsHeader>(ws, L.hdr);
   const float inv_tau = 1.0f / tau;
@@ -656,7 +679,7 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
     fill_forward_params(&p, L, ws, s0, rows, H, V, K, inv_tau, live_c);
     const uint8_t* live_m = p.m_live;
     stage_mark(ST_F1, st);
-    if ((rc = launch_gemm<EPI_LSE_E, false, false>(tmA, tmW, tmGout, p, di.sm_count, st))) return rc;
+    if ((rc = launch_gemm<EPI_LSE_E, false, false>(tmA, tmW, tmGout, p, di, st))) return rc;
     stage_mark(ST_COMBINE, st);
     combine_kernel<<<(unsigned)((rows + 31) / 32), COMBINE_WARPS * 32, 0, st>>>(
         at<float>(ws, L.part_m), at<float>(ws, L.part_s), L.Cpad, (int)L.n_tiles_v, (int)rows, s0, K, inv_tau,
@@ -679,7 +702,7 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
     // dH[chunk] = G W and dW (+)= G^T h, exactly as in kdkl_backward
     ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, nullptr, live_m, live_c,
                 (ci > 0 || o.accumulate_dweight) ? 1 : 0};
-    if ((rc = launch_chunk_outputs(co, tmWmn, tmdW, di.sm_count, st))) return rc;
+    if ((rc = launch_chunk_outputs(co, tmWmn, tmdW, di, st))) return rc;
   }
   stage_mark(ST_REDUCE, st);
   loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, tau, H, V, K,
@@ -979,9 +1002,9 @@ static int teacher_topk_impl(const void* hidden, const void* weight, int64_t T, 
     if (stored) {
       CUtensorMap tmZ;
       if ((rc = make_tmap_out_f32(&tmZ, at<float>(ws, L.z), (uint64_t)V, (uint64_t)rows, (uint64_t)L.ldz))) return rc;
-      if ((rc = launch_gemm<EPI_LSE_Z, false, false>(tmA, tmW, tmZ, p, di.sm_count, st))) return rc;
+      if ((rc = launch_gemm<EPI_LSE_Z, false, false>(tmA, tmW, tmZ, p, di, st))) return rc;
     } else {
-      if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA, p, di.sm_count, st))) return rc;
+      if ((rc = launch_gemm<EPI_LSE, false, false>(tmA, tmW, tmA, p, di, st))) return rc;
     }
     topk_threshold_kernel<<<(unsigned)rows, 32, (size_t)L.npad * 4, st>>>(
         at<float>(ws, L.part_m), at<float>(ws, L.part_s), L.Cpad, (int)L.n_tiles, L.npad, K, at<float>(ws, L.thr),
@@ -998,7 +1021,7 @@ static int teacher_topk_impl(const void* hidden, const void* weight, int64_t T, 
       // sweep 2: recompute, emit everything at or above the row's threshold
       p.thr = at<float>(ws, L.thr); p.cand_cnt = at<int>(ws, L.cnt);
       p.cand_idx = at<int>(ws, L.cidx); p.cand_val = at<float>(ws, L.cval); p.cand_cap = L.cap;
-      if ((rc = launch_gemm<EPI_TOPK, false, false>(tmA, tmW, tmA, p, di.sm_count, st))) return rc;
+      if ((rc = launch_gemm<EPI_TOPK, false, false>(tmA, tmW, tmA, p, di, st))) return rc;
     }
     KDKL_CUDA(cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.cpad * 8));
     topk_select_kernel<<<(unsigned)rows, 32, (size_t)L.cpad * 8, st>>>(
@@ -1125,10 +1148,10 @@ int kdkl_gemm_bf16(const void* A, const void* B, float* C, int64_t M, int64_t N,
   p.status = status; p.accumulate = 0;
   CUtensorMap tc;
   if ((rc = make_tmap_out_f32(&tc, C, (uint64_t)N, (uint64_t)M, (uint64_t)N))) return rc;
-  if (a_mn && b_mn) return launch_gemm<EPI_STORE_F32, true, true>(ta, tb, tc, p, di.sm_count, st);
-  if (a_mn) return launch_gemm<EPI_STORE_F32, true, false>(ta, tb, tc, p, di.sm_count, st);
-  if (b_mn) return launch_gemm<EPI_STORE_F32, false, true>(ta, tb, tc, p, di.sm_count, st);
-  return launch_gemm<EPI_STORE_F32, false, false>(ta, tb, tc, p, di.sm_count, st);
+  if (a_mn && b_mn) return launch_gemm<EPI_STORE_F32, true, true>(ta, tb, tc, p, di, st);
+  if (a_mn) return launch_gemm<EPI_STORE_F32, true, false>(ta, tb, tc, p, di, st);
+  if (b_mn) return launch_gemm<EPI_STORE_F32, false, true>(ta, tb, tc, p, di, st);
+  return launch_gemm<EPI_STORE_F32, false, false>(ta, tb, tc, p, di, st);
 }
 
 }  // extern "C"

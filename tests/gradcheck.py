@@ -21,6 +21,12 @@ C_SIGMA = 8 standard deviations (5e8 elements of a full-size dW never reach it b
 relative Frobenius error must stay below the tolerance stated for the whole matrix (1e-2): about three times
 what the model predicts (u / sqrt 3 = 2.3e-3, plus the output rounding), so a row whose sparse teacher term
 or tail columns went missing fails although it vanishes inside the whole-matrix norm.
+
+Two roundings (single-pass step). The first rounding is of the stored exponential, so its error scales with the
+dense softmax part a_t q_v of an entry, not with G itself; at a support entry where the student already matches
+the teacher (M q ~ p) G is much smaller than that part, and a vocabulary row of dW made of such entries has a
+small norm with an error of ordinary size. With roundings >= 2 every row is therefore judged against at least
+the median row's scale (norm and rms), which is the scale of the dense part.
 """
 import numpy as np
 
@@ -29,9 +35,9 @@ C_SIGMA = 8.0
 ROW_FRO = 1e-2
 
 
-def elementwise_tolerance(ref_block, out_bf16=False, roundings=1):
+def elementwise_tolerance(ref_block, out_bf16=False, roundings=1, rms_floor=0.0):
     """The bound above for a block of whole rows of the oracle's matrix (float64 [rows, cols])."""
-    rms = np.sqrt(np.mean(ref_block * ref_block, axis=1, keepdims=True))
+    rms = np.maximum(np.sqrt(np.mean(ref_block * ref_block, axis=1, keepdims=True)), rms_floor)
     rel = U_BF16 * (2.0 if out_bf16 else 1.0)
     return rel * np.abs(ref_block) + C_SIGMA * np.sqrt(float(roundings)) * (U_BF16 / np.sqrt(3.0)) * rms
 
@@ -47,6 +53,13 @@ def check_grad_matrix(got, ref, name, out_bf16=False, roundings=1, row_fro=ROW_F
     norms = np.empty(rows)
     errs = np.empty(rows)
     worst_ratio, worst_at = 0.0, None
+    norm_floor = 0.0
+    if roundings >= 2 and rows:
+        for r0 in range(0, rows, block):
+            b = np.asarray(ref[r0:r0 + block], dtype=np.float64)
+            norms[r0:r0 + len(b)] = np.sqrt((b * b).sum(axis=1))
+        norm_floor = float(np.median(norms))
+    rms_floor = norm_floor / np.sqrt(ref.shape[1])
     for r0 in range(0, rows, block):
         b = np.asarray(ref[r0:r0 + block], dtype=np.float64)
         a = np.asarray(got[r0:r0 + block], dtype=np.float64)
@@ -54,7 +67,7 @@ def check_grad_matrix(got, ref, name, out_bf16=False, roundings=1, row_fro=ROW_F
         diff = np.abs(a - b)
         norms[r0:r0 + len(b)] = np.sqrt((b * b).sum(axis=1))
         errs[r0:r0 + len(b)] = np.sqrt((diff * diff).sum(axis=1))
-        tol = elementwise_tolerance(b, out_bf16, roundings)
+        tol = elementwise_tolerance(b, out_bf16, roundings, rms_floor)
         if extra_tol is not None:
             tol = tol + (extra_tol if np.ndim(extra_tol) == 0 else np.asarray(extra_tol)[r0:r0 + block])
         # rows the oracle holds as exact zeros (ignored tokens) must be exact zeros
@@ -68,7 +81,7 @@ def check_grad_matrix(got, ref, name, out_bf16=False, roundings=1, row_fro=ROW_F
                                 f"{worst_ratio:.2f} x its tolerance")
     # per-row relative Frobenius error, on every row whose norm is not negligible next to the largest
     live = norms > 1e-6 * norms.max() if rows and norms.max() > 0 else np.zeros(rows, bool)
-    rel = np.where(live, errs / np.where(live, norms, 1.0), 0.0)
+    rel = np.where(live, errs / np.maximum(np.where(live, norms, 1.0), norm_floor), 0.0)
     r = int(np.argmax(rel)) if rows else 0
     assert not rows or rel[r] <= row_fro, f"{name}: row {r} relative error {rel[r]:.3e} > {row_fro:.0e}"
     return (float(rel[r]) if rows else 0.0), worst_ratio

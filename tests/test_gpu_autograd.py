@@ -75,3 +75,30 @@ def test_single_pass_autograd_matches_oracle():
         assert abs(loss.item() - o["loss"]) <= 1e-3 * abs(o["loss"])
         assert _fro(h.grad.float().cpu().double().numpy(), scale * o["dH"]) <= 1e-2
         assert _fro(W.grad.float().cpu().double().numpy(), scale * o["dW"]) <= 1e-2
+
+
+def test_two_live_losses_of_one_shape_do_not_share_state():
+    """loss1 + loss2 with the same shapes, one backward: each forward must own its saved state (prepared teacher,
+    log Z, retained mass) until its backward has run. Compared with the oracle on each batch."""
+    dev = torch.device("cuda:0")
+    cfg = I.CONFIGS["c1"]
+    d1 = I.make_inputs(cfg, device=dev)
+    d2 = I.make_inputs(I.Config("c1b", T=cfg.T, H=cfg.H, V=cfg.V, K=cfg.K, chunk=cfg.chunk, tok_offset=False,
+                                seed=cfg.seed + 7), device=dev)
+    W = d1["weight"].clone().requires_grad_(True)
+    for single_pass in (False, True):
+        W.grad = None
+        h1 = d1["hidden"].clone().requires_grad_(True)
+        h2 = d2["hidden"].clone().requires_grad_(True)
+        l1 = fused_chunked_kl(h1, W, d1["topk_idx"], d1["topk_val"], chunk=cfg.chunk, single_pass=single_pass)
+        l2 = fused_chunked_kl(h2, W, d2["topk_idx"], d2["topk_val"], chunk=cfg.chunk, single_pass=single_pass)
+        (l1 + l2).backward()
+        Wn = d1["weight"].cpu().double().numpy()
+        o1 = kdkl_oracle(d1["hidden"].cpu().double().numpy(), Wn, d1["topk_idx"].cpu().numpy(),
+                         d1["topk_val"].cpu().numpy(), tau=cfg.tau)
+        o2 = kdkl_oracle(d2["hidden"].cpu().double().numpy(), Wn, d2["topk_idx"].cpu().numpy(),
+                         d2["topk_val"].cpu().numpy(), tau=cfg.tau)
+        assert abs(l1.item() - o1["loss"]) <= 1e-3 * abs(o1["loss"]) and abs(l2.item() - o2["loss"]) <= 1e-3 * abs(o2["loss"])
+        assert _fro(h1.grad.float().cpu().double().numpy(), o1["dH"]) <= 1e-2
+        assert _fro(h2.grad.float().cpu().double().numpy(), o2["dH"]) <= 1e-2
+        assert _fro(W.grad.float().cpu().double().numpy(), o1["dW"] + o2["dW"]) <= 1e-2
