@@ -20,6 +20,7 @@ ERRORS = {
     -1: "KDKL_ERR_NULL", -2: "KDKL_ERR_SHAPE", -3: "KDKL_ERR_ALIGN", -4: "KDKL_ERR_WORKSPACE",
     -5: "KDKL_ERR_ARG", -6: "KDKL_ERR_ARCH", -7: "KDKL_ERR_CUDA", -8: "KDKL_ERR_TIMEOUT",
     -9: "KDKL_ERR_STATE", -10: "KDKL_ERR_INDEX", -11: "KDKL_ERR_NONFINITE", -12: "KDKL_ERR_OVERFLOW",
+    -13: "KDKL_ERR_RANGE",
 }
 
 EXPORTS = [
@@ -29,7 +30,8 @@ EXPORTS = [
     "kdkl_wait_selftest", "kdkl_teacher_topk", "kdkl_teacher_topk_workspace_bytes",
     "kdkl_feature_loss", "kdkl_feature_loss_workspace_bytes", "kdkl_step_host_record", "kdkl_record_staging_bytes",
     "kdkl_forward_backward", "kdkl_profile_single_pass", "kdkl_teacher_topk_stored",
-    "kdkl_teacher_topk_stored_workspace_bytes", "kdkl_workspace_layout",
+    "kdkl_teacher_topk_stored_workspace_bytes", "kdkl_workspace_layout", "kdkl_count_tokens",
+    "kdkl_debug_guard_bytes",
 ]
 
 FEATURE_MSE, FEATURE_COSINE = 0, 1
@@ -44,7 +46,8 @@ class KdklError(RuntimeError):
 class kdkl_options(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_int32), ("teacher_mode", ctypes.c_int32),
                 ("accumulate_dweight", ctypes.c_int32), ("dhidden_dtype", ctypes.c_int32),
-                ("denom_override", ctypes.c_float), ("stored_exponentials", ctypes.c_int32)]
+                ("denom_override", ctypes.c_float), ("stored_exponentials", ctypes.c_int32),
+                ("denom_device", ctypes.c_void_p)]
 
 
 _lib = None
@@ -64,6 +67,10 @@ def lib() -> ctypes.CDLL:
     L.kdkl_workspace_layout.restype = ctypes.c_int
     L.kdkl_workspace_layout.argtypes = [i64, i64, i64, i32, i64, vp, ctypes.POINTER(ctypes.c_int64),
                                         ctypes.POINTER(ctypes.c_int64), i32]
+    L.kdkl_debug_guard_bytes.restype = ctypes.c_int64
+    L.kdkl_debug_guard_bytes.argtypes = [i64]
+    L.kdkl_count_tokens.restype = ctypes.c_int
+    L.kdkl_count_tokens.argtypes = [vp, i64, vp, vp]
     L.kdkl_forward.restype = ctypes.c_int
     L.kdkl_forward.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i64, f32, vp, vp, sz, vp, vp, vp, vp, vp]
     L.kdkl_forward_shard.restype = ctypes.c_int
@@ -162,9 +169,25 @@ def _stream():
 
 
 def make_options(teacher_mode=0, accumulate_dweight=0, dhidden_dtype=0, denom_override=0.0,
-                 stored_exponentials=0) -> kdkl_options:
+                 stored_exponentials=0, denom_device: Optional[torch.Tensor] = None) -> kdkl_options:
+    """denom_device: a CUDA float64 tensor of one element holding the divisor of the mean (read on the device
+    when the kernels run); the caller keeps it alive until they have run."""
+    ptr = None
+    if denom_device is not None:
+        ptr = _dptr(denom_device, torch.float64, (1,), "denom_device").value
     return kdkl_options(ctypes.sizeof(kdkl_options), teacher_mode, accumulate_dweight, dhidden_dtype, denom_override,
-                        stored_exponentials)
+                        stored_exponentials, ptr)
+
+
+def kdkl_count_tokens(loss_mask: Optional[torch.Tensor], T: int, count_out: torch.Tensor) -> None:
+    """Number of counted tokens (T without a mask) as one float64 on the device; enqueue-only."""
+    _check(lib().kdkl_count_tokens(_dptr(loss_mask, _U8, (T,), "loss_mask"), T,
+                                   _dptr(count_out, torch.float64, (1,), "count_out"), _stream()))
+
+
+def kdkl_debug_guard_bytes(n: int) -> int:
+    """Test hook: n untouched bytes after every workspace slab from now on (0 = compact); returns the old value."""
+    return int(lib().kdkl_debug_guard_bytes(n))
 
 
 def _opt_ptr(opt: Optional[kdkl_options]):
@@ -529,6 +552,8 @@ class TokenShardedFusedKL:
     Rows are independent given the weight, so the only exchanges are three sums over ranks: the number of
     counted tokens (before forward: it is the divisor of the mean), the loss, and the fp32 dweight.
     dhidden needs no communication. ``all_reduce_sum(tensor)`` defaults to torch.distributed (NCCL).
+    The count is taken by the library's kernel and stays on the device: its sum over ranks reaches the
+    kernels through ``kdkl_options.denom_device``, so a step has no host read.
     """
 
     def __init__(self, T_local, H, V, K, chunk=0, temperature=1.0, device="cuda", all_reduce_sum=None):
@@ -539,45 +564,52 @@ class TokenShardedFusedKL:
         self.dhidden = torch.empty(T_local, H, dtype=torch.bfloat16, device=device)
         self.dweight = torch.empty(V, H, dtype=torch.float32, device=device)
         self._all_reduce_sum = all_reduce_sum or ShardedFusedChunkedKL._dist_all_reduce
-        self.opt = None
+        self._launches = [0, 0, 0]
+        self.n_global = torch.zeros(1, dtype=torch.float64, device=device)
+        self.opt = make_options(denom_device=self.n_global)    # every rank divides by the global count
 
     def count_tokens(self, loss_mask=None):
-        """Global number of counted tokens (one small all-reduce and a host read)."""
-        n = torch.tensor([float(self.T if loss_mask is None else int(loss_mask.sum().item()))], device=self.device)
-        self._all_reduce_sum(n)
-        return float(n.item())
+        """Global number of counted tokens, left on the device (one kernel, one small all-reduce)."""
+        kdkl_count_tokens(loss_mask, self.T, self.n_global)
+        self._launches = [kdkl_last_launch_count(), 0, 0]
+        self._all_reduce_sum(self.n_global)
+        return self.n_global
 
-    def forward_local(self, hidden, weight, topk_idx, topk_val, n_global, teacher_lse=None, loss_mask=None):
-        self.opt = make_options(denom_override=n_global)      # every rank divides by the global count
+    def launches_total(self) -> int:
+        """Kernels this rank's last step enqueued (count + forward + backward)."""
+        return sum(self._launches)
+
+    def forward_local(self, hidden, weight, topk_idx, topk_val, teacher_lse=None, loss_mask=None):
         kdkl_forward(hidden, weight, topk_idx, topk_val, self.workspace, self.loss, teacher_lse=teacher_lse,
                      loss_mask=loss_mask, chunk=self.chunk, temperature=self.temperature, opt=self.opt)
+        self._launches[1] = kdkl_last_launch_count()
 
     def forward(self, hidden, weight, topk_idx, topk_val, teacher_lse=None, loss_mask=None):
-        n_global = self.count_tokens(loss_mask)
-        self.forward_local(hidden, weight, topk_idx, topk_val, n_global, teacher_lse, loss_mask)
+        self.count_tokens(loss_mask)
+        self.forward_local(hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask)
         self._all_reduce_sum(self.loss)                        # partial means add up to the global mean
         return self.loss
 
     def backward_local(self, hidden, weight, loss_mask=None, grad_loss=1.0):
         kdkl_backward(hidden, weight, self.K, self.workspace, self.dhidden, self.dweight, loss_mask=loss_mask,
                       chunk=self.chunk, temperature=self.temperature, opt=self.opt, grad_loss=grad_loss)
+        self._launches[2] = kdkl_last_launch_count()
 
     def backward(self, hidden, weight, loss_mask=None, grad_loss=1.0):
         self.backward_local(hidden, weight, loss_mask, grad_loss)
         self._all_reduce_sum(self.dweight)                     # the data-parallel gradient reduction
         return self.dhidden, self.dweight
 
-    def forward_backward_local(self, hidden, weight, topk_idx, topk_val, n_global, teacher_lse=None, loss_mask=None,
+    def forward_backward_local(self, hidden, weight, topk_idx, topk_val, teacher_lse=None, loss_mask=None,
                                grad_loss=1.0):
         """Single-pass step of this rank (three projections) with the global divisor."""
-        self.opt = make_options(denom_override=n_global)
         kdkl_forward_backward(hidden, weight, topk_idx, topk_val, self.workspace, self.loss, self.dhidden,
                               self.dweight, teacher_lse=teacher_lse, loss_mask=loss_mask, chunk=self.chunk,
                               temperature=self.temperature, opt=self.opt, grad_loss=grad_loss)
 
     def forward_backward(self, hidden, weight, topk_idx, topk_val, teacher_lse=None, loss_mask=None, grad_loss=1.0):
-        self.forward_backward_local(hidden, weight, topk_idx, topk_val, self.count_tokens(loss_mask), teacher_lse,
-                                    loss_mask, grad_loss)
+        self.count_tokens(loss_mask)
+        self.forward_backward_local(hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, grad_loss)
         self._all_reduce_sum(self.loss)
         self._all_reduce_sum(self.dweight)
         return self.loss, self.dhidden, self.dweight

@@ -440,6 +440,25 @@ size_t kdkl_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t 
   return ws_layout(T, H, V, K, chunk).total;
 }
 
+int64_t kdkl_debug_guard_bytes(int64_t n) {
+  const int64_t before = (int64_t)g_guard_bytes;
+  if (n < 0) n = 0;
+  if (n > (1ll << 20)) n = 1ll << 20;
+  g_guard_bytes = up((size_t)n, 256);
+  return before;
+}
+
+int kdkl_count_tokens(const uint8_t* loss_mask, int64_t T, double* count_out, void* cuda_stream) {
+  g_launches = 0;
+  if (!count_out) return KDKL_ERR_NULL;
+  if (T < 1 || T >= (1ll << 31)) return KDKL_ERR_SHAPE;
+  if ((uintptr_t)count_out & 7) return KDKL_ERR_ALIGN;
+  count_tokens_kernel<<<1, 1024, 0, reinterpret_cast<cudaStream_t>(cuda_stream)>>>(loss_mask, T, 0.f, nullptr, nullptr,
+                                                                                  count_out);
+  KDKL_LAUNCHED("count_tokens_kernel");
+  return KDKL_OK;
+}
+
 // Forward over the vocabulary rows [v0, v0 + V) this caller holds. Unsharded: v0 = 0, V_total = V,
 // shard_stats = NULL and the loss is finished here. Sharded: the per-token local normaliser and cross
 // term go to shard_stats [2, T] and kdkl_forward_finish completes the loss after the gather.
@@ -491,13 +510,13 @@ static int forward_impl(const void* hidden, const void* weight, const int32_t* t
         at<int>(ws, L.nvalid), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<float>(ws, L.zg),
         at<int>(ws, L.colread), at<float>(ws, L.M), at<float>(ws, L.Hent), loss_mask, at<float>(ws, L.lz2),
         at<float>(ws, L.logZ), at<float>(ws, L.loss_tok), loss_per_token, gathered_logits, gathered_idx, (int)v0,
-        shard_stats, T, hdr);
+        shard_stats, T, hdr, o.stored_exponentials);
     KDKL_LAUNCHED("combine_kernel");
   }
   if (shard_stats != nullptr) return KDKL_OK;   // the loss is completed by kdkl_forward_finish
   stage_mark(ST_REDUCE, st);
-  loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, tau, H, V, K,
-                                         loss_out, hdr);
+  loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, o.denom_device, tau,
+                                         H, V, K, L.C, o.stored_exponentials ? G_EXPONENTIALS : G_NONE, loss_out, hdr);
   KDKL_LAUNCHED("loss_reduce_kernel");
   return KDKL_OK;
 }
@@ -541,8 +560,9 @@ int kdkl_forward_finish(const float* all_stats, int32_t n_shards, const uint8_t*
                                                                    at<float>(ws, L.lz2), at<float>(ws, L.logZ),
                                                                    at<float>(ws, L.loss_tok), loss_per_token, hdr);
   KDKL_LAUNCHED("shard_finish_kernel");
-  loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, tau, H, V_local, K,
-                                         loss_out, hdr);
+  loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, o.denom_device, tau,
+                                         H, V_local, K, L.C, o.stored_exponentials ? G_EXPONENTIALS : G_NONE, loss_out,
+                                         hdr);
   KDKL_LAUNCHED("loss_reduce_kernel");
   return KDKL_OK;
 }
@@ -564,9 +584,9 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
   const float inv_tau = 1.0f / tau;
 
   stage_mark(ST_COEF, st);
-  bwd_coef_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(at<float>(ws, L.M), loss_mask, T, H, V, K, grad_loss,
-                                                               inv_tau, at<float>(ws, L.coefA),
-                                                               at<float>(ws, L.coefB), hdr);
+  bwd_coef_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(at<float>(ws, L.M), loss_mask, T, H, V, K, L.C, tau,
+                                                               o.stored_exponentials, grad_loss, inv_tau,
+                                                               at<float>(ws, L.coefA), at<float>(ws, L.coefB), hdr);
   KDKL_LAUNCHED("bwd_coef_kernel");
 
   __nv_bfloat16* G = at<__nv_bfloat16>(ws, L.G);
@@ -653,7 +673,7 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
   if ((rc = launch_prep(L, o, ws, topk_idx, topk_val, teacher_lse, loss_mask, T, V, 0, V, K, inv_tau, &live, st)))
     return rc;
   // the divisor of the mean and the per-token gradient coefficients are needed before the first chunk here
-  count_tokens_kernel<<<1, 1024, 0, st>>>(loss_mask, T, o.denom_override, hdr);
+  count_tokens_kernel<<<1, 1024, 0, st>>>(loss_mask, T, o.denom_override, o.denom_device, hdr, nullptr);
   KDKL_LAUNCHED("count_tokens_kernel");
   step_coef_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(at<float>(ws, L.M), loss_mask, T, grad_loss, inv_tau,
                                                                 at<float>(ws, L.coefA), at<float>(ws, L.coefB), hdr);
@@ -685,7 +705,7 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
         at<float>(ws, L.part_m), at<float>(ws, L.part_s), L.Cpad, (int)L.n_tiles_v, (int)rows, s0, K, inv_tau,
         at<int>(ws, L.nvalid), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<float>(ws, L.zg),
         at<int>(ws, L.colread), at<float>(ws, L.M), at<float>(ws, L.Hent), loss_mask, at<float>(ws, L.lz2),
-        at<float>(ws, L.logZ), at<float>(ws, L.loss_tok), loss_per_token, nullptr, nullptr, 0, nullptr, T, hdr);
+        at<float>(ws, L.logZ), at<float>(ws, L.loss_tok), loss_per_token, nullptr, nullptr, 0, nullptr, T, hdr, 1);
     KDKL_LAUNCHED("combine_kernel");
 
     // e -> G in place, now that the chunk's log Z is known
@@ -705,8 +725,8 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
     if ((rc = launch_chunk_outputs(co, tmWmn, tmdW, di, st))) return rc;
   }
   stage_mark(ST_REDUCE, st);
-  loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, tau, H, V, K,
-                                         loss_out, hdr);
+  loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, o.denom_device, tau,
+                                         H, V, K, L.C, G_NONE, loss_out, hdr);
   KDKL_LAUNCHED("loss_reduce_kernel");
   return KDKL_OK;
 }

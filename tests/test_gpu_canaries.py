@@ -1,7 +1,7 @@
 """Out-of-bounds write detection without a sanitizer: guard bytes after every workspace slab and around every
 output buffer are pre-filled with a pattern and must survive a forward + backward (both forms).
 
-KDKL_WS_GUARD_BYTES makes the library leave untouched bytes after each slab of its workspace layout;
+kdkl_debug_guard_bytes makes the library leave untouched bytes after each slab of its workspace layout;
 kdkl_workspace_layout gives the slab table, so everything between a slab's used length and the next slab's start
 can be checked. Outputs are views into one larger buffer with 1 KiB guard zones before and after each.
 """
@@ -37,6 +37,14 @@ class Carver:
         return bool((self.buf[keep] == PATTERN).all())
 
 
+@pytest.fixture
+def guard_bytes():
+    """4 KiB of guard bytes after every workspace slab for the duration of one test."""
+    before = B.kdkl_debug_guard_bytes(4096)
+    yield 4096
+    B.kdkl_debug_guard_bytes(before)
+
+
 @pytest.mark.parametrize("single_pass", [False, True])
 @pytest.mark.parametrize("T,H,V,K,chunk,masked", [
     (300, 72, 1001, 7, 100, True),       # ragged everything, three chunks, dead row tiles
@@ -44,8 +52,7 @@ class Carver:
     (1300, 128, 520, 33, 512, True),     # several chunks, a dead chunk
     (64, 4104, 300, 5, 0, False),        # ragged last k-block
 ])
-def test_no_kernel_writes_outside_its_buffers(monkeypatch, T, H, V, K, chunk, masked, single_pass):
-    monkeypatch.setenv("KDKL_WS_GUARD_BYTES", "4096")
+def test_no_kernel_writes_outside_its_buffers(guard_bytes, T, H, V, K, chunk, masked, single_pass):
     dev = torch.device("cuda:0")
     g = torch.Generator().manual_seed(T + V)
     h = torch.randn(T, H, generator=g).to(torch.bfloat16).to(dev)

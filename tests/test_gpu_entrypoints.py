@@ -101,3 +101,94 @@ def test_profile_single_pass_accounts_for_every_stage_and_changes_nothing():
     assert st["prep"][1] == 1 and st["loss_reduce"][1] == 1 and "bwd_coef" not in st
     assert all(ms > 0 for ms, n in st.values())
     assert torch.equal(op.loss, ref[0]) and torch.equal(op.dhidden, ref[1]) and torch.equal(op.dweight, ref[2])
+
+
+def _random_case(T, H, V, K, seed, dev):
+    g = torch.Generator().manual_seed(seed)
+    h = torch.randn(T, H, generator=g).to(torch.bfloat16).to(dev)
+    W = (torch.randn(V, H, generator=g) / H ** 0.5).to(torch.bfloat16).to(dev)
+    idx = torch.stack([torch.randperm(V, generator=g)[:K] for _ in range(T)]).to(torch.int32).to(dev)
+    val = torch.randn(T, K, generator=g).float().to(dev)
+    return h, W, idx, val
+
+
+def test_count_tokens_and_device_side_divisor():
+    """kdkl_count_tokens counts on the device; a divisor handed over through kdkl_options.denom_device gives bit
+    for bit what the same number gives through denom_override (the data-parallel wrapper relies on this)."""
+    dev = torch.device("cuda:0")
+    T, H, V, K = 700, 72, 1001, 7
+    h, W, idx, val = _random_case(T, H, V, K, 3, dev)
+    mask = (torch.rand(T, generator=torch.Generator().manual_seed(4)) >= 0.3).to(torch.uint8).to(dev)
+    n = torch.full((1,), -1.0, dtype=torch.float64, device=dev)
+    B.kdkl_count_tokens(mask, T, n)
+    assert n.item() == float(mask.sum().item())
+    B.kdkl_count_tokens(None, T, n)
+    assert n.item() == float(T)
+    n.fill_(1234.0)
+    for single_pass in (False, True):
+        a = B.FusedChunkedKL(T, H, V, K, chunk=256, device=dev, opt=B.make_options(denom_override=1234.0))
+        b = B.FusedChunkedKL(T, H, V, K, chunk=256, device=dev, opt=B.make_options(denom_device=n))
+        for op in (a, b):
+            if single_pass:
+                op.forward_backward(h, W, idx, val, loss_mask=mask)
+            else:
+                op.forward(h, W, idx, val, loss_mask=mask)
+                op.backward(h, W, loss_mask=mask)
+            assert op.status()[0] == 0
+        assert torch.equal(a.loss, b.loss) and torch.equal(a.dhidden, b.dhidden) and torch.equal(a.dweight, b.dweight)
+
+
+def test_backward_refuses_a_state_it_cannot_use():
+    """Device-side state check of kdkl_backward: another temperature or chunk size than the forward call's, and a
+    second backward on stored exponentials (the in-place conversion can run once). Reported as KDKL_ERR_STATE,
+    outputs untouched."""
+    dev = torch.device("cuda:0")
+    T, H, V, K = 300, 72, 1001, 7
+    h, W, idx, val = _random_case(T, H, V, K, 5, dev)
+    op = B.FusedChunkedKL(T, H, V, K, chunk=128, temperature=1.0, device=dev)
+    op.forward(h, W, idx, val)
+    op.dhidden.fill_(7.0); op.dweight.fill_(7.0)
+    B.kdkl_backward(h, W, K, op.workspace, op.dhidden, op.dweight, chunk=128, temperature=1.5)
+    assert op.status()[0] == -9
+    assert (op.dhidden.float() == 7.0).all() and (op.dweight == 7.0).all()
+    op.forward(h, W, idx, val)
+    B.kdkl_backward(h, W, K, op.workspace, op.dhidden, op.dweight, chunk=64, temperature=1.0)
+    assert op.status()[0] == -9
+    assert (op.dhidden.float() == 7.0).all() and (op.dweight == 7.0).all()
+    op.forward(h, W, idx, val)
+    op.backward(h, W)                                         # the matching call goes through
+    assert op.status()[0] == 0 and torch.isfinite(op.dweight).all()
+
+    st = B.FusedChunkedKL(T, H, V, K, chunk=0, device=dev, opt=B.make_options(stored_exponentials=1))
+    st.forward(h, W, idx, val)
+    st.backward(h, W)
+    assert st.status()[0] == 0
+    first = (st.dhidden.clone(), st.dweight.clone())
+    assert torch.allclose(first[1], op.dweight, rtol=0, atol=2e-2 * op.dweight.abs().max().item())
+    st.dhidden.fill_(7.0); st.dweight.fill_(7.0)
+    st.backward(h, W)                                         # the exponentials are gone: refused
+    assert st.status()[0] == -9
+    assert (st.dhidden.float() == 7.0).all() and (st.dweight == 7.0).all()
+    # a forward without the option followed by a backward with it is refused as well
+    plain = B.FusedChunkedKL(T, H, V, K, chunk=0, device=dev)
+    plain.forward(h, W, idx, val)
+    plain.dweight.fill_(7.0)
+    B.kdkl_backward(h, W, K, plain.workspace, plain.dhidden, plain.dweight, opt=B.make_options(stored_exponentials=1))
+    assert plain.status()[0] == -9 and (plain.dweight == 7.0).all()
+
+
+def test_stored_exponentials_report_rows_below_their_range():
+    """Every logit of a row at -64: the fixed-bias bf16 exponentials of the single-pass step would flush to zero
+    there. The single-pass call says so (KDKL_ERR_RANGE); the two-call path has no such limit."""
+    dev = torch.device("cuda:0")
+    T, H, V, K = 40, 64, 600, 4
+    h = torch.ones(T, H, dtype=torch.bfloat16, device=dev)
+    W = -torch.ones(V, H, dtype=torch.bfloat16, device=dev)
+    idx = torch.arange(K, dtype=torch.int32, device=dev).repeat(T, 1).contiguous()
+    val = torch.zeros(T, K, device=dev)
+    op = B.FusedChunkedKL(T, H, V, K, device=dev)
+    op.forward(h, W, idx, val)
+    op.backward(h, W)
+    assert op.status()[0] == 0 and torch.isfinite(op.dweight).all()
+    op.forward_backward(h, W, idx, val)
+    assert op.status()[0] == -13

@@ -99,17 +99,26 @@ def test_token_shards_match_oracle(single_pass):
     dev = torch.device("cuda:0")
     gd = {k: v.to(dev) for k, v in d.items()}
     bounds = [0, 77, 200, T]
-    n_global = float(d["mask"].sum().item())
-    ranks = []
+    # the ranks run one after the other here, so the "all-reduce" of the count is a running sum over a first
+    # pass of the library's count kernel; each rank then reads the global divisor from the device
+    ops, counts = [], []
     for r in range(3):
         a, b = bounds[r], bounds[r + 1]
         op = B.TokenShardedFusedKL(b - a, H, V, K, chunk=64, temperature=tau, device=dev, all_reduce_sum=lambda t: t)
+        counts.append(op.count_tokens(gd["mask"][a:b].contiguous()).clone())
+        ops.append(op)
+    n_global = torch.stack(counts).sum(0)
+    assert n_global.item() == float(d["mask"].sum().item())
+    ranks = []
+    for r in range(3):
+        a, b = bounds[r], bounds[r + 1]
+        op = ops[r]
+        op.n_global.copy_(n_global)
         sl = {k: (v[a:b].contiguous() if k != "weight" else v) for k, v in gd.items()}
         if single_pass:
-            op.forward_backward_local(sl["hidden"], sl["weight"], sl["topk_idx"], sl["topk_val"], n_global,
-                                      loss_mask=sl["mask"])
+            op.forward_backward_local(sl["hidden"], sl["weight"], sl["topk_idx"], sl["topk_val"], loss_mask=sl["mask"])
         else:
-            op.forward_local(sl["hidden"], sl["weight"], sl["topk_idx"], sl["topk_val"], n_global, loss_mask=sl["mask"])
+            op.forward_local(sl["hidden"], sl["weight"], sl["topk_idx"], sl["topk_val"], loss_mask=sl["mask"])
             op.backward_local(sl["hidden"], sl["weight"], loss_mask=sl["mask"])
         assert op.status()[0] == 0
         ranks.append(op)

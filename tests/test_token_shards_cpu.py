@@ -1,8 +1,9 @@
 """Host-side logic of the token-sharded (data-parallel) wrapper under real collectives: two gloo ranks on CPU.
 
 The CUDA entry points are replaced inside each worker by torch float64 stand-ins with the same argument contract,
-so the test exercises what the wrapper adds: the count of counted tokens summed over ranks before forward (the
-divisor of the mean), the sum of the partial losses, and the sum of dweight; for the two-call form and for the
+so the test exercises what the wrapper adds: the count of counted tokens (the library's count call) summed over
+ranks before forward and handed to the kernels as a device-side divisor, the sum of the partial losses, and the
+sum of dweight; for the two-call form and for the
 single-pass form. Uneven token slices, a mask on one rank only. Compared with the dense oracle over all tokens.
 """
 import os
@@ -35,7 +36,7 @@ def _install_stand_ins(B, state):
 
     def fwd(hidden, weight, idx, val, ws, loss_out, *, teacher_lse=None, loss_mask=None, chunk=0, temperature=1.0,
             opt=None, loss_per_token=None, gathered_logits=None, gathered_idx=None):
-        loss, G = _loss_and_G(hidden, weight, idx, val, loss_mask, temperature, opt.denom_override)
+        loss, G = _loss_and_G(hidden, weight, idx, val, loss_mask, temperature, float(opt.denom_device.item()))
         loss_out[0] = loss.float()
         state["G"] = G
 
@@ -49,7 +50,15 @@ def _install_stand_ins(B, state):
         fwd(hidden, weight, idx, val, ws, loss_out, loss_mask=loss_mask, temperature=temperature, opt=opt)
         bwd(hidden, weight, idx.shape[1], ws, dh, dw, grad_loss=grad_loss)
 
+    def count(mask, T, out):
+        out[0] = float(T if mask is None else int((mask != 0).sum()))
+
+    def options(**kw):                                      # the wrapper passes the divisor as a tensor to read later
+        import types
+        return types.SimpleNamespace(**kw)
+
     B.kdkl_workspace_bytes, B.kdkl_forward, B.kdkl_backward, B.kdkl_forward_backward = ws_bytes, fwd, bwd, fwd_bwd
+    B.kdkl_count_tokens, B.make_options = count, options
 
 
 def _worker(rank, world, port, out, single_pass):
