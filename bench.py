@@ -49,7 +49,9 @@ FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_g
 # device; profiles/dram_traffic_pair_build_C4096_V32768.md). A launch's traffic is proportional to the vocabulary
 # rows it sweeps, so the figure for another V at this chunk and H is scaled by V / 32768. The dW figure is the
 # reduce-add form (every chunk after the first).
-TRAFFIC_REF = {"chunk": 4096, "H": 4096, "V": 32768, "bytes": {}}
+TRAFFIC_REF = {"chunk": 4096, "H": 4096, "V": 32768,
+               "bytes": {"fwd_gemm_lse": 306605312 + 9421568, "bwd_gemm_dlogits": 377513472 + 247802880,
+                         "dhidden_gemm": 1392504320 + 116503808, "dweight_gemm": 975120384 + 496788736}}
 
 SWEEP_FUSED = [("c2", 10), ("c3", 5), ("c4a", 4), ("c4b", 3), ("c4c", 3), ("c5", 5)]
 SWEEP_DENSE = [("c2", 3), ("c3", 3), ("c4a", 2)]
