@@ -394,8 +394,11 @@ def run_context_sweep(args, peaks) -> dict:
     sust = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
     rows = []
     plan = [("fused", SWEEP_FUSED), ("dense", SWEEP_DENSE), ("fwdchunk", SWEEP_FWDCHUNK)]
-    if args.sweep_methods:
-        plan = [(m, s) for m, s in plan if m in args.sweep_methods.split(",")]
+    if args.sweep_plan:                               # e.g. "fused=c2:5,c3:3;dense=c2:2"
+        plan = []
+        for part in args.sweep_plan.split(";"):
+            method, sizes = part.split("=")
+            plan.append((method, [(x.split(":")[0], int(x.split(":")[1])) for x in sizes.split(",")]))
     t_start = time.time()
     for method, sizes in plan:
         for name, steps in sizes:
@@ -442,12 +445,14 @@ def main():
     ap.add_argument("--parallel", default="", choices=["", "independent", "tokens", "vocab"],
                     help="how N > 1 ranks share the work (default: tokens)")
     ap.add_argument("--ref-rows", type=int, default=0,
-                    help="tokens in the CPU-oracle sample (0: 768 for the cpu_baseline leg, 128 per reference step)")
+                    help="tokens in the CPU-oracle sample (0: 2048 for the cpu_baseline leg, 128 per reference step)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the context sweep (child processes)")
-    ap.add_argument("--sweep-methods", default="", help="comma list out of fused,dense,fwdchunk (default: all)")
+    ap.add_argument("--sweep-plan", default="",
+                    help='which sizes the context sweep runs, "method=workload:steps,...;method=..." with method out '
+                         'of fused, dense, fwdchunk (default: the benchmark sizes 4K ... 256K)')
     ap.add_argument("--sweep-timeout", type=int, default=240)
     ap.add_argument("--sweep-worker", default="", help=argparse.SUPPRESS)
     ap.add_argument("--capture", action="store_true",
@@ -703,9 +708,10 @@ def main():
 
     cpu_baseline = None
     if not args.no_cpu_baseline and not args.capture and world == 1:
-        tps, threads, dt = oracle_sample(cfg, oracle_data(cfg, args.ref_rows or 768, d))
+        n_cpu = args.ref_rows or 2048
+        tps, threads, dt = oracle_sample(cfg, oracle_data(cfg, n_cpu, d))
         cpu_baseline = {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle",
-                        "sample": f"{args.ref_rows or 768} tokens of {cfg.name}, forward + gradients, dense fp64, {dt:.1f} s"}
+                        "sample": f"{min(n_cpu, T)} tokens of {cfg.name}, forward + gradients, dense fp64, {dt:.1f} s"}
 
     tokens_per_s = run["tokens_per_step"] / (ms_step * 1e-3)
     step_flops = 8.0 * run["tokens_per_step"] * H * V / world        # per GPU

@@ -21,7 +21,7 @@ def _run(*extra):
 
 
 def test_gpu_arm_line():
-    d = _run("--ref-rows", "64")
+    d = _run("--ref-rows", "64", "--sweep-plan", "fused=c1:3;dense=c1:2;fwdchunk=c1:2")
     assert d["unit"] == "tokens/s" and d["higher_is_better"] is True and d["scaling"] == "weak"
     assert d["n_gpus"] == 1 and d["steps"] == 3 and d["warmup"] >= 3
     assert d["value"] > 0 and d["ms_per_step"] > 0 and d["ms_per_step_min"] <= d["ms_per_step_median"]
@@ -44,6 +44,15 @@ def test_gpu_arm_line():
     f = d["feature_loss"]
     assert 0 < f["mse"]["frac_of_hbm_copy"] < 1.3 and 0 < f["cosine"]["frac_of_hbm_copy"] < 1.3
     assert set(d["stages"]) >= {"fwd_gemm_lse", "bwd_gemm_dlogits", "dhidden_gemm", "dweight_gemm"}
+    assert d["stage_clocks"]["sm_mhz"] > 0 and d["stage_check"]["sum_of_stage_ms"] > 0
+    assert all(v["ms_x_mhz_per_launch"] > 0 for k, v in d["stages"].items() if v["launches_per_step"])
+    rows = d["context_sweep"]["rows"]
+    assert [r["method"] for r in rows] == ["fused", "dense", "fwdchunk"]
+    for r in rows:                                           # measured, in a process of its own, same loss
+        assert r["ms_per_iter"] > 0 and r["peak_gb"] > 0 and r["driver_delta_gb"] >= 0 and r["steps"] >= 2
+        assert abs(r["loss"] - d["loss"]) <= 1e-3 * abs(d["loss"])
+    assert rows[0]["status"] == 0 and 0 < rows[0]["frac_of_bf16_burst_peak"] < 1.2
+    assert d["collective"] is None and d["config"]["parallelism"].startswith("independent")
 
 
 def test_reference_arm_line():
