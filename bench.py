@@ -205,6 +205,19 @@ def workload_name(cfg):
             f"bf16 hidden/weight, top-K teacher ({cfg.idx_dist} indices)")
 
 
+def resolve_config(name: str):
+    """A named config, or one at another chunk size ("c3@8192"), or the 4K shape at another length ("T8192")."""
+    from paper_2608_03796_b200 import inputs as I
+    if "@" in name:
+        base, chunk = name.split("@")
+        return dataclasses.replace(resolve_config(base), name=name, chunk=int(chunk))
+    if name in I.CONFIGS:
+        return I.CONFIGS[name]
+    if name.startswith("T") and name[1:].isdigit():
+        return dataclasses.replace(I.CONFIGS["c2"], name=name, T=int(name[1:]))
+    raise SystemExit(f"unknown workload {name}")
+
+
 def shard_bounds(n: int, world: int, rank: int):
     """Contiguous near-even split of n items: [a, b) of this rank."""
     base, extra = divmod(n, world)
@@ -234,6 +247,8 @@ def mode_tokens(cfg, rank, world, dev, B, I, all_reduce_sum=None):
     gcfg = dataclasses.replace(cfg, T=cfg.T * world)
     rows = torch.arange(rank * cfg.T, (rank + 1) * cfg.T, dtype=torch.int64)
     d = I.make_inputs(gcfg, device=dev, rows=rows)
+    if all_reduce_sum is None and world == 1:
+        all_reduce_sum = lambda t: t                    # one rank: every sum over ranks is the value itself
     kw = {} if all_reduce_sum is None else {"all_reduce_sum": all_reduce_sum}
     op = B.TokenShardedFusedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev, **kw)
     cuda = torch.device(dev).type == "cuda"
@@ -286,6 +301,9 @@ def mode_vocab(cfg, rank, world, dev, B, I, all_gather=None, all_reduce_sum=None
     """The paper's tensor-parallel setting: rank r holds vocabulary rows [v0, v1) and every token."""
     import torch
     v0, v1 = shard_bounds(cfg.V, world, rank)
+    if world == 1:                                      # one rank: its statistics are the gathered ones
+        all_gather = all_gather or (lambda out, local: out.copy_(local.view(out.shape)))
+        all_reduce_sum = all_reduce_sum or (lambda t: t)
     d = I.make_inputs(cfg, device=dev)
     d["weight"] = d["weight"][v0:v1].contiguous()
     op = B.ShardedFusedChunkedKL(cfg.T, cfg.H, v1 - v0, v0, cfg.V, cfg.K, world, chunk=cfg.chunk,
@@ -326,12 +344,14 @@ MODES = {"independent": mode_independent, "tokens": mode_tokens, "vocab": mode_v
 
 # ------------------------------------------------------------------------------------------ context sweep
 def sweep_worker(method: str, name: str, steps: int) -> dict:
-    """One method at one size in this (fresh) process: iteration time, measured peak memory, loss."""
+    """One method at one size in this (fresh) process: iteration time, measured peak memory, loss. Methods: fused
+    (the two calls), single (the single-pass call), dense / fwdchunk (the comparison losses), teacher /
+    teacher_stored (the teacher cache kernel, whose "loss" column is the first token's log-sum-exp)."""
     import torch
     from paper_2608_03796_b200 import binding as B
     from paper_2608_03796_b200 import comparators as C
     from paper_2608_03796_b200 import inputs as I
-    cfg = I.CONFIGS[name]
+    cfg = resolve_config(name)
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
     torch.zeros(1, device=dev)                      # context up before the driver's free-memory reading
@@ -343,7 +363,24 @@ def sweep_worker(method: str, name: str, steps: int) -> dict:
     out = {"method": method, "workload": name, "T": cfg.T, "H": cfg.H, "V": cfg.V, "K": cfg.K, "chunk": cfg.chunk,
            "steps": steps, "input_gb": torch.cuda.memory_allocated() / 1e9}
     op = None
-    if method == "fused":
+    if method in ("teacher", "teacher_stored"):
+        # the teacher cache kernel on the same shape: hidden / weight play the teacher's role
+        stored = method == "teacher_stored"
+        _, _, _, tws = B.kdkl_teacher_topk(d["hidden"], d["weight"], cfg.K, temperature=cfg.tau, stored=stored)
+        out["workspace_gb"] = tws.numel() / 1e9
+        out["flops_per_iter"] = (0.25 if stored else 0.5) * cfg.flops      # one or two projections
+
+        def step():
+            return B.kdkl_teacher_topk(d["hidden"], d["weight"], cfg.K, temperature=cfg.tau, workspace=tws,
+                                       stored=stored)[2][:1]
+    elif method == "single":
+        op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev)
+        out["workspace_gb"] = op.workspace.numel() / 1e9
+
+        def step():
+            op.forward_backward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], loss_mask=d["mask"])
+            return op.loss
+    elif method == "fused":
         op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev)
         out["workspace_gb"] = op.workspace.numel() / 1e9
 
@@ -372,7 +409,9 @@ def sweep_worker(method: str, name: str, steps: int) -> dict:
                    clock_reasons=clk.summary()["reasons"])
         if op is not None:
             out["status"] = op.status()[0]
-            out["tflops"] = cfg.flops / (ms * 1e-3) / 1e12
+            out["tflops"] = (0.75 if method == "single" else 1.0) * cfg.flops / (ms * 1e-3) / 1e12
+        elif "flops_per_iter" in out:
+            out["tflops"] = out["flops_per_iter"] / (ms * 1e-3) / 1e12
     except torch.OutOfMemoryError:
         out.update(oom=True, peak_gb=torch.cuda.max_memory_allocated() / 1e9)
     return out
@@ -460,7 +499,7 @@ def main():
     args = ap.parse_args()
 
     from paper_2608_03796_b200 import inputs as I
-    cfg = I.CONFIGS[args.workload]
+    cfg = resolve_config(args.workload)
     if args.impl == "reference":
         run_reference(args, cfg)
         return

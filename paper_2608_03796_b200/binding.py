@@ -13,7 +13,7 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("KDKL_LIB_PATH", os.path.join(_HERE, "libkdkl.so"))
+LIB_PATH = os.path.join(_HERE, "libkdkl.so")
 
 KDKL_OK = 0
 ERRORS = {

@@ -111,10 +111,7 @@ static int make_tmap_out_bf16(CUtensorMap* m, void* base, uint64_t cols, uint64_
 
 // ------------------------------------------------------------------ device / launch helpers
 // All GEMMs of the loss run as CTA pairs (256 x 256 tile per pair, see GemmCfg).
-#ifndef KDKL_NCTA
-#define KDKL_NCTA 2
-#endif
-constexpr int kNCTA = KDKL_NCTA;
+constexpr int kNCTA = 2;
 constexpr int kTileM = GemmCfg<kNCTA>::TILE_M;
 constexpr int kBRows = GemmCfg<kNCTA>::B_ROWS;
 // What the library has learnt about each device, asked once per device and process (a benign race: two

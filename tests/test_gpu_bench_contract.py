@@ -61,3 +61,15 @@ def test_reference_arm_line():
     assert d["dtype"] == "f64" and d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] == d["value"]
     assert d["e2e"]["value"] == d["value"] and d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0
     assert "workload" in d["config"]
+
+
+def test_sharded_modes_on_one_rank_give_the_same_loss():
+    """--parallel tokens / vocab with a single rank: the same batch through the data-parallel and the
+    tensor-parallel call sequences (count kernel + device-side divisor; shard statistics + finish) must give the
+    loss of the plain two calls, and the line must say what crosses ranks per step."""
+    base = _run("--no-sweep", "--no-e2e", "--no-cpu-baseline")
+    for mode, scaling in (("tokens", "weak"), ("vocab", "strong")):
+        d = _run("--no-sweep", "--no-e2e", "--no-cpu-baseline", "--parallel", mode)
+        assert abs(d["loss"] - base["loss"]) <= 1e-6 * abs(base["loss"])
+        assert d["scaling"] == scaling and d["collective"]["bytes_per_step"] > 0 and d["gpu_launches"] > 0
+        assert d["value"] > 0 and d["roofline"] is None and d["stages"] is None
