@@ -582,7 +582,7 @@ def main():
 
     single_pass = stages = stage_clocks = e2e = e2e_record = feature = None
     dom = dom_tflops = traffic = None
-    flops_per_launch = 2.0 * min(cfg.chunk, T) * H * (V if mode_name != "vocab" else op.V_local)
+    gemm_flops_per_step = 2.0 * T * H * V            # each of the four GEMM kinds: 2*T*H*V per step
     long_step = ms_total > 1000.0
     peak_key = "bf16_tflops_sustained" if long_step else "bf16_tflops"
     peak = float(peaks.get(peak_key, FALLBACK_PEAKS[peak_key]))
@@ -609,12 +609,14 @@ def main():
                       "ms_x_mhz_per_launch": ((v[0] / v[1]) * smhz if (v[1] and smhz) else None)}
                   for k, v in stage_acc.items()}
         for k in gemm_stages:
-            stages[k]["tflops"] = flops_per_launch / (stages[k]["ms_per_launch"] * 1e-3) / 1e12
+            stages[k]["tflops"] = gemm_flops_per_step / (stages[k]["ms_per_step"] * 1e-3) / 1e12
         dom = max(gemm_stages, key=lambda k: stages[k]["ms_per_step"])
         dom_tflops = stages[dom]["tflops"]
+        flops_per_launch = gemm_flops_per_step / stages[dom]["launches_per_step"]
         ref = TRAFFIC_REF
         if (min(cfg.chunk, T), H) == (ref["chunk"], ref["H"]) and dom in ref["bytes"]:
-            traffic = int(ref["bytes"][dom] * V / ref["V"])
+            # per chunk of tokens in the capture; a launch that covers several chunks moves that many times as much
+            traffic = int(ref["bytes"][dom] * V / ref["V"] * (T / cfg.chunk) / stages[dom]["launches_per_step"])
         stage_sum = sum(v["ms_per_step"] for v in stages.values())
         stage_check = {"sum_of_stage_ms": stage_sum, "ms_per_step": ms_step, "sm_mhz_stage_run": smhz,
                        "sm_mhz_timed_region": clocks["sm_mhz"],

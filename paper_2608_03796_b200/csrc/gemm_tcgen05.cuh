@@ -7,7 +7,9 @@
 //               a time); two TMEM accumulator stages let tile i's epilogue overlap tile
 //               i+1's MMAs
 //
-// One CTA per SM; tiles of 128 x 256 per CTA (256 x 256 per CTA pair, see GemmCfg), k-blocks of 64.
+// One CTA per SM; tiles of 128 x 256 per CTA (256 x 256 per CTA pair, see GemmCfg), k-blocks of 64. WIDE tiles
+// (256 x 512 per pair) use both TMEM halves as one accumulator: a quarter less operand traffic per flop, no
+// overlap of a tile's epilogue with the next tile's MMAs (for the two output GEMMs, whose epilogues are short).
 // Either operand may be K-major (its rows are contiguous along K) or MN-major (stored
 // [K, M] / [K, N], contiguous along M / N); the difference is confined to the TMA boxes
 // and the shared-memory descriptors.
@@ -46,10 +48,18 @@ constexpr int STAGING_BYTES = 4 * STAGING_WARP_BYTES;
 // shares one 256 x 256 tile: each CTA stages its 128 rows of A and its 128 rows of B, the leader
 // issues one MMA for both, and each CTA keeps the 128 x 256 half of D in its own TMEM. A pair
 // moves a third less operand data per flop through shared memory and L2.
-template <int NCTA>
+// WIDE: the tile is 512 columns wide - two 256-column halves, each fed by its own MMA per K = 16 slice from the same
+// A operand, together filling all 512 TMEM columns. Per flop a quarter less operand data comes through L2 and
+// shared memory than with two 256 x 256 tiles, which is what the two output GEMMs need: dH = G W streams both
+// operands from HBM once per wave of tiles (half the waves now), and in dW += G^T h every stored byte takes
+// load bandwidth from the SM's memory port. The price: one accumulator stage, so the epilogue does not overlap
+// the next tile's MMAs - acceptable where a tile's contraction is long next to its epilogue.
+template <int NCTA, bool WIDE = false>
 struct GemmCfg {
   static constexpr int TILE_M = BM * NCTA;
-  static constexpr int B_ROWS = BN / NCTA;               // rows of B each CTA stages
+  static constexpr int N_HALVES = WIDE ? 2 : 1;
+  static constexpr int TILE_N = BN * N_HALVES;
+  static constexpr int B_ROWS = TILE_N / NCTA;           // rows of B each CTA stages (HALF_ROWS per accumulator half)
   static constexpr int A_STAGE_BYTES = BM * BK * 2;      // 16 KiB
   static constexpr int B_STAGE_BYTES = B_ROWS * BK * 2;  // 32 / 16 KiB
   static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
@@ -66,7 +76,7 @@ constexpr float kExpBias = 64.f;
 
 struct GemmParams {
   int M, N, K;               // valid extents of this launch
-  int m_tiles, n_tiles;
+  int m_tiles, n_tiles;      // tiles of TILE_M rows and of TILE_N columns (256, or 512 for the WIDE instantiation)
   int m_inner;               // 1: consecutive tile ids walk M first (B panel shared), 0: N first
   int k_splits;              // >= 1: each tile's contraction is cut into this many work units, each
                              // writing its own partial output (split s goes to output rows + s * split_rows)
@@ -137,13 +147,15 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 __device__ __forceinline__ int kblocks_all(int K) { return (K + BK - 1) / BK; }
 
-template <int EPI, bool A_MN, bool B_MN, int NCTA>
+template <int EPI, bool A_MN, bool B_MN, int NCTA, bool WIDE = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
-  using Cfg = GemmCfg<NCTA>;
+  using Cfg = GemmCfg<NCTA, WIDE>;
   constexpr int STAGES = Cfg::STAGES, STAGE_BYTES = Cfg::STAGE_BYTES, A_STAGE_BYTES = Cfg::A_STAGE_BYTES;
-  constexpr int TILE_M = Cfg::TILE_M, B_ROWS = Cfg::B_ROWS;
+  constexpr int TILE_M = Cfg::TILE_M, B_ROWS = Cfg::B_ROWS, TILE_N = Cfg::TILE_N, N_HALVES = Cfg::N_HALVES;
+  constexpr int HALF_ROWS = B_ROWS / N_HALVES;            // rows of B this CTA stages per accumulator half
+  constexpr uint32_t HALF_BYTES = HALF_ROWS * BK * 2;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -261,7 +273,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         unit_decode(unit, tile, split, kb0, kb1);
         tile_coords(tile, mt, nt);
         const int m0 = mt * TILE_M + (int)cta_rank * BM;      // this CTA's rows of A
-        const int n0 = nt * BN + (int)cta_rank * B_ROWS;      // this CTA's rows of B
+        const int n0 = nt * TILE_N + (int)cta_rank * HALF_ROWS;   // this CTA's rows of B (of the first half)
         const int nkb = kskip ? *n_live_kb : kb1 - kb0;
         for (int i = 0; i < nkb; ++i, ++it) {
           const int kb = kskip ? (int)live_kb[i] : kb0 + i;
@@ -282,11 +294,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
             for (int i = 0; i < BM / 64; ++i) load(sa + i * (BK * 128), &tmA, m0 + 64 * i, k0, fb);
           }
-          if (!B_MN) {
-            load(sb, &tmB, k0, n0, fb);
-          } else {
 #pragma unroll
-            for (int i = 0; i < B_ROWS / 64; ++i) load(sb + i * (BK * 128), &tmB, n0 + 64 * i, k0, fb);
+          for (int hf = 0; hf < N_HALVES; ++hf) {         // half hf of the tile: columns [nt * TILE_N + hf * BN, + BN)
+            const uint32_t sbh = sb + hf * HALF_BYTES;
+            const int nh = n0 + hf * BN;
+            if (!B_MN) {
+              load(sbh, &tmB, k0, nh, fb);
+            } else {
+#pragma unroll
+              for (int i = 0; i < HALF_ROWS / 64; ++i) load(sbh + i * (BK * 128), &tmB, nh + 64 * i, k0, fb);
+            }
           }
           issued |= 1u << s;
           last_par = (last_par & ~(1u << s)) | (ph << s);
@@ -333,8 +350,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int tile, split, kb0, kb1, mt, nt;
         unit_decode(unit, tile, split, kb0, kb1);
         tile_coords(tile, mt, nt);
-        const uint32_t acc = lt & 1u;
-        const uint32_t aph = (lt >> 1) & 1u;
+        const uint32_t acc = WIDE ? 0u : (lt & 1u);       // WIDE: one accumulator stage (all 512 columns)
+        const uint32_t aph = WIDE ? (lt & 1u) : ((lt >> 1) & 1u);
         if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + acc * BN;
@@ -348,7 +365,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const uint32_t alo = a_lo0 + s * STAGE_STEP, blo = b_lo0 + s * STAGE_STEP;
 #pragma unroll
           for (int j = 0; j < BK / UMMA_K; ++j) {
-            mma(tmem_d, desc(alo + j * A_STEP, a_hi), desc(blo + j * B_STEP, b_hi), accf);
+#pragma unroll
+            for (int hf = 0; hf < N_HALVES; ++hf)
+              mma(tmem_d + hf * BN, desc(alo + j * A_STEP, a_hi), desc(blo + hf * (HALF_BYTES >> 4) + j * B_STEP, b_hi),
+                  accf);
             accf = 1u;
           }
           commit(empty_bar(s));                // frees the stage (in both CTAs) when these MMAs have read it
@@ -377,10 +397,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int split = zu / (n_dead * p.n_tiles);
         const int rem = zu - split * (n_dead * p.n_tiles);
         const int mt = live_m[m_count + rem / p.n_tiles], nt = rem % p.n_tiles;
-        const int r0 = mt * TILE_M + (int)cta_rank * BM + lg * 32, n0 = nt * BN;
+        const int r0 = mt * TILE_M + (int)cta_rank * BM + lg * 32, n0 = nt * TILE_N;
         if (r0 >= p.M) continue;
         // zero boxes through the same staging / bulk-group protocol as the regular output path
-        for (int c0 = n0; c0 < n0 + BN && c0 < p.N; c0 += BOX_COLS) {
+        for (int c0 = n0; c0 < n0 + TILE_N && c0 < p.N; c0 += BOX_COLS) {
           const uint32_t sbox = staging0 + (warp - 2) * STAGING_WARP_BYTES + (nbox & 1u) * 4096u;
           if (lane == 0) bulk_wait_read<1>();
           __syncwarp();
@@ -400,11 +420,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       int tile, split, kb0, kb1, mt, nt;
       unit_decode(unit, tile, split, kb0, kb1);
       tile_coords(tile, mt, nt);
-      const int m0 = mt * TILE_M + (int)cta_rank * BM, n0 = nt * BN;   // this CTA's 128 x 256 part of D
+      const int m0 = mt * TILE_M + (int)cta_rank * BM, n0 = nt * TILE_N;   // this CTA's 128 x TILE_N part of D
       const int row = m0 + row_in_tile;
       const bool row_ok = row < p.M;
-      const uint32_t acc = lt & 1u;
-      const uint32_t aph = (lt >> 1) & 1u;
+      const uint32_t acc = WIDE ? 0u : (lt & 1u);
+      const uint32_t aph = WIDE ? (lt & 1u) : ((lt >> 1) & 1u);
 
       // per-row state that does not need the accumulator: fetched before the wait
       int cur = 0, nv = 0, next_idx = 0x7fffffff;
@@ -435,7 +455,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int box_row0 = m0 + lg * 32;       // first output row of this warp's boxes
       const bool box_ok = box_row0 < p.M;      // warp-uniform
 #pragma unroll 1
-      for (int w = 0; w < BN / 32; ++w) {
+      for (int w = 0; w < TILE_N / 32; ++w) {
         const int col0 = n0 + w * 32;
         // uniform: whole window past the edge. bf16 outputs are staged as pairs of windows
         // (64 columns = one 128-byte row), so a pair is always completed.

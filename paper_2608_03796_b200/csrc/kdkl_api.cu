@@ -113,7 +113,13 @@ static int make_tmap_out_bf16(CUtensorMap* m, void* base, uint64_t cols, uint64_
 // All GEMMs of the loss run as CTA pairs (256 x 256 tile per pair, see GemmCfg).
 constexpr int kNCTA = 2;
 constexpr int kTileM = GemmCfg<kNCTA>::TILE_M;
-constexpr int kBRows = GemmCfg<kNCTA>::B_ROWS;
+constexpr int kBRows = GemmCfg<kNCTA>::B_ROWS;             // rows of a K-major B box (also per half of a WIDE tile)
+constexpr int kWideN = GemmCfg<kNCTA, true>::TILE_N;
+static_assert(GemmCfg<kNCTA, true>::B_ROWS / 2 == kBRows, "a WIDE tile's halves take the narrow tile's B boxes");
+// The two output GEMMs (N = H) use WIDE tiles when rounding H up to whole 512-column tiles wastes at most a
+// tenth of the tensor work (H = 4096, 3072, 1024, 1000 ...); narrow 256-column tiles otherwise.
+static bool use_wide(long long N) { return ((N + kWideN - 1) / kWideN) * kWideN * 10 <= N * 11; }
+static long long n_tiles_for(long long N, bool wide) { return wide ? (N + kWideN - 1) / kWideN : (N + BN - 1) / BN; }
 // What the library has learnt about each device, asked once per device and process (a benign race: two
 // threads asking at the same time store the same values).
 constexpr int kMaxDevices = 64;
@@ -146,11 +152,12 @@ static int sm_count_or_default() {
   return di.sm_count;
 }
 
-template <int EPI, bool A_MN, bool B_MN>
+template <int EPI, bool A_MN, bool B_MN, bool WIDE = false>
 static int launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const GemmParams& p,
                        const DeviceInfo& di, cudaStream_t st) {
-  auto kern = gemm_tcgen05_kernel<EPI, A_MN, B_MN, kNCTA>;
-  constexpr int smem = GemmCfg<kNCTA>::SMEM_BYTES;
+  auto kern = gemm_tcgen05_kernel<EPI, A_MN, B_MN, kNCTA, WIDE>;
+  constexpr int smem = GemmCfg<kNCTA, WIDE>::SMEM_BYTES;
+  static_assert(smem <= 227 * 1024, "shared memory per CTA");
   // The shared-memory limit belongs to the current device's copy of this instantiation: set once per device
   // (a process may drive several), not per launch.
   static bool attr_set[kMaxDevices];
@@ -206,6 +213,8 @@ static int choose_k_splits(long long tiles, long long kblocks, int sm_count) {
 struct WsLayout {
   long long C, Cpad, Vpad, n_tiles_v;
   int dh_splits;             // split-K factor of the dH GEMM at full chunks
+  int dw_group;              // chunks whose G is kept so that one dW pass contracts over all of them (1 or 2)
+  long long g_rows;          // rows of the G buffer
   size_t hdr, idx_sorted, p_sorted, perm, zg, colread, nvalid, M, Hent, lz2, logZ, loss_tok, coefA, coefB;
   size_t part_m, part_s, G, dh_part, live, total;
   static constexpr int kMaxSlabs = 24;
@@ -252,8 +261,14 @@ static WsLayout ws_layout(long long T, long long H, long long V, int K, long lon
   L.coefB = take((size_t)T * 4);
   L.part_m = take((size_t)L.n_tiles_v * L.Cpad * 4);
   L.part_s = take((size_t)L.n_tiles_v * L.Cpad * 4);
-  L.G = take((size_t)L.Cpad * L.Vpad * 2);
-  L.dh_splits = choose_k_splits(((L.C + kTileM - 1) / kTileM) * ((H + BN - 1) / BN), (V + BK - 1) / BK,
+  // dW += G^T h is read-modify-write of the whole fp32 dW per pass, and every byte a GEMM stores costs its SM
+  // load bandwidth: with the G of two consecutive chunks kept, one pass contracts over both and the dW traffic
+  // halves (one more [chunk, V] bf16 buffer). Up to 8192 tokens per pass (the kernel's k-block skip list).
+  L.dw_group = (T > L.C && 2 * L.C <= 8192) ? 2 : 1;
+  const long long g_tokens = (long long)L.dw_group * L.C < T ? (long long)L.dw_group * L.C : T;
+  L.g_rows = (long long)up((size_t)g_tokens, 128);
+  L.G = take((size_t)L.g_rows * L.Vpad * 2);
+  L.dh_splits = choose_k_splits(((L.C + kTileM - 1) / kTileM) * n_tiles_for(H, use_wide(H)), (V + BK - 1) / BK,
                                 sm_count_or_default());
   L.dh_part = take(L.dh_splits > 1 ? (size_t)L.dh_splits * L.Cpad * H * 4 : 0);
   L.tiles_per_chunk = (L.C + kTileM - 1) / kTileM;
@@ -349,30 +364,30 @@ static void fill_forward_params(GemmParams* p, const WsLayout& L, void* ws, long
   p->m_live = (live_c && p->m_tiles <= MAX_LIVE_M) ? live_c : nullptr;
 }
 
-// The two output GEMMs of one chunk, shared by kdkl_backward and kdkl_forward_backward: G holds the chunk's
-// dlogits (bf16 [rows, Vpad]).
+// The two output GEMMs, shared by kdkl_backward and kdkl_forward_backward. G holds the dlogits (bf16, rows of
+// Vpad elements) of the chunk, or of the group of chunks one dW pass contracts over.
 //   dH[chunk] = G W        (M = rows, N = H, K = V; split-K with a fixed-order fix-up when the tiles are few)
-//   dW (+)= G^T h[chunk]   (M = V, N = H, K = rows; both operands MN-major: G is [t, v] with v contiguous,
-//                           h is [t, h] with h contiguous)
+//   dW (+)= G^T h[group]   (M = V, N = H, K = rows of the group; both operands MN-major: G is [t, v] with v
+//                           contiguous, h is [t, h] with h contiguous)
 struct ChunkOut {
   const __nv_bfloat16* G; const __nv_bfloat16* hA; void* dhidden; long long s0, rows, H, V;
   const WsLayout* L; const kdkl_options* o; WsHeader* hdr; void* ws; const int* go;
   const uint8_t* live_m;   // row-tile flags for the dH GEMM (nullptr: none)
-  const uint8_t* live_c;   // the chunk's row-tile flags for the dW contraction (nullptr: none)
+  const uint8_t* live_c;   // row-tile flags of the dW contraction (nullptr: none)
   int accumulate_dw;
 };
-static int launch_chunk_outputs(const ChunkOut& c, const CUtensorMap& tmWmn, const CUtensorMap& tmdW,
-                                const DeviceInfo& di, cudaStream_t st) {
+static int launch_dhidden(const ChunkOut& c, const CUtensorMap& tmWmn, const DeviceInfo& di, cudaStream_t st) {
   const WsLayout& L = *c.L;
   const long long rows = c.rows, H = c.H, V = c.V, s0 = c.s0;
   int rc;
-  CUtensorMap tmG, tmGmn, tmhmn, tmdH;
+  CUtensorMap tmG, tmdH;
   stage_mark(ST_B2, st);
   if ((rc = make_tmap_bf16(&tmG, c.G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, BK, BM))) return rc;
+  const bool wide = use_wide(H);
   GemmParams p2;
   memset(&p2, 0, sizeof(p2));
   p2.M = (int)rows; p2.N = (int)H; p2.K = (int)V;
-  p2.m_tiles = (int)((rows + kTileM - 1) / kTileM); p2.n_tiles = (int)((H + BN - 1) / BN); p2.m_inner = 0;
+  p2.m_tiles = (int)((rows + kTileM - 1) / kTileM); p2.n_tiles = (int)n_tiles_for(H, wide); p2.m_inner = 0;
   p2.status = &c.hdr->status; p2.go = c.go;
   p2.m_live = c.live_m;              // dead row tiles: their dH rows are written as zeros
   // a short last chunk may want a different split; never more than the workspace was sized for
@@ -386,33 +401,63 @@ static int launch_chunk_outputs(const ChunkOut& c, const CUtensorMap& tmWmn, con
     float* part = at<float>(c.ws, L.dh_part);
     p2.split_rows = (int)L.Cpad;
     if ((rc = make_tmap_out_f32(&tmdH, part, (uint64_t)H, (uint64_t)sp * L.Cpad, (uint64_t)H))) return rc;
-    if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, di, st))) return rc;
+    rc = wide ? launch_gemm<EPI_STORE_F32, false, true, true>(tmG, tmWmn, tmdH, p2, di, st)
+              : launch_gemm<EPI_STORE_F32, false, true, false>(tmG, tmWmn, tmdH, p2, di, st);
+    if (rc) return rc;
     const long long n4 = rows * H / 4;
     splitk_fixup_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(part, (long long)L.Cpad * H, sp, n4, dh16, dh32,
                                                                      c.go);
     KDKL_LAUNCHED("splitk_fixup_kernel");
-  } else if (dh16 != nullptr) {
-    if ((rc = make_tmap_out_bf16(&tmdH, dh16, (uint64_t)H, (uint64_t)rows, (uint64_t)H))) return rc;
-    if ((rc = launch_gemm<EPI_STORE_BF16, false, true>(tmG, tmWmn, tmdH, p2, di, st))) return rc;
-  } else {
-    if ((rc = make_tmap_out_f32(&tmdH, dh32, (uint64_t)H, (uint64_t)rows, (uint64_t)H))) return rc;
-    if ((rc = launch_gemm<EPI_STORE_F32, false, true>(tmG, tmWmn, tmdH, p2, di, st))) return rc;
+    return KDKL_OK;
   }
+  if (dh16 != nullptr) {
+    if ((rc = make_tmap_out_bf16(&tmdH, dh16, (uint64_t)H, (uint64_t)rows, (uint64_t)H))) return rc;
+    return wide ? launch_gemm<EPI_STORE_BF16, false, true, true>(tmG, tmWmn, tmdH, p2, di, st)
+                : launch_gemm<EPI_STORE_BF16, false, true, false>(tmG, tmWmn, tmdH, p2, di, st);
+  }
+  if ((rc = make_tmap_out_f32(&tmdH, dh32, (uint64_t)H, (uint64_t)rows, (uint64_t)H))) return rc;
+  return wide ? launch_gemm<EPI_STORE_F32, false, true, true>(tmG, tmWmn, tmdH, p2, di, st)
+              : launch_gemm<EPI_STORE_F32, false, true, false>(tmG, tmWmn, tmdH, p2, di, st);
+}
 
+// c.G / c.hA / c.rows: the whole group (rows = tokens of all its chunks, contiguous in G and in hidden).
+static int launch_dweight(const ChunkOut& c, const CUtensorMap& tmdW, const DeviceInfo& di, cudaStream_t st) {
+  const WsLayout& L = *c.L;
+  const long long rows = c.rows, H = c.H, V = c.V;
+  int rc;
+  CUtensorMap tmGmn, tmhmn;
   if ((rc = make_tmap_bf16(&tmGmn, c.G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad * 2, 64, BK))) return rc;
   if ((rc = make_tmap_bf16(&tmhmn, c.hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, 64, BK))) return rc;
+  const bool wide = use_wide(H);
   GemmParams p3;
   memset(&p3, 0, sizeof(p3));
   p3.M = (int)V; p3.N = (int)H; p3.K = (int)rows;
-  p3.m_tiles = (int)((V + kTileM - 1) / kTileM); p3.n_tiles = (int)((H + BN - 1) / BN); p3.m_inner = 0; p3.k_splits = 1;
+  p3.m_tiles = (int)((V + kTileM - 1) / kTileM); p3.n_tiles = (int)n_tiles_for(H, wide); p3.m_inner = 0; p3.k_splits = 1;
   p3.status = &c.hdr->status; p3.go = c.go;
   p3.accumulate = c.accumulate_dw;
   // dead row tiles of G are zeros: they are left out of the contraction over tokens (the kernel takes up to 32 flags)
   p3.k_live = (rows <= 32ll * kTileM && (rows + BK - 1) / BK <= MAX_LIVE_KB) ? c.live_c : nullptr;
   stage_mark(ST_B3, st);
-  return launch_gemm<EPI_STORE_F32, true, true>(tmGmn, tmhmn, tmdW, p3, di, st);
+  return wide ? launch_gemm<EPI_STORE_F32, true, true, true>(tmGmn, tmhmn, tmdW, p3, di, st)
+              : launch_gemm<EPI_STORE_F32, true, true, false>(tmGmn, tmhmn, tmdW, p3, di, st);
 }
 
+// Where chunk ci's G lives inside the group buffer, and whether a dW pass is due after it.
+struct GroupPos { long long j, row0; bool last; };
+static GroupPos group_pos(const WsLayout& L, long long ci, long long s0, long long rows, long long T) {
+  GroupPos g;
+  g.j = ci % L.dw_group;
+  g.row0 = g.j * L.C;
+  g.last = g.j == L.dw_group - 1 || s0 + rows >= T;
+  return g;
+}
+// The row-tile flags of a group are those of its chunks one after the other; they line up with the group's
+// 256-row tiles only when every chunk but the last is a whole number of tiles.
+static const uint8_t* group_flags(const WsLayout& L, const uint8_t* live, long long ci_first) {
+  if (live == nullptr) return nullptr;
+  if (L.dw_group > 1 && (L.C % kTileM) != 0) return nullptr;
+  return live + ci_first * L.tiles_per_chunk;
+}
 
 }  // namespace kdkl
 
@@ -586,7 +631,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
                                                                at<float>(ws, L.coefA), at<float>(ws, L.coefB), hdr);
   KDKL_LAUNCHED("bwd_coef_kernel");
 
-  __nv_bfloat16* G = at<__nv_bfloat16>(ws, L.G);
+  __nv_bfloat16* Gbuf = at<__nv_bfloat16>(ws, L.G);
   // W as the K-major B operand of the recompute GEMM, and as the MN-major B operand of dH = G W
   CUtensorMap tmW, tmWmn;
   if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, kBRows))) return rc;
@@ -602,6 +647,8 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
     const uint8_t* live_c = live ? live + ci * L.tiles_per_chunk : nullptr;
     const __nv_bfloat16* hA = reinterpret_cast<const __nv_bfloat16*>(hidden) + s0 * H;
+    const GroupPos gp = group_pos(L, ci, s0, rows, T);
+    __nv_bfloat16* G = Gbuf + gp.row0 * L.Vpad;            // this chunk's rows inside the group buffer
     CUtensorMap tmA;
     if ((rc = make_tmap_bf16(&tmA, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, BK, BM))) return rc;
 
@@ -639,9 +686,15 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
       if ((rc = launch_gemm<EPI_DLOGITS, false, false>(tmA, tmW, tmGout, p, di, st))) return rc;
     }
 
-    ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, go, live_m, live_c,
-                (ci > 0 || o.accumulate_dweight) ? 1 : 0};
-    if ((rc = launch_chunk_outputs(co, tmWmn, tmdW, di, st))) return rc;
+    ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, go, live_m, live_c, 0};
+    if ((rc = launch_dhidden(co, tmWmn, di, st))) return rc;
+    if (gp.last) {
+      // one dW pass over the group that ends here: its chunks' G rows and hidden rows are contiguous
+      const long long ci0 = ci - gp.j, g_s0 = s0 - gp.row0;
+      ChunkOut cg{Gbuf, reinterpret_cast<const __nv_bfloat16*>(hidden) + g_s0 * H, nullptr, g_s0, gp.row0 + rows, H, V,
+                  &L, &o, hdr, ws, go, nullptr, group_flags(L, live, ci0), (ci0 > 0 || o.accumulate_dweight) ? 1 : 0};
+      if ((rc = launch_dweight(cg, tmdW, di, st))) return rc;
+    }
   }
   return KDKL_OK;
 }
@@ -676,7 +729,7 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
                                                                 at<float>(ws, L.coefA), at<float>(ws, L.coefB), hdr);
   KDKL_LAUNCHED("step_coef_kernel");
 
-  __nv_bfloat16* G = at<__nv_bfloat16>(ws, L.G);
+  __nv_bfloat16* Gbuf = at<__nv_bfloat16>(ws, L.G);
   CUtensorMap tmW, tmWmn, tmdW;
   if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, kBRows))) return rc;
   if ((rc = make_tmap_bf16(&tmWmn, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, 64, BK))) return rc;
@@ -687,6 +740,8 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
     const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
     const uint8_t* live_c = live ? live + ci * L.tiles_per_chunk : nullptr;
     const __nv_bfloat16* hA = reinterpret_cast<const __nv_bfloat16*>(hidden) + s0 * H;
+    const GroupPos gp = group_pos(L, ci, s0, rows, T);
+    __nv_bfloat16* G = Gbuf + gp.row0 * L.Vpad;
     CUtensorMap tmA, tmGout;
     if ((rc = make_tmap_bf16(&tmA, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, BK, BM))) return rc;
     if ((rc = make_tmap_out_bf16(&tmGout, G, (uint64_t)V, (uint64_t)rows, (uint64_t)L.Vpad))) return rc;
@@ -717,9 +772,14 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
     KDKL_LAUNCHED("e_to_g_kernel");
 
     // dH[chunk] = G W and dW (+)= G^T h, exactly as in kdkl_backward
-    ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, nullptr, live_m, live_c,
-                (ci > 0 || o.accumulate_dweight) ? 1 : 0};
-    if ((rc = launch_chunk_outputs(co, tmWmn, tmdW, di, st))) return rc;
+    ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, nullptr, live_m, live_c, 0};
+    if ((rc = launch_dhidden(co, tmWmn, di, st))) return rc;
+    if (gp.last) {
+      const long long ci0 = ci - gp.j, g_s0 = s0 - gp.row0;
+      ChunkOut cg{Gbuf, reinterpret_cast<const __nv_bfloat16*>(hidden) + g_s0 * H, nullptr, g_s0, gp.row0 + rows, H, V,
+                  &L, &o, hdr, ws, nullptr, nullptr, group_flags(L, live, ci0), (ci0 > 0 || o.accumulate_dweight) ? 1 : 0};
+      if ((rc = launch_dweight(cg, tmdW, di, st))) return rc;
+    }
   }
   stage_mark(ST_REDUCE, st);
   loss_reduce_kernel<<<1, 1024, 0, st>>>(at<float>(ws, L.loss_tok), loss_mask, T, o.denom_override, o.denom_device, tau,
@@ -1160,11 +1220,18 @@ int kdkl_gemm_bf16(const void* A, const void* B, float* C, int64_t M, int64_t N,
   GemmParams p;
   memset(&p, 0, sizeof(p));
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
-  p.m_tiles = (int)((M + kTileM - 1) / kTileM); p.n_tiles = (int)((N + BN - 1) / BN); p.k_splits = 1;
+  const bool wide = use_wide(N);                // the same choice of tile width as the loss's output GEMMs
+  p.m_tiles = (int)((M + kTileM - 1) / kTileM); p.n_tiles = (int)n_tiles_for(N, wide); p.k_splits = 1;
   p.m_inner = p.m_tiles <= p.n_tiles ? 1 : 0;   // walk the shorter dimension first: the other operand streams once
   p.status = status; p.accumulate = 0;
   CUtensorMap tc;
   if ((rc = make_tmap_out_f32(&tc, C, (uint64_t)N, (uint64_t)M, (uint64_t)N))) return rc;
+  if (wide) {
+    if (a_mn && b_mn) return launch_gemm<EPI_STORE_F32, true, true, true>(ta, tb, tc, p, di, st);
+    if (a_mn) return launch_gemm<EPI_STORE_F32, true, false, true>(ta, tb, tc, p, di, st);
+    if (b_mn) return launch_gemm<EPI_STORE_F32, false, true, true>(ta, tb, tc, p, di, st);
+    return launch_gemm<EPI_STORE_F32, false, false, true>(ta, tb, tc, p, di, st);
+  }
   if (a_mn && b_mn) return launch_gemm<EPI_STORE_F32, true, true>(ta, tb, tc, p, di, st);
   if (a_mn) return launch_gemm<EPI_STORE_F32, true, false>(ta, tb, tc, p, di, st);
   if (b_mn) return launch_gemm<EPI_STORE_F32, false, true>(ta, tb, tc, p, di, st);

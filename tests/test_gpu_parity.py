@@ -109,7 +109,8 @@ def _small_case(T, H, V, K, seed, mask_frac=0.0, dup=False, empty=False):
 
 # ------------------------------------------------------------------------------------------ GEMM
 @pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 0), (1, 1)])
-@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (328, 520, 200), (1024, 1280, 520)])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (328, 520, 200), (1024, 1280, 520),
+                                   (328, 1000, 200), (520, 1024, 328), (264, 2048, 136)])   # N >= 1000: 512-wide tiles
 def test_bare_gemm_all_operand_layouts(M, N, K, a_mn, b_mn):
     g = torch.Generator().manual_seed(M + N + K)
     A = torch.randn(M, K, generator=g).to(torch.bfloat16)
@@ -156,6 +157,51 @@ def test_ragged_shapes_mask_temperature(chunk):
     d["topk_idx"], d["topk_val"] = I.poison_masked(d["topk_idx"], d["topk_val"], d["mask"])
     op = _run(d, T, H, V, K, chunk, tau)
     _compare(op, _oracle(d, tau), d)
+
+
+@pytest.mark.parametrize("T,H,V,K,chunk,masked", [
+    (700, 1000, 1100, 9, 256, True),     # 512-wide output tiles (ragged last tile), three chunks = groups of 2 + 1
+    (700, 1024, 1100, 9, 100, True),     # chunk not a multiple of the row tile: the grouped dW pass takes no flags
+    (1300, 1024, 520, 5, 512, True),     # a dead chunk inside a group, a dead tail
+    (600, 1536, 777, 4, 0, False),       # one chunk: no grouping, wide tiles, several k-splits of dH
+])
+def test_wide_output_tiles_and_grouped_dweight(T, H, V, K, chunk, masked):
+    """The two output GEMMs at hidden widths that select 512-column tiles, with the dW pass contracting over
+    groups of two chunks: ragged widths, short last chunks and groups, ignored runs that kill whole row tiles."""
+    d = _small_case(T, H, V, K, seed=T + H)
+    if masked:
+        mask = torch.ones(T, dtype=torch.uint8)
+        mask[::9] = 0
+        mask[T // 2: T // 2 + 300] = 0
+        mask[T - 40:] = 0
+        d["mask"] = mask
+        d["topk_idx"], d["topk_val"] = I.poison_masked(d["topk_idx"], d["topk_val"], mask)
+    op = _run(d, T, H, V, K, chunk, 1.0)
+    _compare(op, _oracle(d, 1.0), d)
+    # fp32 dHidden and dW += onto existing contents through the same kernels
+    dev = _dev()
+    opt = B.make_options(accumulate_dweight=1, dhidden_dtype=1)
+    op2 = B.FusedChunkedKL(T, H, V, K, chunk=chunk, temperature=1.0, opt=opt, device=dev, want_gathered=True,
+                           want_per_token=True)
+    base = torch.randn(V, H, generator=torch.Generator().manual_seed(2)) * 1e-4
+    op2.dweight.copy_(base)
+    op2.dhidden.fill_(float("nan"))
+    g = {k: (v.to(dev) if v is not None else None) for k, v in d.items()}
+    op2.forward(g["hidden"], g["weight"], g["topk_idx"], g["topk_val"], loss_mask=g["mask"])
+    op2.backward(g["hidden"], g["weight"], loss_mask=g["mask"])
+    o = _oracle(d, 1.0)
+    o["dW"] = o["dW"] + base.double().numpy()
+    _compare(op2, o, d, dw_base=base.double().numpy())
+    # and the single-pass call on the same shapes
+    op2.dweight.copy_(base)
+    op2.dhidden.fill_(float("nan"))
+    op2.forward_backward(g["hidden"], g["weight"], g["topk_idx"], g["topk_val"], loss_mask=g["mask"])
+    assert op2.status()[0] == 0
+    dW = op2.dweight.cpu().double().numpy() - base.double().numpy()
+    dH = op2.dhidden.cpu().double().numpy()
+    check_grad_matrix(dH, o["dH"], "dH (single pass)", roundings=2)
+    check_grad_matrix(dW, o["dW"] - base.double().numpy(), "dW (single pass)", roundings=2,
+                      extra_tol=2.0 ** -22 * np.abs(base.double().numpy()))
 
 
 def test_duplicates_empty_slots_and_log_prob_mode():
