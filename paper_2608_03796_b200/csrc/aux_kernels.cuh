@@ -585,8 +585,10 @@ constexpr int COLLECT_SEG = 8192;
 __global__ void __launch_bounds__(256)
 topk_collect_kernel(const float* __restrict__ z, long long ldz, int V, float scale_log2, const float* __restrict__ thr,
                     int* __restrict__ cand_cnt, int* __restrict__ cand_idx, float* __restrict__ cand_val, int cap,
-                    int n_seg) {
+                    int n_seg, const int* go) {
+  if (go != nullptr && *go == 0) return;
   const long long row = blockIdx.x / n_seg;
+  if (thr[row] == INFINITY) return;                  // a row that already holds its candidates
   const int c_begin = (int)(blockIdx.x - row * n_seg) * COLLECT_SEG;
   const float t = thr[row];
   const float4* zr = reinterpret_cast<const float4*>(z + row * ldz);
@@ -611,6 +613,34 @@ topk_collect_kernel(const float* __restrict__ z, long long ldz, int V, float sca
         }
       }
     }
+  }
+}
+
+// Between sweep 2 and the record: a row whose candidate list overflowed (more logits reached the tile-maxima
+// threshold than the list holds - large logits clustered in a few vocabulary tiles, as in a frequency-ordered
+// vocabulary) gets a tighter threshold and is scanned again. The K-th largest of the candidates that were kept is
+// a valid one: they are real logits of the row, so at least K logits reach it and every member of the exact
+// top-K does. The kept ones are an arbitrary subset (list slots are handed out atomically), so the tightened
+// scan admits about K / cap of the previous count; the host enqueues two such rounds, each skipped on the device
+// when no row asked for it (*flag stays 0). Rows that fit keep their list and take no further candidates.
+__global__ void __launch_bounds__(32)
+topk_retighten_kernel(int* __restrict__ cand_cnt, const float* __restrict__ cand_val, int cap, int cpad, int K,
+                      float scale_log2, float* __restrict__ thr, int* flag, const int* go) {
+  extern __shared__ float tk_smem[];
+  if (go != nullptr && *go == 0) return;             // second round: only when the first one ran
+  const int row = blockIdx.x, lane = threadIdx.x;
+  const int n = cand_cnt[row];
+  if (n <= cap) {
+    if (lane == 0) thr[row] = INFINITY;
+    return;
+  }
+  for (int i = lane; i < cpad; i += 32) tk_smem[i] = i < cap ? cand_val[(long long)row * cap + i] : -INFINITY;
+  __syncwarp();
+  warp_bitonic_desc(tk_smem, nullptr, cpad, lane);
+  if (lane == 0) {
+    thr[row] = tk_smem[K - 1] * scale_log2;          // the same fp32 product the scan compares with
+    cand_cnt[row] = 0;
+    *flag = 1;
   }
 }
 

@@ -997,7 +997,8 @@ constexpr long long kTopkTakeAllMaxV = 8192;
 struct TopkLayout {
   long long C, Cpad, n_tiles, ldz;
   int npad, cap, cpad;
-  size_t hdr, zeros, part_m, part_s, thr, cnt, cidx, cval, z, total;
+  size_t hdr, flags, zeros, part_m, part_s, thr, cnt, cidx, cval, z, total;
+  long long n_pass;
 };
 static int pow2_at_least(long long x) { int p = 32; while (p < x) p <<= 1; return p; }
 static TopkLayout topk_layout(long long T, long long V, int K, bool stored = false) {
@@ -1017,6 +1018,8 @@ static TopkLayout topk_layout(long long T, long long V, int K, bool stored = fal
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = up(o + bytes, 256); return at; };
   L.hdr = take(256);
+  L.n_pass = (T + L.C - 1) / L.C;
+  L.flags = take((size_t)L.n_pass * 2 * 4);                // per pass: "rescan wanted" of the two tightening rounds
   L.zeros = take((size_t)L.Cpad * 4);
   L.part_m = take((size_t)L.n_tiles * L.Cpad * 4);
   L.part_s = take((size_t)L.n_tiles * L.Cpad * 4);
@@ -1062,7 +1065,8 @@ static int teacher_topk_impl(const void* hidden, const void* weight, int64_t T, 
 
   CUtensorMap tmW;
   if ((rc = make_tmap_bf16(&tmW, weight, (uint64_t)H, (uint64_t)V, (uint64_t)H * 2, BK, kBRows))) return rc;
-  for (long long s0 = 0; s0 < T; s0 += L.C) {
+  long long pass = 0;
+  for (long long s0 = 0; s0 < T; s0 += L.C, ++pass) {
     const long long rows = (T - s0 < L.C) ? (T - s0) : L.C;
     CUtensorMap tmA;
     const __nv_bfloat16* hA = reinterpret_cast<const __nv_bfloat16*>(hidden) + s0 * H;
@@ -1092,13 +1096,38 @@ static int teacher_topk_impl(const void* hidden, const void* weight, int64_t T, 
       const int n_seg = (int)((V + COLLECT_SEG - 1) / COLLECT_SEG);
       topk_collect_kernel<<<(unsigned)(rows * n_seg), 256, 0, st>>>(
           at<float>(ws, L.z), L.ldz, (int)V, p.scale_log2, at<float>(ws, L.thr), at<int>(ws, L.cnt),
-          at<int>(ws, L.cidx), at<float>(ws, L.cval), L.cap, n_seg);
+          at<int>(ws, L.cidx), at<float>(ws, L.cval), L.cap, n_seg, nullptr);
       KDKL_LAUNCHED("topk_collect_kernel");
     } else {
       // sweep 2: recompute, emit everything at or above the row's threshold
       p.thr = at<float>(ws, L.thr); p.cand_cnt = at<int>(ws, L.cnt);
       p.cand_idx = at<int>(ws, L.cidx); p.cand_val = at<float>(ws, L.cval); p.cand_cap = L.cap;
       if ((rc = launch_gemm<EPI_TOPK, false, false>(tmA, tmW, tmA, p, di, st))) return rc;
+    }
+    // Lists that overflowed (more logits at or above the tile-maxima threshold than slots): up to two rounds of
+    // a tighter threshold and a new scan, each skipped on the device when no row of this pass asked for it.
+    if (L.cap < V) {
+      int* flags = at<int>(ws, L.flags) + 2 * pass;
+      KDKL_CUDA(cudaFuncSetAttribute(topk_retighten_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.cpad * 4));
+      for (int round = 0; round < 2; ++round) {
+        topk_retighten_kernel<<<(unsigned)rows, 32, (size_t)L.cpad * 4, st>>>(
+            at<int>(ws, L.cnt), at<float>(ws, L.cval), L.cap, L.cpad, K, p.scale_log2, at<float>(ws, L.thr),
+            flags + round, round == 0 ? nullptr : flags);
+        KDKL_LAUNCHED("topk_retighten_kernel");
+        if (stored) {
+          const int n_seg = (int)((V + COLLECT_SEG - 1) / COLLECT_SEG);
+          topk_collect_kernel<<<(unsigned)(rows * n_seg), 256, 0, st>>>(
+              at<float>(ws, L.z), L.ldz, (int)V, p.scale_log2, at<float>(ws, L.thr), at<int>(ws, L.cnt),
+              at<int>(ws, L.cidx), at<float>(ws, L.cval), L.cap, n_seg, flags + round);
+          KDKL_LAUNCHED("topk_collect_kernel");
+        } else {
+          p.thr = at<float>(ws, L.thr); p.cand_cnt = at<int>(ws, L.cnt);
+          p.cand_idx = at<int>(ws, L.cidx); p.cand_val = at<float>(ws, L.cval); p.cand_cap = L.cap;
+          p.go = flags + round;
+          if ((rc = launch_gemm<EPI_TOPK, false, false>(tmA, tmW, tmA, p, di, st))) return rc;
+          p.go = nullptr;
+        }
+      }
     }
     KDKL_CUDA(cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.cpad * 8));
     topk_select_kernel<<<(unsigned)rows, 32, (size_t)L.cpad * 8, st>>>(

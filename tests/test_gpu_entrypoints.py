@@ -98,7 +98,7 @@ def test_profile_single_pass_accounts_for_every_stage_and_changes_nothing():
                                     op.dhidden, op.dweight, chunk=cfg.chunk, temperature=cfg.tau)
     chunks = cfg.T // cfg.chunk
     assert st["fwd_gemm_lse_exp"][1] == chunks and st["exp_to_dlogits"][1] == chunks and st["combine"][1] == chunks
-    assert st["dhidden_gemm"][1] == chunks and st["dweight_gemm"][1] == chunks
+    assert st["dhidden_gemm"][1] == chunks and st["dweight_gemm"][1] == (chunks + 1) // 2
     assert st["prep"][1] == 1 and st["loss_reduce"][1] == 1 and "bwd_coef" not in st
     assert all(ms > 0 for ms, n in st.values())
     assert torch.equal(op.loss, ref[0]) and torch.equal(op.dhidden, ref[1]) and torch.equal(op.dweight, ref[2])

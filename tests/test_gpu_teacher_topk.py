@@ -86,6 +86,25 @@ def test_ties_break_by_smaller_index_and_overflow_is_reported():
     assert B.kdkl_status(ws2)[0] == -12
 
 
+@pytest.mark.parametrize("stored", [False, True])
+def test_large_logits_clustered_in_a_few_tiles(stored):
+    """A frequency-ordered vocabulary: the first 3000 entries carry systematically larger logits, so thousands of
+    logits reach the K-th largest tile maximum and the first candidate list (max(4K, 256) slots) overflows. The
+    kernel tightens the threshold on the device and scans again; the record must still be the exact top-K."""
+    T, H, V, K = 300, 64, 40000, 32
+    g = torch.Generator().manual_seed(77)
+    u = torch.randn(H, generator=g)
+    u = u / u.norm()
+    h = (torch.randn(T, H, generator=g) * 0.5 + 4.0 * u).to(torch.bfloat16)
+    W = torch.randn(V, H, generator=g) / H ** 0.5
+    W[:3000] += 1.5 * u * torch.rand(3000, 1, generator=g)          # logits of the head entries shifted up by ~0..6
+    W = W.to(torch.bfloat16)
+    z = h.double() @ W.double().T
+    thr = torch.topk(z.view(T, -1, 250).amax(-1), K, dim=1).values[:, -1]   # roughly the tile-maxima threshold
+    assert ((z >= thr[:, None]).sum(1) > 4 * max(4 * K, 256)).any()           # far more than the first list holds
+    _check(h, W, K, 1.0, stored)
+
+
 def test_cache_feeds_the_loss_with_exact_retained_mass():
     """Teacher kernel -> cache record -> fused loss with teacher_lse: the paper's un-renormalised M < 1 path,
     end to end on the GPU, against the oracles fed with their own (fp64) cache."""
