@@ -466,7 +466,7 @@ def run_context_sweep(args, peaks) -> dict:
                    "comparison losses as torch programs (paper_2608_03796_b200/comparators.py), oom = out of memory"}
     pts = [(r["T"], r["peak_gb"]) for r in rows if r.get("method") == "fused" and "ms_per_iter" in r
            and r["H"] == 4096 and r["V"] == 131072 and r["T"] >= 32768]
-    if len(pts) >= 3:
+    if len({p[0] for p in pts}) >= 3:                 # a line needs three distinct lengths to mean anything
         a, b, res = linear_fit(pts)
         out["fused_peak_memory_fit"] = {"intercept_gb": a, "kb_per_token": b * 1e6, "largest_relative_residual": res,
                                         "over_T": [p[0] for p in pts]}

@@ -78,6 +78,10 @@ struct GemmParams {
   int M, N, K;               // valid extents of this launch
   int m_tiles, n_tiles;      // tiles of TILE_M rows and of TILE_N columns (256, or 512 for the WIDE instantiation)
   int m_inner;               // 1: consecutive tile ids walk M first (B panel shared), 0: N first
+  int m_group;               // m_inner only, 0 = all: row tiles per group. Tiles walk group by group (all column
+                             // tiles of one group of row tiles before the next group), so that the A rows in use
+                             // at any time are one group's (sized by the host to stay resident in L2) while B is
+                             // streamed once per group
   int k_splits;              // >= 1: each tile's contraction is cut into this many work units, each
                              // writing its own partial output (split s goes to output rows + s * split_rows)
   int split_rows;
@@ -254,8 +258,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   };
 
   auto tile_coords = [&](int tile, int& mt, int& nt) {
-    if (p.m_inner) { mt = tile % m_count; nt = tile / m_count; }
-    else           { nt = tile % p.n_tiles; mt = tile / p.n_tiles; }
+    if (p.m_inner) {
+      const int gm = (p.m_group > 0 && p.m_group < m_count) ? p.m_group : m_count;
+      const int g = tile / (gm * p.n_tiles);           // only the last group can be short
+      const int r = tile - g * gm * p.n_tiles;
+      const int m_here = m_count - g * gm < gm ? m_count - g * gm : gm;
+      mt = g * gm + r % m_here; nt = r / m_here;
+    } else { nt = tile % p.n_tiles; mt = tile / p.n_tiles; }
     if (mskip) mt = live_m[mt];
   };
 

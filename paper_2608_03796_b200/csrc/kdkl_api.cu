@@ -118,6 +118,13 @@ constexpr int kWideN = GemmCfg<kNCTA, true>::TILE_N;
 static_assert(GemmCfg<kNCTA, true>::B_ROWS / 2 == kBRows, "a WIDE tile's halves take the narrow tile's B boxes");
 // The two output GEMMs (N = H) use WIDE tiles when rounding H up to whole 512-column tiles wastes at most a
 // tenth of the tensor work (H = 4096, 3072, 1024, 1000 ...); narrow 256-column tiles otherwise.
+// Row tiles per raster group of the two vocabulary sweeps (forward, recompute): as many as keep the group's hidden
+// rows within 32 MiB, i.e. resident in either half of the L2 while the weight streams past (4096 tokens at H = 4096).
+static int m_group_for(long long H) {
+  const long long rows = (32ll << 20) / (H * 2);
+  const long long g = rows / kTileM;
+  return (int)(g < 1 ? 1 : g);
+}
 static bool use_wide(long long N) { return ((N + kWideN - 1) / kWideN) * kWideN * 10 <= N * 11; }
 static long long n_tiles_for(long long N, bool wide) { return wide ? (N + kWideN - 1) / kWideN : (N + BN - 1) / BN; }
 // What the library has learnt about each device, asked once per device and process (a benign race: two
@@ -354,6 +361,7 @@ static void fill_forward_params(GemmParams* p, const WsLayout& L, void* ws, long
   memset(p, 0, sizeof(*p));
   p->M = (int)rows; p->N = (int)V; p->K = (int)H;
   p->m_tiles = (int)((rows + kTileM - 1) / kTileM); p->n_tiles = (int)L.n_tiles_v; p->m_inner = 1; p->k_splits = 1;
+  p->m_group = m_group_for(H);
   p->status = &hdr->status; p->go = nullptr;
   p->scale_log2 = kLog2e * inv_tau; p->Ktop = K;
   p->idx_sorted = at<int>(ws, L.idx_sorted) + s0 * K;
@@ -657,6 +665,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     memset(&p, 0, sizeof(p));
     p.M = (int)rows; p.N = (int)V; p.K = (int)H;
     p.m_tiles = (int)((rows + kTileM - 1) / kTileM); p.n_tiles = (int)L.n_tiles_v; p.m_inner = 1; p.k_splits = 1;
+    p.m_group = m_group_for(H);
     p.status = &hdr->status; p.go = go;
     p.scale_log2 = kLog2e * inv_tau; p.Ktop = K;
     p.idx_sorted = at<int>(ws, L.idx_sorted) + s0 * K;
