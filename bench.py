@@ -44,14 +44,14 @@ if ROOT not in sys.path:
 METRIC = "KL fwd+bwd tokens/s & % of bf16 tensor peak; peak HBM GB vs sequence length"
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 
-# DRAM bytes (read + write) per launch of each tensor-core kernel, from one ncu capture of the shipped CTA-pair
-# build on a reduced case (chunk 4096, H = 4096, V = 32768: every operand larger than L2, about 1.3 GB on the
-# device; profiles/dram_traffic_pair_build_C4096_V32768.md). A launch's traffic is proportional to the vocabulary
-# rows it sweeps, so the figure for another V at this chunk and H is scaled by V / 32768. The dW figure is the
-# reduce-add form (every chunk after the first).
+# DRAM bytes (read + write) of each tensor-core kernel per chunk of 4096 tokens, from one ncu capture of the shipped
+# build on a reduced case (chunk 4096, H = 4096, V = 32768, four chunks: every operand larger than L2, 2 GB on the
+# device; profiles/dram_traffic_C4096_V32768.md). A kernel's traffic is proportional to the vocabulary rows it
+# sweeps, so the figure for another V at this chunk and H is scaled by V / 32768. The dW kernel contracts over
+# two chunks per launch (reduce-add form: 2,042,949,888 B read + 504,135,936 B written per launch).
 TRAFFIC_REF = {"chunk": 4096, "H": 4096, "V": 32768,
-               "bytes": {"fwd_gemm_lse": 306605312 + 9421568, "bwd_gemm_dlogits": 377513472 + 247802880,
-                         "dhidden_gemm": 1392504320 + 116503808, "dweight_gemm": 975120384 + 496788736}}
+               "bytes": {"fwd_gemm_lse": 306816768 + 9341696, "bwd_gemm_dlogits": 363689472 + 247999744,
+                         "dhidden_gemm": 959217920 + 232837376, "dweight_gemm": (2042949888 + 504135936) // 2}}
 
 SWEEP_FUSED = [("c2", 10), ("c3", 5), ("c4a", 4), ("c4b", 3), ("c4c", 3), ("c5", 5)]
 SWEEP_DENSE = [("c2", 3), ("c3", 3), ("c4a", 2)]
@@ -764,7 +764,7 @@ def main():
                     "frac_of_burst": dom_tflops / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"])),
                     "traffic": traffic,
                     "traffic_source": (None if traffic is None else
-                                       "ncu, CTA-pair build, reduced case (chunk 4096, V 32768), scaled by V / 32768"),
+                                       "ncu, reduced case (chunk 4096, V 32768), scaled by V / 32768 and by the chunks per launch"),
                     "ms_per_launch": stages[dom]["ms_per_launch"], "flops_per_launch": flops_per_launch,
                     "sm_mhz_during_stage_run": stage_clocks["sm_mhz"]}
     line = {

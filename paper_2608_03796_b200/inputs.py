@@ -107,9 +107,10 @@ CONFIGS = {
     "c4c": Config("c4c", T=262144, H=4096, V=131072, K=100, chunk=4096),
     # a reduced case for profiler captures: operands still larger than L2, about 1.5 GB on the device
     "prof": Config("prof", T=2048, H=4096, V=32768, K=100, chunk=2048),
-    # two full-size chunks over a quarter of the vocabulary: every GEMM launch has the benchmark's chunk and H (so a
-    # launch's DRAM traffic is the benchmark's scaled by V / 131072), about 1.5 GB on the device
-    "prof2": Config("prof2", T=8192, H=4096, V=32768, K=100, chunk=4096),
+    # four full-size chunks over a quarter of the vocabulary: every GEMM launch has the benchmark's chunk and H (so a
+    # launch's DRAM traffic is the benchmark's scaled by V / 131072) and the second dW pass accumulates; about 2 GB
+    # on the device
+    "prof2": Config("prof2", T=16384, H=4096, V=32768, K=100, chunk=4096),
     "c5": Config("c5", T=32768, H=3072, V=128256, K=100, chunk=2048, tau=2.0,
                  idx_dist="zipf", tok_offset=False, packed_docs=8, pad_frac=0.05),
 }
