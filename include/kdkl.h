@@ -76,6 +76,15 @@ typedef struct kdkl_options {
                                  the mean (takes precedence over denom_override). For data-parallel callers that
                                  sum kdkl_count_tokens over their ranks on the device: no host read of the count.
                                  A struct of a previous size (without this field) is accepted */
+  int32_t dw_chunks_per_pass; /* 0 (default): with chunks of at most 4096 tokens, dweight += G^T h runs once per two
+                                 chunks (the dlogits of both are kept: one more [chunk, V] bf16 buffer in the
+                                 workspace, 1 GiB at chunk 4096 and V = 131072), which halves the fp32
+                                 read-modify-write traffic of dweight; 1: once per chunk, without that buffer;
+                                 2: as 0. Measured on one B200 at T = 131072, H = 4096, V = 131072: 413-416 ms with
+                                 8.15 GB peak (default) against 415-420 ms with 7.07 GB (1); at chunk 2048,
+                                 H = 3072: 74.9 against 77.0 ms. Same results up to fp32 reassociation in dweight.
+                                 kdkl_workspace_bytes must be given the same options as the calls.
+                                 A struct of a previous size (without this field) is accepted */
 } kdkl_options;
 
 /* Number of counted tokens of a batch (mask = 1; T when loss_mask is NULL), written as one double to

@@ -47,7 +47,7 @@ class kdkl_options(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_int32), ("teacher_mode", ctypes.c_int32),
                 ("accumulate_dweight", ctypes.c_int32), ("dhidden_dtype", ctypes.c_int32),
                 ("denom_override", ctypes.c_float), ("stored_exponentials", ctypes.c_int32),
-                ("denom_device", ctypes.c_void_p)]
+                ("denom_device", ctypes.c_void_p), ("dw_chunks_per_pass", ctypes.c_int32)]
 
 
 _lib = None
@@ -169,14 +169,15 @@ def _stream():
 
 
 def make_options(teacher_mode=0, accumulate_dweight=0, dhidden_dtype=0, denom_override=0.0,
-                 stored_exponentials=0, denom_device: Optional[torch.Tensor] = None) -> kdkl_options:
+                 stored_exponentials=0, denom_device: Optional[torch.Tensor] = None,
+                 dw_chunks_per_pass=0) -> kdkl_options:
     """denom_device: a CUDA float64 tensor of one element holding the divisor of the mean (read on the device
     when the kernels run); the caller keeps it alive until they have run."""
     ptr = None
     if denom_device is not None:
         ptr = _dptr(denom_device, torch.float64, (1,), "denom_device").value
     return kdkl_options(ctypes.sizeof(kdkl_options), teacher_mode, accumulate_dweight, dhidden_dtype, denom_override,
-                        stored_exponentials, ptr)
+                        stored_exponentials, ptr, dw_chunks_per_pass)
 
 
 def kdkl_count_tokens(loss_mask: Optional[torch.Tensor], T: int, count_out: torch.Tensor) -> None:

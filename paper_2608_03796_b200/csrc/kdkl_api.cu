@@ -236,7 +236,8 @@ struct WsLayout {
 static size_t g_guard_bytes = 0;
 static size_t ws_guard_bytes() { return g_guard_bytes; }
 
-static WsLayout ws_layout(long long T, long long H, long long V, int K, long long chunk) {
+// chunks_per_pass: the caller's kdkl_options.dw_chunks_per_pass (0 = default).
+static WsLayout ws_layout(long long T, long long H, long long V, int K, long long chunk, int chunks_per_pass) {
   WsLayout L;
   L.C = chunk <= 0 ? 4096 : chunk;
   if (L.C > T) L.C = T;
@@ -271,7 +272,7 @@ static WsLayout ws_layout(long long T, long long H, long long V, int K, long lon
   // dW += G^T h is read-modify-write of the whole fp32 dW per pass, and every byte a GEMM stores costs its SM
   // load bandwidth: with the G of two consecutive chunks kept, one pass contracts over both and the dW traffic
   // halves (one more [chunk, V] bf16 buffer). Up to 8192 tokens per pass (the kernel's k-block skip list).
-  L.dw_group = (T > L.C && 2 * L.C <= 8192) ? 2 : 1;
+  L.dw_group = (T > L.C && 2 * L.C <= 8192 && chunks_per_pass != 1) ? 2 : 1;
   const long long g_tokens = (long long)L.dw_group * L.C < T ? (long long)L.dw_group * L.C : T;
   L.g_rows = (long long)up((size_t)g_tokens, 128);
   L.G = take((size_t)L.g_rows * L.Vpad * 2);
@@ -285,18 +286,28 @@ static WsLayout ws_layout(long long T, long long H, long long V, int K, long lon
   return L;
 }
 
-// Options of this or of an earlier struct size (without denom_device; without stored_exponentials) are accepted.
+// Options of this or of an earlier struct size (without dw_chunks_per_pass; without denom_device; without
+// stored_exponentials) are accepted.
 static int copy_options(const kdkl_options* opt, kdkl_options* eff) {
   memset(eff, 0, sizeof(*eff));
   if (!opt) return KDKL_OK;
   constexpr int32_t kSize1 = (int32_t)offsetof(kdkl_options, stored_exponentials);
   constexpr int32_t kSize2 = (int32_t)(offsetof(kdkl_options, stored_exponentials) + sizeof(int32_t));
-  if (opt->struct_size != (int32_t)sizeof(kdkl_options) && opt->struct_size != kSize1 && opt->struct_size != kSize2)
+  constexpr int32_t kSize3 = (int32_t)(offsetof(kdkl_options, denom_device) + sizeof(const double*));
+  if (opt->struct_size != (int32_t)sizeof(kdkl_options) && opt->struct_size != kSize1 && opt->struct_size != kSize2 &&
+      opt->struct_size != kSize3)
     return KDKL_ERR_ARG;
   memcpy(eff, opt, (size_t)opt->struct_size);
   eff->struct_size = (int32_t)sizeof(kdkl_options);
   if (eff->stored_exponentials < 0 || eff->stored_exponentials > 1) return KDKL_ERR_ARG;
   return KDKL_OK;
+}
+
+// dw_chunks_per_pass of an option struct as the caller passed it (older, shorter structs do not have the field).
+static int chunks_per_pass_of(const kdkl_options* opt) {
+  if (opt == nullptr) return 0;
+  if (opt->struct_size < (int32_t)(offsetof(kdkl_options, dw_chunks_per_pass) + sizeof(int32_t))) return 0;
+  return opt->dw_chunks_per_pass;
 }
 
 static int check_common(const void* hidden, const void* weight, long long T, long long H, long long V, int K,
@@ -311,7 +322,8 @@ static int check_common(const void* hidden, const void* weight, long long T, lon
   if (eff->teacher_mode == 1 && tau != 1.0f) return KDKL_ERR_ARG;
   if (eff->dhidden_dtype < 0 || eff->dhidden_dtype > 1) return KDKL_ERR_ARG;
   if (((uintptr_t)hidden & 15) || ((uintptr_t)weight & 15) || ((uintptr_t)ws & 15)) return KDKL_ERR_ALIGN;
-  *L = ws_layout(T, H, V, K, chunk);
+  if (eff->dw_chunks_per_pass < 0 || eff->dw_chunks_per_pass > 2) return KDKL_ERR_ARG;
+  *L = ws_layout(T, H, V, K, chunk, eff->dw_chunks_per_pass);
   if (eff->stored_exponentials && T > L->C) return KDKL_ERR_ARG;   // needs one chunk over all tokens
   if (ws_bytes < L->total) return KDKL_ERR_WORKSPACE;
   int rc = device_info(di);
@@ -476,18 +488,18 @@ extern "C" {
 const char* kdkl_last_error(void) { return g_err; }
 int64_t kdkl_last_launch_count(void) { return g_launches; }
 
-int kdkl_workspace_layout(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options*,
+int kdkl_workspace_layout(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options* opt,
                           int64_t* offsets, int64_t* lengths, int32_t capacity) {
   if (T < 1 || H < 1 || V < 1 || K < 1 || !offsets || !lengths) return 0;
-  const WsLayout L = ws_layout(T, H, V, K, chunk);
+  const WsLayout L = ws_layout(T, H, V, K, chunk, chunks_per_pass_of(opt));
   const int n = L.n_slabs < capacity ? L.n_slabs : capacity;
   for (int i = 0; i < n; ++i) { offsets[i] = (int64_t)L.slab_off[i]; lengths[i] = (int64_t)L.slab_len[i]; }
   return L.n_slabs;
 }
 
-size_t kdkl_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options*) {
+size_t kdkl_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options* opt) {
   if (T < 1 || H < 1 || V < 1 || K < 1) return 0;
-  return ws_layout(T, H, V, K, chunk).total;
+  return ws_layout(T, H, V, K, chunk, chunks_per_pass_of(opt)).total;
 }
 
 int64_t kdkl_debug_guard_bytes(int64_t n) {
@@ -601,7 +613,7 @@ int kdkl_forward_finish(const float* all_stats, int32_t n_shards, const uint8_t*
   kdkl_options o;
   memset(&o, 0, sizeof(o));
   if (copy_options(opt, &o) != KDKL_OK) return KDKL_ERR_ARG;
-  WsLayout L = ws_layout(T, H, V_local, K, chunk);
+  WsLayout L = ws_layout(T, H, V_local, K, chunk, o.dw_chunks_per_pass);
   if (ws_bytes < L.total) return KDKL_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   WsHeader* hdr = at<WsHeader>(ws, L.hdr);
@@ -808,11 +820,11 @@ int kdkl_status(const void* ws, void* cuda_stream, int32_t* code, int64_t* detai
   return KDKL_OK;
 }
 
-int kdkl_saved_state(void* ws, int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options*,
+int kdkl_saved_state(void* ws, int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options* opt,
                      const float** logZ, const float** mass) {
   if (!ws) return KDKL_ERR_NULL;
   if (T < 1 || H < 1 || V < 1 || K < 1) return KDKL_ERR_SHAPE;
-  WsLayout L = ws_layout(T, H, V, K, chunk);
+  WsLayout L = ws_layout(T, H, V, K, chunk, chunks_per_pass_of(opt));
   if (logZ) *logZ = at<float>(ws, L.logZ);
   if (mass) *mass = at<float>(ws, L.M);
   return KDKL_OK;
@@ -820,7 +832,8 @@ int kdkl_saved_state(void* ws, int64_t T, int64_t H, int64_t V, int32_t K, int64
 
 // ------------------------------------------------------------------ host-buffer entry point
 struct ArenaLayout { size_t hidden, weight, idx, val, lse, mask, loss, dh, dw, ws, total; };
-static ArenaLayout arena_layout(long long T, long long H, long long V, int K, long long chunk, int dh_fp32) {
+static ArenaLayout arena_layout(long long T, long long H, long long V, int K, long long chunk, int dh_fp32,
+                                int chunks_per_pass) {
   ArenaLayout A;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = up(o + bytes, 256); return at; };
@@ -833,14 +846,14 @@ static ArenaLayout arena_layout(long long T, long long H, long long V, int K, lo
   A.loss = take(256);
   A.dh = take((size_t)T * H * (dh_fp32 ? 4 : 2));
   A.dw = take((size_t)V * H * 4);
-  A.ws = take(ws_layout(T, H, V, K, chunk).total);
+  A.ws = take(ws_layout(T, H, V, K, chunk, chunks_per_pass).total);
   A.total = o;
   return A;
 }
 
 size_t kdkl_host_arena_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk, const kdkl_options* opt) {
   if (T < 1 || H < 1 || V < 1 || K < 1) return 0;
-  return arena_layout(T, H, V, K, chunk, opt ? opt->dhidden_dtype : 0).total;
+  return arena_layout(T, H, V, K, chunk, opt ? opt->dhidden_dtype : 0, chunks_per_pass_of(opt)).total;
 }
 
 int kdkl_forward_backward_host(const void* hidden, const void* weight, const int32_t* topk_idx, const float* topk_val,
@@ -852,7 +865,7 @@ int kdkl_forward_backward_host(const void* hidden, const void* weight, const int
   if (T < 1 || H < 1 || V < 1 || K < 1) return KDKL_ERR_SHAPE;
   if ((uintptr_t)arena & 255) return KDKL_ERR_ALIGN;
   const int dh32 = opt ? opt->dhidden_dtype : 0;
-  ArenaLayout A = arena_layout(T, H, V, K, chunk, dh32);
+  ArenaLayout A = arena_layout(T, H, V, K, chunk, dh32, chunks_per_pass_of(opt));
   if (arena_bytes < A.total) return KDKL_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   uint8_t* d = reinterpret_cast<uint8_t*>(arena);
@@ -862,7 +875,7 @@ int kdkl_forward_backward_host(const void* hidden, const void* weight, const int
   KDKL_CUDA(cudaMemcpyAsync(d + A.val, topk_val, (size_t)T * K * 4, cudaMemcpyHostToDevice, st));
   if (teacher_lse) KDKL_CUDA(cudaMemcpyAsync(d + A.lse, teacher_lse, (size_t)T * 4, cudaMemcpyHostToDevice, st));
   if (loss_mask) KDKL_CUDA(cudaMemcpyAsync(d + A.mask, loss_mask, (size_t)T, cudaMemcpyHostToDevice, st));
-  const size_t ws_bytes = ws_layout(T, H, V, K, chunk).total;
+  const size_t ws_bytes = ws_layout(T, H, V, K, chunk, chunks_per_pass_of(opt)).total;
   int rc = kdkl_forward(d + A.hidden, d + A.weight, reinterpret_cast<int32_t*>(d + A.idx),
                         reinterpret_cast<float*>(d + A.val), teacher_lse ? reinterpret_cast<float*>(d + A.lse) : nullptr,
                         loss_mask ? d + A.mask : nullptr, T, H, V, K, chunk, tau, opt, d + A.ws, ws_bytes,

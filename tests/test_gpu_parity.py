@@ -377,3 +377,21 @@ def test_invariances_offset_and_slot_permutation():
     # the teacher's normaliser is summed in slot order, so p moves in its last bits and single bf16 roundings of G flip
     assert ((b.dweight - base.dweight).norm() / base.dweight.norm()).item() < 2e-3
     assert ((b.dhidden.float() - base.dhidden.float()).norm() / base.dhidden.float().norm()).item() < 2e-3
+
+
+def test_one_dweight_pass_per_chunk_option():
+    """kdkl_options.dw_chunks_per_pass = 1: one dW pass per chunk instead of per two chunks. One [chunk, V] buffer
+    less in the workspace; per-token outputs and dH bitwise the same, dW up to fp32 reassociation; and it matches
+    the oracle on its own."""
+    T, H, V, K, chunk = 1300, 1024, 900, 6, 256
+    d = _small_case(T, H, V, K, seed=44, mask_frac=0.1)
+    two = _run(d, T, H, V, K, chunk, 1.0)
+    opt = B.make_options(dw_chunks_per_pass=1)
+    one = _run(d, T, H, V, K, chunk, 1.0, opt=opt)
+    assert B.kdkl_workspace_bytes(T, H, V, K, chunk) - B.kdkl_workspace_bytes(T, H, V, K, chunk, opt) >= chunk * V * 2
+    assert torch.equal(one.loss_per_token, two.loss_per_token) and torch.equal(one.dhidden, two.dhidden)
+    assert _fro(one.dweight.cpu().double().numpy(), two.dweight.cpu().double().numpy()) < 1e-5
+    _compare(one, _oracle(d, 1.0), d)
+    with pytest.raises(B.KdklError) as e:
+        _run(d, T, H, V, K, chunk, 1.0, opt=B.make_options(dw_chunks_per_pass=3))
+    assert e.value.code == -5

@@ -40,7 +40,7 @@ def test_sizes_without_a_gpu():
 
 def test_options_struct_layout():
     o = binding.make_options(teacher_mode=1, denom_override=3.0)
-    assert o.struct_size == 32 and o.teacher_mode == 1 and o.denom_override == 3.0 and o.stored_exponentials == 0
+    assert o.struct_size == 40 and o.teacher_mode == 1 and o.denom_override == 3.0 and o.stored_exponentials == 0
     assert o.denom_device is None and binding.kdkl_options.denom_device.offset == 24
 
 
