@@ -206,7 +206,12 @@ int kdkl_saved_state(void* workspace, int64_t T, int64_t H, int64_t V, int32_t K
  * arena, runs both passes, copies loss, dhidden and dweight back, and synchronises the stream.
  * Host pointers: hidden, weight, topk_idx, topk_val, teacher_lse (or NULL), loss_mask (or NULL),
  * loss_out [1], dhidden_out [T,H] (dtype per options), dweight_out [V,H] fp32 (either may be NULL
- * to skip that copy). device_arena is a device buffer of at least kdkl_host_arena_bytes(). */
+ * to skip that copy). device_arena is a device buffer of at least kdkl_host_arena_bytes().
+ * With more than one chunk the call overlaps what it can with the chunk loop: the hidden rows of chunk i are
+ * uploaded on a second stream (created and destroyed inside the call, like the events that order the two
+ * streams; no device memory is allocated) while earlier chunks are swept, and the dhidden rows of chunk i are
+ * downloaded while later chunks are differentiated; the weight, the teacher record and dweight, which the whole
+ * step needs or produces, travel on the caller's stream. Use pinned host memory, or the copies serialise. */
 size_t kdkl_host_arena_bytes(int64_t T, int64_t H, int64_t V, int32_t K, int64_t chunk,
                              const kdkl_options* opt);
 int kdkl_forward_backward_host(const void* hidden_bf16, const void* weight_bf16, const int32_t* topk_idx,

@@ -57,6 +57,17 @@ static void stage_mark(int stage, cudaStream_t st) {
   g_timer.stage.push_back(stage);
 }
 
+// ------------------------------------------------------------------ host-buffer pipeline
+// Set (per thread) only while kdkl_forward_backward_host runs its two calls: the hidden rows of chunk i arrive on a
+// copy stream (the forward sweep of chunk i waits for in_ready[i]), and chunk i's dhidden rows leave on it as soon
+// as they are final (dh_ready[i] is recorded after the chunk's dH kernels). Everything else stays on the caller's
+// stream. Events and the copy stream are host-side objects: no device memory is allocated.
+struct HostPipe {
+  cudaStream_t side = nullptr;
+  std::vector<cudaEvent_t> in_ready, dh_ready;
+};
+static thread_local HostPipe* g_pipe = nullptr;
+
 // ------------------------------------------------------------------ tensor maps
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -555,6 +566,8 @@ static int forward_impl(const void* hidden, const void* weight, const int32_t* t
     if ((rc = make_tmap_bf16(&tmA, hA, (uint64_t)H, (uint64_t)rows, (uint64_t)H * 2, BK, BM))) return rc;
     GemmParams p;
     fill_forward_params(&p, L, ws, s0, rows, H, V, K, inv_tau, live ? live + fci * L.tiles_per_chunk : nullptr);
+    if (g_pipe != nullptr && fci < (long long)g_pipe->in_ready.size())
+      KDKL_CUDA(cudaStreamWaitEvent(st, g_pipe->in_ready[fci], 0));   // this chunk's hidden rows have arrived
     stage_mark(ST_F1, st);
     if (o.stored_exponentials) {
       // one chunk covers all tokens: leave the exponentials in the G buffer for a backward without recompute
@@ -709,6 +722,8 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
 
     ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, go, live_m, live_c, 0};
     if ((rc = launch_dhidden(co, tmWmn, di, st))) return rc;
+    if (g_pipe != nullptr && ci < (long long)g_pipe->dh_ready.size())
+      KDKL_CUDA(cudaEventRecord(g_pipe->dh_ready[ci], st));            // this chunk's dhidden rows are final
     if (gp.last) {
       // one dW pass over the group that ends here: its chunks' G rows and hidden rows are contiguous
       const long long ci0 = ci - gp.j, g_s0 = s0 - gp.row0;
@@ -869,28 +884,92 @@ int kdkl_forward_backward_host(const void* hidden, const void* weight, const int
   if (arena_bytes < A.total) return KDKL_ERR_WORKSPACE;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   uint8_t* d = reinterpret_cast<uint8_t*>(arena);
-  KDKL_CUDA(cudaMemcpyAsync(d + A.hidden, hidden, (size_t)T * H * 2, cudaMemcpyHostToDevice, st));
-  KDKL_CUDA(cudaMemcpyAsync(d + A.weight, weight, (size_t)V * H * 2, cudaMemcpyHostToDevice, st));
-  KDKL_CUDA(cudaMemcpyAsync(d + A.idx, topk_idx, (size_t)T * K * 4, cudaMemcpyHostToDevice, st));
-  KDKL_CUDA(cudaMemcpyAsync(d + A.val, topk_val, (size_t)T * K * 4, cudaMemcpyHostToDevice, st));
-  if (teacher_lse) KDKL_CUDA(cudaMemcpyAsync(d + A.lse, teacher_lse, (size_t)T * 4, cudaMemcpyHostToDevice, st));
-  if (loss_mask) KDKL_CUDA(cudaMemcpyAsync(d + A.mask, loss_mask, (size_t)T, cudaMemcpyHostToDevice, st));
+  const long long C = ws_layout(T, H, V, K, chunk, chunks_per_pass_of(opt)).C;
+  const long long n_chunks = (T + C - 1) / C;
+  const size_t dh_elem = dh32 ? 4 : 2;
+
+  // Copies that overlap the chunk loop go over a second stream: the hidden rows of chunk i upstream while the
+  // forward sweeps of earlier chunks run, the dhidden rows of chunk i downstream while later chunks are still
+  // being differentiated. With one chunk there is nothing to overlap and everything stays on the caller's stream.
+  HostPipe pipe;
+  const bool piped = n_chunks > 1;
+  auto cleanup = [&]() {
+    for (cudaEvent_t e : pipe.in_ready) cudaEventDestroy(e);
+    for (cudaEvent_t e : pipe.dh_ready) cudaEventDestroy(e);
+    if (pipe.side) cudaStreamDestroy(pipe.side);
+    g_pipe = nullptr;
+  };
+#define KDKL_PIPE(call)                                                          \
+  do {                                                                           \
+    cudaError_t e__ = (call);                                                    \
+    if (e__ != cudaSuccess) { cleanup(); return cuda_fail(#call, e__); }         \
+  } while (0)
+  if (piped) {
+    cudaEvent_t start;
+    KDKL_PIPE(cudaStreamCreateWithFlags(&pipe.side, cudaStreamNonBlocking));
+    KDKL_PIPE(cudaEventCreateWithFlags(&start, cudaEventDisableTiming));
+    pipe.in_ready.push_back(start);                       // slot 0 doubles as "the caller's stream has reached this call"
+    for (long long i = 0; i < n_chunks; ++i) {
+      cudaEvent_t a, b;
+      KDKL_PIPE(cudaEventCreateWithFlags(&a, cudaEventDisableTiming));
+      pipe.in_ready.push_back(a);
+      KDKL_PIPE(cudaEventCreateWithFlags(&b, cudaEventDisableTiming));
+      pipe.dh_ready.push_back(b);
+    }
+    // the copy stream starts where the caller's stream stands (earlier work on the arena has finished by then)
+    KDKL_PIPE(cudaEventRecord(pipe.in_ready[0], st));
+    KDKL_PIPE(cudaStreamWaitEvent(pipe.side, pipe.in_ready[0], 0));
+    cudaEventDestroy(pipe.in_ready[0]);
+    pipe.in_ready.erase(pipe.in_ready.begin());
+  }
+  KDKL_PIPE(cudaMemcpyAsync(d + A.weight, weight, (size_t)V * H * 2, cudaMemcpyHostToDevice, st));
+  KDKL_PIPE(cudaMemcpyAsync(d + A.idx, topk_idx, (size_t)T * K * 4, cudaMemcpyHostToDevice, st));
+  KDKL_PIPE(cudaMemcpyAsync(d + A.val, topk_val, (size_t)T * K * 4, cudaMemcpyHostToDevice, st));
+  if (teacher_lse) KDKL_PIPE(cudaMemcpyAsync(d + A.lse, teacher_lse, (size_t)T * 4, cudaMemcpyHostToDevice, st));
+  if (loss_mask) KDKL_PIPE(cudaMemcpyAsync(d + A.mask, loss_mask, (size_t)T, cudaMemcpyHostToDevice, st));
+  if (piped) {
+    for (long long i = 0; i < n_chunks; ++i) {
+      const long long s0 = i * C, rows = (T - s0 < C) ? (T - s0) : C;
+      KDKL_PIPE(cudaMemcpyAsync(d + A.hidden + (size_t)s0 * H * 2, reinterpret_cast<const uint8_t*>(hidden) + (size_t)s0 * H * 2,
+                                (size_t)rows * H * 2, cudaMemcpyHostToDevice, pipe.side));
+      KDKL_PIPE(cudaEventRecord(pipe.in_ready[i], pipe.side));
+    }
+    g_pipe = &pipe;
+  } else {
+    KDKL_PIPE(cudaMemcpyAsync(d + A.hidden, hidden, (size_t)T * H * 2, cudaMemcpyHostToDevice, st));
+  }
   const size_t ws_bytes = ws_layout(T, H, V, K, chunk, chunks_per_pass_of(opt)).total;
   int rc = kdkl_forward(d + A.hidden, d + A.weight, reinterpret_cast<int32_t*>(d + A.idx),
                         reinterpret_cast<float*>(d + A.val), teacher_lse ? reinterpret_cast<float*>(d + A.lse) : nullptr,
                         loss_mask ? d + A.mask : nullptr, T, H, V, K, chunk, tau, opt, d + A.ws, ws_bytes,
                         reinterpret_cast<float*>(d + A.loss), nullptr, nullptr, nullptr, cuda_stream);
-  if (rc) return rc;
+  if (rc) { cleanup(); return rc; }
   const int64_t fl = g_launches;
   rc = kdkl_backward(d + A.hidden, d + A.weight, loss_mask ? d + A.mask : nullptr, T, H, V, K, chunk, tau, opt,
                      grad_loss, d + A.ws, ws_bytes, d + A.dh, reinterpret_cast<float*>(d + A.dw), cuda_stream);
-  if (rc) return rc;
+  g_pipe = nullptr;
+  if (rc) { cleanup(); return rc; }
   g_launches += fl;
-  KDKL_CUDA(cudaMemcpyAsync(loss_out, d + A.loss, 4, cudaMemcpyDeviceToHost, st));
-  if (dhidden_out)
-    KDKL_CUDA(cudaMemcpyAsync(dhidden_out, d + A.dh, (size_t)T * H * (dh32 ? 4 : 2), cudaMemcpyDeviceToHost, st));
-  if (dweight_out) KDKL_CUDA(cudaMemcpyAsync(dweight_out, d + A.dw, (size_t)V * H * 4, cudaMemcpyDeviceToHost, st));
-  KDKL_CUDA(cudaStreamSynchronize(st));
+  KDKL_PIPE(cudaMemcpyAsync(loss_out, d + A.loss, 4, cudaMemcpyDeviceToHost, st));
+  if (dhidden_out) {
+    if (piped) {
+      // every dh_ready event has been recorded (enqueued) by kdkl_backward above, so these waits bind to them
+      for (long long i = 0; i < n_chunks; ++i) {
+        const long long s0 = i * C, rows = (T - s0 < C) ? (T - s0) : C;
+        KDKL_PIPE(cudaStreamWaitEvent(pipe.side, pipe.dh_ready[i], 0));
+        KDKL_PIPE(cudaMemcpyAsync(reinterpret_cast<uint8_t*>(dhidden_out) + (size_t)s0 * H * dh_elem,
+                                  d + A.dh + (size_t)s0 * H * dh_elem, (size_t)rows * H * dh_elem,
+                                  cudaMemcpyDeviceToHost, pipe.side));
+      }
+    } else {
+      KDKL_PIPE(cudaMemcpyAsync(dhidden_out, d + A.dh, (size_t)T * H * dh_elem, cudaMemcpyDeviceToHost, st));
+    }
+  }
+  if (dweight_out) KDKL_PIPE(cudaMemcpyAsync(dweight_out, d + A.dw, (size_t)V * H * 4, cudaMemcpyDeviceToHost, st));
+  KDKL_PIPE(cudaStreamSynchronize(st));
+  if (piped) KDKL_PIPE(cudaStreamSynchronize(pipe.side));
+#undef KDKL_PIPE
+  cleanup();
   return KDKL_OK;
 }
 
