@@ -148,12 +148,16 @@ int kdkl_backward(const void* hidden_bf16, const void* weight_bf16, const uint8_
 /* Forward and backward in one call, with three projections instead of four. The paper's backward recomputes
  * each chunk's logits (Algorithm 1, "Backward": a second output projection) because it runs as a separate
  * autograd phase; when the gradient is wanted right away - the loss is the last operation of a training step -
- * the forward sweep of a chunk can leave the unnormalised exponentials 2^(z log2e / tau - 64) in the chunk's
- * [chunk, V] bf16 buffer, and as soon as the chunk's log Z is known they are turned, in place, into
- * G = (M q - p) g / tau (Eq. "grad"). Same workspace, same peak memory, same outputs as kdkl_forward followed
- * by kdkl_backward up to one more bf16 rounding inside G. A scaled logit z log2e / tau beyond about +190 overflows
- * the stored exponential: the gradients are then not finite and kdkl_status reports KDKL_ERR_NONFINITE with the
- * row (use the two-call path for such inputs). 6 T H V flops instead of 8 T H V.
+ * the forward sweep of a chunk can leave the unnormalised exponentials e = 2^(z log2e / tau - 64) in the chunk's
+ * [chunk, V] bf16 buffer. As soon as the chunk's log Z is known, G = (M q - p) g / tau (Eq. "grad") is
+ * s_t e - b_t p with one scale s_t per token, and that scale is taken out of the two contractions instead of being
+ * written into the buffer: dhidden rows are multiplied by it in fp32, dweight is contracted against hidden rows
+ * scaled by it (rounded to bf16), and only the <= K teacher entries of a row are patched in place. Same workspace
+ * size class, same outputs as kdkl_forward followed by kdkl_backward up to two more bf16 roundings (the stored
+ * exponential; for dweight also the scaled hidden rows). Limits of the stored exponential: a scaled logit
+ * z log2e / tau beyond +192 cannot be stored (kdkl_status: KDKL_ERR_NONFINITE with the token), and a token whose log2
+ * normaliser is below -40 would lose entries to underflow (KDKL_ERR_RANGE); use the two-call path for such inputs.
+ * 6 T H V flops instead of 8 T H V.
  * Arguments as the two calls; grad_loss must be known here. The workspace afterwards holds the same saved
  * state (kdkl_saved_state, kdkl_status). Vocabulary shards need the cross-shard exchange before log Z is known:
  * there the same saving is available through option stored_exponentials when one chunk covers all tokens. */

@@ -357,7 +357,7 @@ def kdkl_profile_stages(hidden, weight, topk_idx, topk_val, workspace, loss_out,
     return {STAGES[i]: (float(ms[i]), int(nl[i])) for i in range(8)}
 
 
-STAGES_SINGLE = ["prep", "fwd_gemm_lse_exp", "combine", "loss_reduce", "bwd_coef", "exp_to_dlogits", "dhidden_gemm",
+STAGES_SINGLE = ["prep", "fwd_gemm_lse_exp", "combine", "loss_reduce", "bwd_coef", "scale_and_patch", "dhidden_gemm",
                  "dweight_gemm"]
 
 

@@ -283,6 +283,53 @@ e_to_g_kernel(__nv_bfloat16* __restrict__ G, long long ldg /* elements per row *
   }
 }
 
+// Single-pass step without a dense conversion pass. With e = 2^(s - bias) stored by the forward sweep and log Z
+// known, G = s_t e - b_t p with the row scale s_t = a_t 2^(bias - lz2_t) (Eq. "grad"). Instead of rewriting the
+// whole [chunk, V] buffer, the scale is taken out of the two contractions:
+//   dH[t,:] = s_t * (e' W)[t,:]           (applied in fp32 by the split-K fix-up)
+//   dW      = e'^T (s (.) h)              (the chunk's hidden rows scaled once: chunk x H elements)
+// with e' = e - (b_t / s_t) p at the <= K support entries of the row (patched in place). Rows without gradient
+// (a_t = 0) were stored as zeros by the sweep and get scale 0.
+__global__ void __launch_bounds__(256)
+sp_scale_kernel(const uint4* __restrict__ h, int nvec /* H / 8 */, const float* __restrict__ coefA,
+                const float* __restrict__ lz2, float bias, float* __restrict__ rs, uint4* __restrict__ hs) {
+  const long long row = blockIdx.x;
+  const float a = coefA[row];
+  const float sc = a != 0.f ? a * exp2f(bias - lz2[row]) : 0.f;
+  if (threadIdx.x == 0) rs[row] = sc;
+  for (int v = threadIdx.x; v < nvec; v += 256) {
+    uint4 x = h[row * nvec + v];
+    __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&x);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = __bfloat1622float2(h2[j]);
+      h2[j] = __floats2bfloat162_rn(f.x * sc, f.y * sc);
+    }
+    hs[row * nvec + v] = x;
+  }
+}
+
+// One warp per row: e'[t, v] = e[t, v] - (b_t / s_t) p_v at the row's support (sorted, duplicates merged by prep).
+__global__ void __launch_bounds__(256)
+sp_patch_kernel(__nv_bfloat16* __restrict__ G, long long ldg, long long rows, const float* __restrict__ rs,
+                const float* __restrict__ coefB, const int* __restrict__ idx_sorted,
+                const float* __restrict__ p_sorted, const int* __restrict__ nvalid, int Ktop) {
+  const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const float sc = rs[row];
+  if (sc == 0.f) return;
+  const float c = coefB[row] / sc;
+  const int nv = nvalid[row];
+  __nv_bfloat16* g = G + row * ldg;
+  for (int k = threadIdx.x & 31; k < nv; k += 32) {
+    const float pk = p_sorted[row * Ktop + k];
+    if (pk != 0.f) {
+      const int col = idx_sorted[row * Ktop + k];
+      g[col] = __float2bfloat16_rn(__bfloat162float(g[col]) - c * pk);
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------ live row tiles
 // live[c * tiles_per_chunk + i] = 1 when at least one token of rows [c*chunk + i*tile_rows, ... + tile_rows)
 // (clipped to the chunk and to T) is counted. The GEMM kernels skip row tiles whose flag is 0: a padding
@@ -504,11 +551,13 @@ __global__ void bwd_coef_kernel(const float* __restrict__ Mv, const uint8_t* __r
 }
 
 // ------------------------------------------------------------------------------------ split-K fix-up
-// out = part[0] + part[1] + ... in that fixed order (fp32), then one rounding to bf16 if asked.
+// out = part[0] + part[1] + ... in that fixed order (fp32), times the row's scale if given, then one rounding to
+// bf16 if asked.
 // part holds `splits` slabs `slab` elements apart; n4 = number of float4 groups to produce.
 __global__ void __launch_bounds__(256)
 splitk_fixup_kernel(const float* __restrict__ part, long long slab, int splits, long long n4,
-                    __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32, const int* go) {
+                    __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32, const int* go,
+                    const float* __restrict__ row_scale, int row_n4 /* float4 groups per row */) {
   if (go != nullptr && *go == 0) return;
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n4) return;
@@ -516,6 +565,11 @@ splitk_fixup_kernel(const float* __restrict__ part, long long slab, int splits, 
   for (int sidx = 1; sidx < splits; ++sidx) {
     const float4 b = reinterpret_cast<const float4*>(part + (long long)sidx * slab)[i];
     a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+  }
+  if (row_scale != nullptr) {                  // single-pass step: the row's scale, taken out of the contraction
+    const float sc = row_scale[i / row_n4];
+    if (sc == 0.f) a = make_float4(0.f, 0.f, 0.f, 0.f);
+    else { a.x *= sc; a.y *= sc; a.z *= sc; a.w *= sc; }
   }
   if (out_f32) reinterpret_cast<float4*>(out_f32)[i] = a;
   if (out_bf16) {

@@ -110,7 +110,8 @@ struct GemmParams {
   int* colread;              // [rows, Ktop] column actually read, sorted order
   const float* lz2;          // [rows] log2-domain log-normaliser
   int neg_a;                 // 1 when the upstream gradient is negative (coefA <= 0 for every row)
-  const float* coefA;        // [rows] g_t * M_t / tau
+  long long row_base;        // token index of row 0 of this launch (for error reports)
+  const float* coefA;        // [rows] g_t * M_t / tau (EPI_DLOGITS; EPI_LSE_E, optional: rows with 0 store zeros)
   const float* coefB;        // [rows] g_t / tau
   const float* p_sorted;     // [rows, Ktop]
   // EPI_TOPK: every logit with z * scale_log2 >= thr[row] is appended to the row's candidate list
@@ -439,6 +440,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       int cur = 0, nv = 0, next_idx = 0x7fffffff;
       const int* idxrow = nullptr;
       float row_b = 0.f, row_off = -INFINITY, row_thr = INFINITY;
+      bool row_zero = false;                   // EPI_LSE_E: a row without gradient stores zeros, not exponentials
+      if (EPI == EPI_LSE_E) { if (row_ok && p.coefA != nullptr) row_zero = p.coefA[row] == 0.f; }
       if (EPI == EPI_TOPK) { if (row_ok) row_thr = p.thr[row]; }
       if (kLse || EPI == EPI_DLOGITS) {
         if (row_ok) {
@@ -505,7 +508,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 acc_s += tj;
                 r[j] = __float_as_uint(tj);
               }
-              e_fac = ex2_approx(m_new - kExpBias);
+              e_fac = row_zero ? 0.f : ex2_approx(m_new - kExpBias);
+              // bf16 tops out just below 2^128: a scaled logit beyond bias + 128 cannot be stored
+              if (m_new - kExpBias >= 128.f && !row_zero && p.status != nullptr) {
+                atomicCAS(p.status, 0, -11);               // KDKL_ERR_NONFINITE, with the token
+                atomicCAS(p.status + 1, 0, (int)(p.row_base + row));
+              }
             } else {
 #pragma unroll
               for (int j = 0; j < 32; ++j) acc_s += ex2_approx(fmaf(__uint_as_float(r[j]), p.scale_log2, -m_new));

@@ -234,7 +234,7 @@ struct WsLayout {
   int dw_group;              // chunks whose G is kept so that one dW pass contracts over all of them (1 or 2)
   long long g_rows;          // rows of the G buffer
   size_t hdr, idx_sorted, p_sorted, perm, zg, colread, nvalid, M, Hent, lz2, logZ, loss_tok, coefA, coefB;
-  size_t part_m, part_s, G, dh_part, live, total;
+  size_t part_m, part_s, G, dh_part, live, rs, hs, total;
   static constexpr int kMaxSlabs = 24;
   int n_slabs;
   size_t slab_off[kMaxSlabs], slab_len[kMaxSlabs];   // every slab in layout order (for kdkl_workspace_layout)
@@ -289,7 +289,9 @@ static WsLayout ws_layout(long long T, long long H, long long V, int K, long lon
   L.G = take((size_t)L.g_rows * L.Vpad * 2);
   L.dh_splits = choose_k_splits(((L.C + kTileM - 1) / kTileM) * n_tiles_for(H, use_wide(H)), (V + BK - 1) / BK,
                                 sm_count_or_default());
-  L.dh_part = take(L.dh_splits > 1 ? (size_t)L.dh_splits * L.Cpad * H * 4 : 0);
+  L.dh_part = take((size_t)L.dh_splits * L.Cpad * H * 4);    // at least one slab: the single-pass step always fixes up
+  L.rs = take((size_t)T * 4);                                 // single-pass step: the row scales ...
+  L.hs = take((size_t)L.g_rows * H * 2);                      // ... and the scaled hidden rows of the group in flight
   L.tiles_per_chunk = (L.C + kTileM - 1) / kTileM;
   L.n_live = ((T + L.C - 1) / L.C) * L.tiles_per_chunk;
   L.live = take((size_t)L.n_live);
@@ -406,6 +408,7 @@ struct ChunkOut {
   const uint8_t* live_m;   // row-tile flags for the dH GEMM (nullptr: none)
   const uint8_t* live_c;   // row-tile flags of the dW contraction (nullptr: none)
   int accumulate_dw;
+  const float* row_scale;  // single-pass step: per-row scale applied by the dH fix-up (nullptr: none)
 };
 static int launch_dhidden(const ChunkOut& c, const CUtensorMap& tmWmn, const DeviceInfo& di, cudaStream_t st) {
   const WsLayout& L = *c.L;
@@ -427,7 +430,7 @@ static int launch_dhidden(const ChunkOut& c, const CUtensorMap& tmWmn, const Dev
   p2.k_splits = sp;
   __nv_bfloat16* dh16 = c.o->dhidden_dtype == 0 ? reinterpret_cast<__nv_bfloat16*>(c.dhidden) + s0 * H : nullptr;
   float* dh32 = c.o->dhidden_dtype == 1 ? reinterpret_cast<float*>(c.dhidden) + s0 * H : nullptr;
-  if (sp > 1) {
+  if (sp > 1 || c.row_scale != nullptr) {
     // partial sums of each split go to fp32 slabs [split][Cpad, H]; a fixed-order fix-up adds them
     float* part = at<float>(c.ws, L.dh_part);
     p2.split_rows = (int)L.Cpad;
@@ -437,7 +440,7 @@ static int launch_dhidden(const ChunkOut& c, const CUtensorMap& tmWmn, const Dev
     if (rc) return rc;
     const long long n4 = rows * H / 4;
     splitk_fixup_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(part, (long long)L.Cpad * H, sp, n4, dh16, dh32,
-                                                                     c.go);
+                                                                     c.go, c.row_scale, (int)(H / 4));
     KDKL_LAUNCHED("splitk_fixup_kernel");
     return KDKL_OK;
   }
@@ -720,7 +723,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
       if ((rc = launch_gemm<EPI_DLOGITS, false, false>(tmA, tmW, tmGout, p, di, st))) return rc;
     }
 
-    ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, go, live_m, live_c, 0};
+    ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, go, live_m, live_c, 0, nullptr};
     if ((rc = launch_dhidden(co, tmWmn, di, st))) return rc;
     if (g_pipe != nullptr && ci < (long long)g_pipe->dh_ready.size())
       KDKL_CUDA(cudaEventRecord(g_pipe->dh_ready[ci], st));            // this chunk's dhidden rows are final
@@ -728,7 +731,8 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
       // one dW pass over the group that ends here: its chunks' G rows and hidden rows are contiguous
       const long long ci0 = ci - gp.j, g_s0 = s0 - gp.row0;
       ChunkOut cg{Gbuf, reinterpret_cast<const __nv_bfloat16*>(hidden) + g_s0 * H, nullptr, g_s0, gp.row0 + rows, H, V,
-                  &L, &o, hdr, ws, go, nullptr, group_flags(L, live, ci0), (ci0 > 0 || o.accumulate_dweight) ? 1 : 0};
+                  &L, &o, hdr, ws, go, nullptr, group_flags(L, live, ci0), (ci0 > 0 || o.accumulate_dweight) ? 1 : 0,
+                  nullptr};
       if ((rc = launch_dweight(cg, tmdW, di, st))) return rc;
     }
   }
@@ -785,6 +789,8 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
     // F1': logits tile by tile -> online log-sum-exp partials, gathered teacher logits, and e = 2^(s - bias) into G
     GemmParams p;
     fill_forward_params(&p, L, ws, s0, rows, H, V, K, inv_tau, live_c);
+    p.coefA = at<float>(ws, L.coefA) + s0;         // rows without gradient store zeros instead of exponentials
+    p.row_base = s0;
     const uint8_t* live_m = p.m_live;
     stage_mark(ST_F1, st);
     if ((rc = launch_gemm<EPI_LSE_E, false, false>(tmA, tmW, tmGout, p, di, st))) return rc;
@@ -796,24 +802,29 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
         at<float>(ws, L.logZ), at<float>(ws, L.loss_tok), loss_per_token, nullptr, nullptr, 0, nullptr, T, hdr, 1);
     KDKL_LAUNCHED("combine_kernel");
 
-    // e -> G in place, now that the chunk's log Z is known
+    // With the chunk's log Z known: G = s_t e - b_t p. The row scale s_t leaves the contractions (the dH fix-up
+    // multiplies by it, the dW pass reads hidden rows scaled by it) and only the <= K support entries per row
+    // are patched in place: no pass over the [chunk, V] buffer.
     stage_mark(ST_B1, st);
-    const int n_cols = (int)(((V + 7) / 8) * 8);
-    const int n_seg = (n_cols + E2G_SEG - 1) / E2G_SEG;
-      if ((long long)rows * n_seg > 2147483647ll) return KDKL_ERR_SHAPE;   // one block per (row, segment)
-    e_to_g_kernel<<<(unsigned)(rows * n_seg), 256, 0, st>>>(
-        G, L.Vpad, n_cols, (int)V, at<float>(ws, L.coefA) + s0, at<float>(ws, L.coefB) + s0, at<float>(ws, L.lz2) + s0,
-        at<int>(ws, L.idx_sorted) + s0 * K, at<float>(ws, L.p_sorted) + s0 * K, at<int>(ws, L.nvalid) + s0, K, kExpBias,
-        n_seg, hdr, nullptr);
-    KDKL_LAUNCHED("e_to_g_kernel");
+    float* rs = at<float>(ws, L.rs) + s0;
+    __nv_bfloat16* hs_group = at<__nv_bfloat16>(ws, L.hs);
+    sp_scale_kernel<<<(unsigned)rows, 256, 0, st>>>(reinterpret_cast<const uint4*>(hA), (int)(H / 8),
+                                                    at<float>(ws, L.coefA) + s0, at<float>(ws, L.lz2) + s0, kExpBias, rs,
+                                                    reinterpret_cast<uint4*>(hs_group + gp.row0 * H));
+    KDKL_LAUNCHED("sp_scale_kernel");
+    sp_patch_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(
+        G, L.Vpad, rows, rs, at<float>(ws, L.coefB) + s0, at<int>(ws, L.idx_sorted) + s0 * K,
+        at<float>(ws, L.p_sorted) + s0 * K, at<int>(ws, L.nvalid) + s0, K);
+    KDKL_LAUNCHED("sp_patch_kernel");
 
-    // dH[chunk] = G W and dW (+)= G^T h, exactly as in kdkl_backward
-    ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, nullptr, live_m, live_c, 0};
+    // dH[chunk] = s (e' W) and dW (+)= e'^T (s h): the kernels of kdkl_backward, the scale applied outside them
+    ChunkOut co{G, hA, dhidden, s0, rows, H, V, &L, &o, hdr, ws, nullptr, live_m, live_c, 0, rs};
     if ((rc = launch_dhidden(co, tmWmn, di, st))) return rc;
     if (gp.last) {
       const long long ci0 = ci - gp.j, g_s0 = s0 - gp.row0;
-      ChunkOut cg{Gbuf, reinterpret_cast<const __nv_bfloat16*>(hidden) + g_s0 * H, nullptr, g_s0, gp.row0 + rows, H, V,
-                  &L, &o, hdr, ws, nullptr, nullptr, group_flags(L, live, ci0), (ci0 > 0 || o.accumulate_dweight) ? 1 : 0};
+      ChunkOut cg{Gbuf, hs_group, nullptr, g_s0, gp.row0 + rows, H, V,
+                  &L, &o, hdr, ws, nullptr, nullptr, group_flags(L, live, ci0), (ci0 > 0 || o.accumulate_dweight) ? 1 : 0,
+                  nullptr};
       if ((rc = launch_dweight(cg, tmdW, di, st))) return rc;
     }
   }

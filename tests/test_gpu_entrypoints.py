@@ -97,7 +97,8 @@ def test_profile_single_pass_accounts_for_every_stage_and_changes_nothing():
     st = B.kdkl_profile_single_pass(g["hidden"], g["weight"], g["topk_idx"], g["topk_val"], op.workspace, op.loss,
                                     op.dhidden, op.dweight, chunk=cfg.chunk, temperature=cfg.tau)
     chunks = cfg.T // cfg.chunk
-    assert st["fwd_gemm_lse_exp"][1] == chunks and st["exp_to_dlogits"][1] == chunks and st["combine"][1] == chunks
+    assert st["fwd_gemm_lse_exp"][1] == chunks and st["combine"][1] == chunks
+    assert st["scale_and_patch"][1] == chunks                # per chunk: row scales + scaled hidden rows, support patch
     assert st["dhidden_gemm"][1] == chunks and st["dweight_gemm"][1] == (chunks + 1) // 2
     assert st["prep"][1] == 1 and st["loss_reduce"][1] == 1 and "bwd_coef" not in st
     assert all(ms > 0 for ms, n in st.values())
