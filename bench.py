@@ -333,7 +333,7 @@ def mode_vocab(cfg, rank, world, dev, B, I, all_gather=None, all_reduce_sum=None
         return ev[0].elapsed_time(ev[1]) + ev[2].elapsed_time(ev[3])
     nbytes = world * 2 * cfg.T * 4 + cfg.T * cfg.H * 4
     return {"step": step, "drain": lambda: None, "loss": lambda: float(op.loss.item()),
-            "launches": lambda: B.kdkl_last_launch_count(), "tokens_per_step": cfg.T, "scaling": "strong", "op": op,
+            "launches": lambda: op.launches_total(), "tokens_per_step": cfg.T, "scaling": "strong", "op": op,
             "inputs": d, "status": op.status, "parallelism": f"vocabulary shards (tensor parallel) x{world}",
             "collective": {"what": "all-gather of [R,2,T] shard statistics, fp32 all-reduce of dHidden",
                            "bytes_per_step": nbytes}, "collective_ms": collective_ms}

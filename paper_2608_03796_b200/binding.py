@@ -507,6 +507,7 @@ class ShardedFusedChunkedKL:
         self.dweight = torch.empty(V_local, H, dtype=torch.float32, device=device)
         self._all_gather = all_gather or self._dist_all_gather
         self._all_reduce_sum = all_reduce_sum or self._dist_all_reduce
+        self._launches = [0, 0, 0]
 
     @staticmethod
     def _dist_all_gather(out, local):
@@ -522,12 +523,18 @@ class ShardedFusedChunkedKL:
         kdkl_forward_shard(hidden, weight_local, topk_idx, topk_val, self.workspace, self.stats_local,
                            vocab_offset=self.vocab_offset, V_total=self.V_total, teacher_lse=teacher_lse,
                            loss_mask=loss_mask, chunk=self.chunk, temperature=self.temperature, opt=self.opt)
+        self._launches = [kdkl_last_launch_count(), 0, 0]
 
     def forward_finish(self, loss_mask=None):
         kdkl_forward_finish(self.stats_all, self.n_shards, self.T, self.H, self.V_local, self.K, self.workspace,
                             self.loss, loss_mask=loss_mask, chunk=self.chunk, temperature=self.temperature,
                             opt=self.opt, loss_per_token=self.loss_per_token)
+        self._launches[1] = kdkl_last_launch_count()
         return self.loss
+
+    def launches_total(self) -> int:
+        """Kernels this rank's last step enqueued (local sweep + finish + backward)."""
+        return sum(self._launches)
 
     def forward(self, hidden, weight_local, topk_idx, topk_val, teacher_lse=None, loss_mask=None):
         self.forward_local(hidden, weight_local, topk_idx, topk_val, teacher_lse, loss_mask)
@@ -537,6 +544,7 @@ class ShardedFusedChunkedKL:
     def backward_local(self, hidden, weight_local, loss_mask=None, grad_loss=1.0):
         kdkl_backward(hidden, weight_local, self.K, self.workspace, self.dhidden, self.dweight, loss_mask=loss_mask,
                       chunk=self.chunk, temperature=self.temperature, opt=self.opt, grad_loss=grad_loss)
+        self._launches[2] = kdkl_last_launch_count()
 
     def backward(self, hidden, weight_local, loss_mask=None, grad_loss=1.0):
         self.backward_local(hidden, weight_local, loss_mask, grad_loss)
