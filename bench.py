@@ -46,7 +46,7 @@ FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_g
 
 # DRAM bytes (read + write) of each tensor-core kernel per chunk of 4096 tokens, from one ncu capture of the shipped
 # build on a reduced case (chunk 4096, H = 4096, V = 32768, four chunks: every operand larger than L2, 2 GB on the
-# device; profiles/dram_traffic_C4096_V32768.md). A kernel's traffic is proportional to the vocabulary rows it
+# device; its summary is kept with the other profiler summaries). A kernel's traffic is proportional to the vocabulary rows it
 # sweeps, so the figure for another V at this chunk and H is scaled by V / 32768. The dW kernel contracts over
 # two chunks per launch (reduce-add form: 2,042,949,888 B read + 504,135,936 B written per launch).
 TRAFFIC_REF = {"chunk": 4096, "H": 4096, "V": 32768,
