@@ -588,16 +588,18 @@ def main():
     peak = float(peaks.get(peak_key, FALLBACK_PEAKS[peak_key]))
     gemm_stages = ["fwd_gemm_lse", "bwd_gemm_dlogits", "dhidden_gemm", "dweight_gemm"]
 
-    if mode_name == "independent":
+    stage_check = None
+    if mode_name in ("independent", "tokens"):
         # per-kernel times, live, with an event between kernels: right after the timed region, so under the
-        # same power state, with the clocks sampled during this run as well
+        # same power state, with the clocks sampled during this run as well (token shards: this rank's own two
+        # calls, no collective inside)
         stage_acc = {}
         n_prof = 1 if args.capture else (2 if T > 65536 else 3)
         with ClockSampler(local_rank) as sclk:
             for _ in range(n_prof):
                 st = B.kdkl_profile_stages(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], op.workspace,
                                            op.loss, op.dhidden, op.dweight, loss_mask=d["mask"], chunk=cfg.chunk,
-                                           temperature=cfg.tau)
+                                           temperature=cfg.tau, opt=getattr(op, "opt", None))
                 for k, (ms, n) in st.items():
                     a = stage_acc.setdefault(k, [0.0, 0])
                     a[0] += ms
@@ -623,8 +625,9 @@ def main():
                        "sum_x_clock_ratio_over_step": (stage_sum * smhz / (clocks["sm_mhz"] * ms_step)
                                                        if (smhz and clocks["sm_mhz"]) else None)}
 
+    if mode_name == "independent":
         # the single-pass step (kdkl_forward_backward: three projections instead of four, same memory, same outputs
-        # up to one more bf16 rounding inside G), timed like the headline; reported beside it, not instead of it
+        # up to two more bf16 roundings), timed like the headline; reported beside it, not instead of it
         def step1():
             op.forward_backward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], loss_mask=d["mask"])
         sp_steps = args.steps if T <= 65536 else max(2, min(args.steps, 4))
@@ -650,8 +653,6 @@ def main():
                        "tflops_executed_per_gpu": 0.75 * cfg.flops / (sp_ms * 1e-3) / 1e12,
                        "launches_per_step": sp_launches,
                        "what": "forward + backward in one call without the second projection (6*T*H*V flops)"}
-    else:
-        stage_check = None
 
     # end to end through the host-buffer entry point (pinned host memory, copies inside the timed region); with
     # several ranks every rank runs the call on its own tokens (no collective on this leg)
