@@ -74,7 +74,8 @@ def kdkl_oracle(hidden, weight, topk_idx, topk_val, tau=1.0, mask=None, teacher_
     (default: number of counted tokens).
 
     Returns a dict with: loss, loss_tok [T] (0 at ignored rows), logZ [T] (of z/tau),
-    M [T], gathered_logits [T,K] (z at the teacher indices, unscaled; NaN at empty
+    M [T], p_k [T,K] (the teacher probability of every slot, 0 at unusable slots) and g [T] (the upstream
+    factor grad_loss * mask / N of every token), gathered_logits [T,K] (z at the teacher indices, unscaled; NaN at empty
     slots), gathered_idx [T,K], n_bad_idx, and with want_grads: dH [T,H], dW [V,H].
     """
     h = _f64(hidden)
@@ -143,7 +144,7 @@ def kdkl_oracle(hidden, weight, topk_idx, topk_val, tau=1.0, mask=None, teacher_
             dW = dWb if dW is None else dW + dWb
 
     loss = float(loss_tok.sum() / N) if N > 0 else 0.0
-    out = {"loss": loss, "loss_tok": loss_tok, "logZ": logZ, "M": M, "gathered_logits": zg,
+    out = {"loss": loss, "loss_tok": loss_tok, "logZ": logZ, "M": M, "p_k": p_k, "g": g, "gathered_logits": zg,
            "gathered_idx": np.asarray(topk_idx).astype(np.int32).copy(), "n_bad_idx": n_bad, "N": N}
     if want_grads:
         out["dH"] = dH

@@ -26,48 +26,94 @@ Two roundings (single-pass step). The first rounding is of the stored exponentia
 dense softmax part a_t q_v of an entry, not with G itself; at a support entry where the student already matches
 the teacher (M q ~ p) G is much smaller than that part, and a vocabulary row of dW made of such entries has a
 small norm with an error of ordinary size. With roundings >= 2 every row is therefore judged against at least
-the median row's scale (norm and rms), which is the scale of the dense part.
+the median row's scale (norm and rms), which is the scale of the dense part, and the relative term of the
+element-wise bound is taken on the dense part where the caller supplies it (`dense_mag`, the magnitude of the
+output computed from M q alone: |oracle + sparse part|, see sparse_parts): u * (dense_mag + 2 |oracle|) - one
+rounding of e, one of the patched entry, one of the scaled hidden row; the per-row relative error is then taken
+against the larger of the row's own norm and its dense part's.
+
+Absolute floor. The logits themselves are fp32 sums of bf16 products pushed through exp2: a relative error of about
+2^-16 on M q and on p separately. Where the two cancel almost completely the element is far below its row-mates and
+its error is set by that, not by its own size: every element is allowed 2e-5 of the largest row's rms.
 """
 import numpy as np
 
 U_BF16 = 2.0 ** -8
 C_SIGMA = 8.0
 ROW_FRO = 1e-2
+ABS_EPS = 2e-5
 
 
-def elementwise_tolerance(ref_block, out_bf16=False, roundings=1, rms_floor=0.0):
+def sparse_parts(o, hidden, weight, topk_idx, tau):
+    """The sparse teacher terms of Eq. "grad" on their own, from the oracle's per-slot probabilities p_k and
+    upstream factors g: S_H[t,:] = (g_t / tau) sum_k p_tk W[idx_tk,:] and S_W[v,:] = sum_{t,k: idx_tk = v}
+    (g_t / tau) p_tk h_t, so that oracle + S is the gradient of the dense part M q alone. float64 numpy."""
+    h = np.asarray(hidden, dtype=np.float64)
+    W = np.asarray(weight, dtype=np.float64)
+    idx = np.asarray(topk_idx).astype(np.int64)
+    T, K = idx.shape
+    V = W.shape[0]
+    coef = (o["g"][:, None] / float(tau)) * o["p_k"]                 # [T, K], 0 at unusable slots
+    ok = coef != 0
+    ii = np.where(ok, np.clip(idx, 0, V - 1), 0)
+    S_H = np.einsum("tk,tkh->th", coef, W[ii]) if T * K * W.shape[1] <= (1 << 27) else \
+        np.stack([coef[t] @ W[ii[t]] for t in range(T)])
+    S_W = np.zeros_like(W)
+    tt = np.repeat(np.arange(T), K).reshape(T, K)
+    np.add.at(S_W, ii[ok], coef[ok][:, None] * h[tt[ok]])
+    return S_H, S_W
+
+
+def dense_dweight(o, hidden, weight, topk_idx, tau):
+    """|dW| of the dense part M q alone (see sparse_parts): the `dense_mag` of a single-pass dW comparison."""
+    return np.abs(o["dW"] + sparse_parts(o, hidden, weight, topk_idx, tau)[1])
+
+
+def elementwise_tolerance(ref_block, out_bf16=False, roundings=1, rms_floor=0.0, dense_block=None, abs_floor=0.0):
     """The bound above for a block of whole rows of the oracle's matrix (float64 [rows, cols])."""
     rms = np.maximum(np.sqrt(np.mean(ref_block * ref_block, axis=1, keepdims=True)), rms_floor)
-    rel = U_BF16 * (2.0 if out_bf16 else 1.0)
-    return rel * np.abs(ref_block) + C_SIGMA * np.sqrt(float(roundings)) * (U_BF16 / np.sqrt(3.0)) * rms
+    rel = U_BF16 * ((2.0 if out_bf16 else 1.0) + (1.0 if dense_block is not None else 0.0))
+    tol = rel * np.abs(ref_block) + C_SIGMA * np.sqrt(float(roundings)) * (U_BF16 / np.sqrt(3.0)) * rms + abs_floor
+    if dense_block is not None:
+        tol = tol + U_BF16 * np.abs(dense_block)
+    return tol
 
 
-def check_grad_matrix(got, ref, name, out_bf16=False, roundings=1, row_fro=ROW_FRO, block=4096, extra_tol=None):
+def check_grad_matrix(got, ref, name, out_bf16=False, roundings=1, row_fro=ROW_FRO, block=4096, extra_tol=None,
+                      dense_mag=None, abs_scale=None):
     """got, ref: [rows, cols] (anything np.asarray takes; compared in float64, row block by row block so that a
     full-size dW does not need several float64 copies). extra_tol (scalar or [rows, cols]) is added to every
-    element's bound: the fp32 rounding of `dW +=` onto existing contents. Raises AssertionError naming the worst
-    row / element.
+    element's bound: the fp32 rounding of `dW +=` onto existing contents. dense_mag ([rows, cols], single-pass
+    step): the output of the dense part alone. abs_scale: the largest row rms of the WHOLE matrix when `ref` is only
+    some of its rows (default: taken from ref). Raises AssertionError naming the worst row / element.
     Returns (largest per-row relative error, largest elementwise error / tolerance)."""
     rows = ref.shape[0]
     assert got.shape == ref.shape, (name, got.shape, ref.shape)
     norms = np.empty(rows)
     errs = np.empty(rows)
+    dnorms = np.zeros(rows)
     worst_ratio, worst_at = 0.0, None
     norm_floor = 0.0
+    for r0 in range(0, rows, block):
+        b = np.asarray(ref[r0:r0 + block], dtype=np.float64)
+        norms[r0:r0 + len(b)] = np.sqrt((b * b).sum(axis=1))
     if roundings >= 2 and rows:
-        for r0 in range(0, rows, block):
-            b = np.asarray(ref[r0:r0 + block], dtype=np.float64)
-            norms[r0:r0 + len(b)] = np.sqrt((b * b).sum(axis=1))
         norm_floor = float(np.median(norms))
     rms_floor = norm_floor / np.sqrt(ref.shape[1])
+    if abs_scale is None:
+        abs_scale = float(norms.max()) / np.sqrt(ref.shape[1]) if rows else 0.0
+    abs_floor = ABS_EPS * abs_scale
     for r0 in range(0, rows, block):
         b = np.asarray(ref[r0:r0 + block], dtype=np.float64)
         a = np.asarray(got[r0:r0 + block], dtype=np.float64)
         assert np.isfinite(a).all(), f"{name}: non-finite values in rows {r0}..{r0 + len(a) - 1}"
         diff = np.abs(a - b)
-        norms[r0:r0 + len(b)] = np.sqrt((b * b).sum(axis=1))
         errs[r0:r0 + len(b)] = np.sqrt((diff * diff).sum(axis=1))
-        tol = elementwise_tolerance(b, out_bf16, roundings, rms_floor)
+        dense = None if dense_mag is None else np.asarray(dense_mag[r0:r0 + block], dtype=np.float64)
+        if dense is not None:
+            dnorms[r0:r0 + len(b)] = np.sqrt((dense * dense).sum(axis=1))
+        tol = elementwise_tolerance(b, out_bf16, roundings, rms_floor, dense, abs_floor)
+        tol = np.where(norms[r0:r0 + len(b), None] > 0, tol, 0.0)
         if extra_tol is not None:
             tol = tol + (extra_tol if np.ndim(extra_tol) == 0 else np.asarray(extra_tol)[r0:r0 + block])
         # rows the oracle holds as exact zeros (ignored tokens) must be exact zeros
@@ -81,13 +127,13 @@ def check_grad_matrix(got, ref, name, out_bf16=False, roundings=1, row_fro=ROW_F
                                 f"{worst_ratio:.2f} x its tolerance")
     # per-row relative Frobenius error, on every row whose norm is not negligible next to the largest
     live = norms > 1e-6 * norms.max() if rows and norms.max() > 0 else np.zeros(rows, bool)
-    rel = np.where(live, errs / np.maximum(np.where(live, norms, 1.0), norm_floor), 0.0)
+    rel = np.where(live, errs / np.maximum(np.maximum(np.where(live, norms, 1.0), norm_floor), dnorms), 0.0)
     r = int(np.argmax(rel)) if rows else 0
     assert not rows or rel[r] <= row_fro, f"{name}: row {r} relative error {rel[r]:.3e} > {row_fro:.0e}"
     return (float(rel[r]) if rows else 0.0), worst_ratio
 
 
-def check_support_rows(got_dw, ref_dw, topk_idx, tokens, name, roundings=1):
+def check_support_rows(got_dw, ref_dw, topk_idx, tokens, name, roundings=1, dense_mag=None):
     """The rows of dW at the teacher indices of the given tokens: the place where the sparse -p term of
     Eq. "grad" lands. Compared like any other rows, but named, so that a missing support correction is
     reported as such."""
@@ -96,5 +142,7 @@ def check_support_rows(got_dw, ref_dw, topk_idx, tokens, name, roundings=1):
     if not rows:
         return
     sel = np.asarray(rows)
-    check_grad_matrix(np.asarray(got_dw)[sel], np.asarray(ref_dw)[sel], f"{name} (support rows)", False, roundings,
-                      block=len(sel))
+    ref = np.asarray(ref_dw)
+    whole = float(np.sqrt((ref * ref).mean(axis=1).max()))     # the floor is set by the whole matrix, not by the selection
+    check_grad_matrix(np.asarray(got_dw)[sel], ref[sel], f"{name} (support rows)", False, roundings, block=len(sel),
+                      dense_mag=None if dense_mag is None else np.asarray(dense_mag)[sel], abs_scale=whole)

@@ -8,7 +8,7 @@ import numpy as np
 import pytest
 import torch
 
-from gradcheck import check_grad_matrix, check_support_rows
+from gradcheck import check_grad_matrix, check_support_rows, dense_dweight
 from oracle.kdkl_oracle import kdkl_oracle
 from paper_2608_03796_b200 import binding as B
 from paper_2608_03796_b200 import inputs as I
@@ -88,9 +88,11 @@ def test_single_pass_matches_oracle_and_two_call_path(T, H, V, K, chunk, tau, ma
     # row by row and element by element; G carries two bf16 roundings here (the stored exponential, then G)
     b64 = base.double().numpy() if opts.get("accumulate") else 0.0
     check_grad_matrix(dH, o["dH"], "dH", out_bf16=one.dhidden.dtype == torch.bfloat16, roundings=2)
-    check_grad_matrix(dW - b64, o["dW"], "dW", roundings=2, extra_tol=2.0 ** -22 * np.abs(b64))
+    dense = dense_dweight(o, h.double().numpy(), W.double().numpy(), idx.numpy(), tau)
+    check_grad_matrix(dW - b64, o["dW"], "dW", roundings=2, extra_tol=2.0 ** -22 * np.abs(b64), dense_mag=dense)
     cnt = np.ones(T, bool) if mask is None else mask_np != 0
-    check_support_rows(dW - b64, o["dW"], idx.numpy(), list(np.flatnonzero(cnt)[:3]), "dW", roundings=2)
+    check_support_rows(dW - b64, o["dW"], idx.numpy(), list(np.flatnonzero(cnt)[:3]), "dW", roundings=2,
+                       dense_mag=dense)
     # and close to the two-call gradients (two independent roundings of G against one)
     assert _fro(dH, two.dhidden.float().cpu().double().numpy()) <= 6e-3
     assert _fro(dW, two.dweight.cpu().double().numpy()) <= 6e-3

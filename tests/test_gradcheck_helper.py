@@ -72,3 +72,45 @@ def test_zero_rows_must_be_exact_zeros():
     got[2, 3] = 1e-9
     with pytest.raises(AssertionError):
         check_grad_matrix(got, ref, "dH", out_bf16=True)
+
+
+def test_sparse_parts_split_the_oracle_gradient():
+    """oracle + sparse part = the gradient of the dense part alone, g/tau * M * softmax(z/tau), written out here;
+    with duplicates, an empty slot, an out-of-range index and an ignored token."""
+    from gradcheck import sparse_parts, dense_dweight
+    from oracle.kdkl_oracle import kdkl_oracle
+    rng = np.random.default_rng(3)
+    T, H, V, K, tau = 6, 5, 11, 4, 1.7
+    h, W = rng.standard_normal((T, H)), rng.standard_normal((V, H))
+    idx = rng.integers(0, V, (T, K))
+    idx[0, 1] = idx[0, 0]; idx[1, 2] = -1; idx[2, 3] = V + 4
+    val = rng.standard_normal((T, K)) * 2
+    mask = np.array([1, 1, 1, 0, 1, 1], np.uint8)
+    o = kdkl_oracle(h, W, idx, val, tau=tau, mask=mask, grad_loss=-0.5, teacher_lse=np.full(T, 3.0))
+    S_H, S_W = sparse_parts(o, h, W, idx, tau)
+    s = (h @ W.T) / tau
+    q = np.exp(s - s.max(1, keepdims=True)); q /= q.sum(1, keepdims=True)
+    dz = (o["g"] / tau * o["M"])[:, None] * q
+    np.testing.assert_allclose(o["dH"] + S_H, dz @ W, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(o["dW"] + S_W, dz.T @ h, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(dense_dweight(o, h, W, idx, tau), np.abs(dz.T @ h), rtol=1e-12, atol=1e-15)
+    assert not S_H[3].any()
+
+
+def test_cancelling_support_entry_of_a_one_token_batch():
+    """T = 1: every dW row is a single product. Where M q ~ p the single-pass entry keeps the rounding error of the
+    stored exponential (u times the dense part), far above u times the net value: accepted with dense_mag,
+    refused without; an error of twice that size is refused either way."""
+    H = 64
+    hrow = np.linspace(0.5, 1.5, H)
+    dense_g = np.array([1e-3, 1e-3, 1.0, 1e-3, 1e-3])     # row 2: a confident student entry that cancels to 1e-3
+    net_g = np.array([1e-3, 1e-3, 1e-3, 1e-3, 1e-3])      # of its dense part; the other rows are dense-only
+    ref, dense = net_g[:, None] * hrow, dense_g[:, None] * hrow
+    got = ref.copy()
+    got[2] += 0.9 * 2.0 ** -8 * dense[2]
+    with pytest.raises(AssertionError):
+        check_grad_matrix(got, ref, "dW", roundings=2)
+    check_grad_matrix(got, ref, "dW", roundings=2, dense_mag=dense)
+    got[2] += 1.5 * 2.0 ** -8 * dense[2]
+    with pytest.raises(AssertionError):
+        check_grad_matrix(got, ref, "dW", roundings=2, dense_mag=dense)
