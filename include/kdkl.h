@@ -278,7 +278,7 @@ int kdkl_gemm_bf16(const void* A, const void* B, float* C, int64_t M, int64_t N,
 int kdkl_logz_noalloc(const void* hidden_bf16, const void* weight_bf16, int64_t T, int64_t H, int64_t V,
                       float temperature, float* logz_out, void* cuda_stream);
 
-#define KDKL_ERR_OVERFLOW (-12) /* teacher top-K: a row's candidate list still overflows after two rounds of a tightened
+#define KDKL_ERR_OVERFLOW (-12) /* teacher top-K: a row's candidate list still overflows after four rounds of a tightened
                                    threshold (in practice: hundreds of logits tied exactly at the K-th value) */
 
 /* The teacher cache record of the offline pipeline (paper, section "Offline Distillation with a Top-K
@@ -290,10 +290,11 @@ int kdkl_logz_noalloc(const void* hidden_bf16, const void* weight_bf16, int64_t 
  * Two tensor-core sweeps: the first gives the log-sum-exp and per-vocab-tile maxima, whose K-th largest
  * is a threshold that every member of the top-K must reach; the second recomputes the logits and keeps
  * those at or above it; a per-row sort finishes. When large logits cluster in a few vocabulary tiles (a
- * frequency-ordered vocabulary) more logits reach that threshold than a row's candidate list holds
- * (max(4 K, 256) slots, at most 1024): the K-th largest kept candidate then serves as a tighter threshold
- * and the row is scanned again, up to twice (sweeps that no row needs return at once). K <= 256, K <= V <= 2^20, H % 8 == 0, and either
- * V >= 256 K (at least K vocabulary tiles, so the threshold exists) or V <= 8192 (every logit is sorted).
+ * frequency-ordered vocabulary), or the vocabulary has fewer than K tiles of 256 columns, more logits reach that
+ * threshold than a row's candidate list holds (max(4 K, 256) slots, at most 1024; the whole vocabulary when
+ * V <= 8192): the list then keeps a uniform sample of them, the K-th largest kept candidate serves as a tighter
+ * threshold and the row is scanned again, up to four times (sweeps that no row needs return at once; each round
+ * keeps about K / slots of the candidates). K <= 256, K <= V <= 2^20, H % 8 == 0.
  * workspace: device, kdkl_teacher_topk_workspace_bytes(); its first words are a status block readable
  * with kdkl_status (KDKL_ERR_OVERFLOW / KDKL_ERR_TIMEOUT). Enqueue-only. */
 size_t kdkl_teacher_topk_workspace_bytes(int64_t T, int64_t H, int64_t V, int32_t K);

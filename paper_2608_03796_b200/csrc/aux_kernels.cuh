@@ -660,8 +660,9 @@ topk_collect_kernel(const float* __restrict__ z, long long ldz, int V, float sca
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       if (c + j < V && v[j] * scale_log2 >= t) {
-        const int slot = atomicAdd(cand_cnt + row, 1);
-        if (slot < cap) {
+        const int arrival = atomicAdd(cand_cnt + row, 1);
+        const int slot = reservoir_slot(arrival, cap, (uint32_t)row, (uint32_t)(c + j));
+        if (slot >= 0) {
           cand_idx[row * cap + slot] = c + j;
           cand_val[row * cap + slot] = v[j];
         }
@@ -674,9 +675,10 @@ topk_collect_kernel(const float* __restrict__ z, long long ldz, int V, float sca
 // threshold than the list holds - large logits clustered in a few vocabulary tiles, as in a frequency-ordered
 // vocabulary) gets a tighter threshold and is scanned again. The K-th largest of the candidates that were kept is
 // a valid one: they are real logits of the row, so at least K logits reach it and every member of the exact
-// top-K does. The kept ones are an arbitrary subset (list slots are handed out atomically), so the tightened
-// scan admits about K / cap of the previous count; the host enqueues two such rounds, each skipped on the device
-// when no row asked for it (*flag stays 0). Rows that fit keep their list and take no further candidates.
+// top-K does. The kept ones are a uniform sample of all that arrived (reservoir_slot), so the tightened scan admits
+// about K / cap of the previous count, whatever the order of arrival; the host enqueues a fixed number of such
+// rounds, each skipped on the device when no row asked for it (*flag stays 0). Rows that fit keep their list and
+// take no further candidates.
 __global__ void __launch_bounds__(32)
 topk_retighten_kernel(int* __restrict__ cand_cnt, const float* __restrict__ cand_val, int cap, int cpad, int K,
                       float scale_log2, float* __restrict__ thr, int* flag, const int* go) {

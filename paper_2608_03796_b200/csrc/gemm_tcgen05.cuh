@@ -534,8 +534,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             while (hits) {
               const int j = __ffs(hits) - 1;
               hits &= hits - 1u;
-              const int slot = atomicAdd(p.cand_cnt + row, 1);     // tiles of one row run on different SMs
-              if (slot < p.cand_cap) {
+              const int arrival = atomicAdd(p.cand_cnt + row, 1);  // tiles of one row run on different SMs
+              const int slot = reservoir_slot(arrival, p.cand_cap, (uint32_t)row, (uint32_t)(col0 + j));
+              if (slot >= 0) {
                 p.cand_idx[(long long)row * p.cand_cap + slot] = col0 + j;
                 p.cand_val[(long long)row * p.cand_cap + slot] = sel32(r, j);
               }

@@ -1106,6 +1106,7 @@ int kdkl_profile_single_pass(const void* hidden, const void* weight, const int32
 
 // ------------------------------------------------------------------ teacher top-K cache record
 constexpr long long kTopkTakeAllMaxV = 8192;
+constexpr int kTopkRounds = 4;      // tightening rounds per pass: a list of 4 K slots then copes with 4 K * 4^4 candidates
 struct TopkLayout {
   long long C, Cpad, n_tiles, ldz;
   int npad, cap, cpad;
@@ -1119,11 +1120,12 @@ static TopkLayout topk_layout(long long T, long long V, int K, bool stored = fal
   L.Cpad = (long long)up((size_t)L.C, 128);
   L.n_tiles = (V + BN - 1) / BN;
   L.npad = pow2_at_least(L.n_tiles);
-  // With at least K vocabulary tiles the threshold admits few more than K logits; with fewer tiles
-  // it says nothing, and every logit is a candidate (small vocabularies only: see kTopkTakeAllMaxV).
+  // With at least K vocabulary tiles the threshold admits few more than K logits. With fewer tiles it says nothing
+  // and every logit is a candidate: small vocabularies get a list that holds them all; larger ones start from
+  // the standard list and rely on the tightening rounds (each keeps about K / cap of the candidates).
   long long cap = 4ll * K > 256 ? 4ll * K : 256;
   if (cap > 1024) cap = 1024;
-  if (L.n_tiles < K) cap = V;
+  if (L.n_tiles < K && V <= kTopkTakeAllMaxV) cap = V;
   if (cap > V) cap = V;
   L.cap = (int)cap;
   L.cpad = pow2_at_least(L.cap);
@@ -1131,7 +1133,7 @@ static TopkLayout topk_layout(long long T, long long V, int K, bool stored = fal
   auto take = [&](size_t bytes) { size_t at = o; o = up(o + bytes, 256); return at; };
   L.hdr = take(256);
   L.n_pass = (T + L.C - 1) / L.C;
-  L.flags = take((size_t)L.n_pass * 2 * 4);                // per pass: "rescan wanted" of the two tightening rounds
+  L.flags = take((size_t)L.n_pass * kTopkRounds * 4);      // per pass: "rescan wanted" of each tightening round
   L.zeros = take((size_t)L.Cpad * 4);
   L.part_m = take((size_t)L.n_tiles * L.Cpad * 4);
   L.part_s = take((size_t)L.n_tiles * L.Cpad * 4);
@@ -1162,7 +1164,6 @@ static int teacher_topk_impl(const void* hidden, const void* weight, int64_t T, 
   if (!hidden || !weight || !ws || !topk_idx || !topk_val || !lse) return KDKL_ERR_NULL;
   if (T < 1 || H < 1 || V < 1 || K < 1 || K > 256 || K > V || (H % 8) != 0 || V > (1ll << 20) || T >= (1ll << 31))
     return KDKL_ERR_SHAPE;
-  if ((V + BN - 1) / BN < K && V > kTopkTakeAllMaxV) return KDKL_ERR_SHAPE;   // needs V >= 256 K or V <= 8192
   if (!(tau > 0.f)) return KDKL_ERR_ARG;
   if (((uintptr_t)hidden & 15) || ((uintptr_t)weight & 15) || ((uintptr_t)ws & 15)) return KDKL_ERR_ALIGN;
   const TopkLayout L = topk_layout(T, V, K, stored);
@@ -1216,15 +1217,15 @@ static int teacher_topk_impl(const void* hidden, const void* weight, int64_t T, 
       p.cand_idx = at<int>(ws, L.cidx); p.cand_val = at<float>(ws, L.cval); p.cand_cap = L.cap;
       if ((rc = launch_gemm<EPI_TOPK, false, false>(tmA, tmW, tmA, p, di, st))) return rc;
     }
-    // Lists that overflowed (more logits at or above the tile-maxima threshold than slots): up to two rounds of
-    // a tighter threshold and a new scan, each skipped on the device when no row of this pass asked for it.
+    // Lists that overflowed (more logits at or above the tile-maxima threshold than slots): rounds of a tighter
+    // threshold and a new scan, each skipped on the device when no row of this pass asked for it.
     if (L.cap < V) {
-      int* flags = at<int>(ws, L.flags) + 2 * pass;
+      int* flags = at<int>(ws, L.flags) + kTopkRounds * pass;
       KDKL_CUDA(cudaFuncSetAttribute(topk_retighten_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.cpad * 4));
-      for (int round = 0; round < 2; ++round) {
+      for (int round = 0; round < kTopkRounds; ++round) {
         topk_retighten_kernel<<<(unsigned)rows, 32, (size_t)L.cpad * 4, st>>>(
             at<int>(ws, L.cnt), at<float>(ws, L.cval), L.cap, L.cpad, K, p.scale_log2, at<float>(ws, L.thr),
-            flags + round, round == 0 ? nullptr : flags);
+            flags + round, round == 0 ? nullptr : flags + round - 1);
         KDKL_LAUNCHED("topk_retighten_kernel");
         if (stored) {
           const int n_seg = (int)((V + COLLECT_SEG - 1) / COLLECT_SEG);

@@ -242,4 +242,17 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
   return d;
 }
 
+// ---------------------------------------------------------------- shared by the top-K candidate collectors
+// A candidate that arrives when its row's list is full replaces a pseudo-random kept one with probability
+// cap / (arrivals so far): the kept candidates stay a uniform sample of all that arrived, whatever the order in
+// which vocabulary tiles are visited (an overflowed list only serves to pick a tighter threshold). Returns the slot
+// to write, or -1.
+__device__ __forceinline__ int reservoir_slot(int arrival, int cap, uint32_t row, uint32_t col) {
+  if (arrival < cap) return arrival;
+  uint32_t x = row * 0x9E3779B1u ^ (col + 0x7F4A7C15u) * 0x85EBCA77u ^ (uint32_t)arrival * 0xC2B2AE3Du;
+  x ^= x >> 15; x *= 0x2C1B3C6Du; x ^= x >> 12; x *= 0x297A2D39u; x ^= x >> 15;
+  const uint32_t r = x % (uint32_t)(arrival + 1);
+  return r < (uint32_t)cap ? (int)r : -1;
+}
+
 }  // namespace kdkl

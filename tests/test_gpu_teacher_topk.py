@@ -105,6 +105,14 @@ def test_large_logits_clustered_in_a_few_tiles(stored):
     _check(h, W, K, 1.0, stored)
 
 
+@pytest.mark.parametrize("stored", [False, True])
+def test_vocabulary_with_fewer_tiles_than_k(stored):
+    """V = 20000 is 79 tiles of 256 columns, fewer than K = 128: the tile maxima give no threshold, every logit is a
+    candidate, and the record comes out of the tightening rounds alone (20000 -> about 5000 -> 1250 -> 310)."""
+    h, W = _case(260, 64, 20000, seed=91)
+    _check(h, W, 128, 1.0, stored)
+
+
 def test_cache_feeds_the_loss_with_exact_retained_mass():
     """Teacher kernel -> cache record -> fused loss with teacher_lse: the paper's un-renormalised M < 1 path,
     end to end on the GPU, against the oracles fed with their own (fp64) cache."""
