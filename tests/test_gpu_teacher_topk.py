@@ -113,6 +113,13 @@ def test_vocabulary_with_fewer_tiles_than_k(stored):
     _check(h, W, 128, 1.0, stored)
 
 
+@pytest.mark.parametrize("T,H,V,K", [(48, 64, 1 << 20, 256),      # the largest vocabulary and K the call takes
+                                     (130, 64, 65000, 256)])       # 254 tiles < K: 65000 -> 16250 -> 4062 -> 1015
+def test_limits_of_vocabulary_and_k(T, H, V, K):
+    h, W = _case(T, H, V, seed=V % 1000 + K)
+    _check(h, W, K, 1.0, False)
+
+
 def test_cache_feeds_the_loss_with_exact_retained_mass():
     """Teacher kernel -> cache record -> fused loss with teacher_lse: the paper's un-renormalised M < 1 path,
     end to end on the GPU, against the oracles fed with their own (fp64) cache."""
