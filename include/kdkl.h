@@ -85,6 +85,11 @@ typedef struct kdkl_options {
                                  H = 3072: 74.9 against 77.0 ms. Same results up to fp32 reassociation in dweight.
                                  kdkl_workspace_bytes must be given the same options as the calls.
                                  A struct of a previous size (without this field) is accepted */
+  const float* grad_loss_device; /* NULL, or a DEVICE pointer to one float read when the kernels run: the upstream
+                                 gradient dL_total/dloss, in place of the grad_loss argument of kdkl_backward,
+                                 kdkl_forward_backward and the host-record step (the argument is then ignored). For
+                                 callers that hold the upstream gradient on the device (an autograd engine): no
+                                 host read. A struct of a previous size (without this field) is accepted */
 } kdkl_options;
 
 /* Number of counted tokens of a batch (mask = 1; T when loss_mask is NULL), written as one double to
@@ -136,7 +141,7 @@ int kdkl_forward(const void* hidden_bf16, const void* weight_bf16, const int32_t
  * memory, form G = (M q - p) g / tau in registers, then dhidden = G W and dweight += G^T h.
  * Same hidden / weight / mask / shape / chunk / temperature / opt as the forward call, and the
  * workspace that call filled.
- *   grad_loss  d(total)/d(loss_out), usually 1
+ *   grad_loss  d(total)/d(loss_out), usually 1 (ignored when kdkl_options.grad_loss_device is set)
  *   dhidden    [T, H] bf16 (or fp32, see options); rows of ignored tokens are exact zeros
  *   dweight    [V, H] fp32
  */

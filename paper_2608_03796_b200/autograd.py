@@ -4,9 +4,13 @@
                             chunk=4096, temperature=1.0)
     loss.backward()          # hidden.grad [T,H] bf16, weight.grad [V,H] bf16 (rounded from the fp32 dW)
 
-Marshalling only: forward runs kdkl_forward, backward runs kdkl_backward with the upstream gradient
-as `grad_loss`; nothing of the loss arithmetic happens in torch ops. The upstream gradient of a scalar
-loss is read to the host once (`grad.item()`), since the C entry point takes it as a plain float.
+Marshalling only: forward runs kdkl_forward, backward runs kdkl_backward; nothing of the loss arithmetic
+happens in torch ops. Neither call waits for the device: the upstream gradient stays where autograd holds it
+(kdkl_options.grad_loss_device), and the device status of a step (a bounded wait that ran out, a state mismatch)
+is copied to pinned host memory behind the step's kernels and looked at when the same buffers are next used, or
+by check_status() - an error of step i is therefore raised during step i+1. `sync_status=True` reads the status
+at the end of backward instead (one stream synchronisation per step). The single-pass form compares the upstream
+gradient with `expected_grad` on the host and so reads it once (`grad.item()`).
 Workspace and gradient buffers are pooled per shape, so repeated steps allocate nothing. A forward call takes a
 buffer set out of the pool and owns it until its backward has run: two losses of one shape that are both alive
 (loss1 + loss2, pipelined micro-batches, activation checkpointing) therefore never share the saved state of
@@ -24,11 +28,44 @@ import torch
 from . import binding as B
 
 _free: dict = {}          # key -> buffer sets (FusedChunkedKL holders) no live loss is using
+_probed: list = []        # buffer sets whose last step's status has not been looked at yet
 
 
 def clear_cache() -> None:
     """Drops the pooled workspaces and gradient buffers (sets in use by a live loss are unaffected)."""
+    check_status()
     _free.clear()
+
+
+def _probe(op) -> None:
+    """Enqueue a copy of the workspace header's status words to pinned host memory behind the step's kernels."""
+    if getattr(op, "probe", None) is None:
+        op.probe = torch.zeros(4, dtype=torch.int32).pin_memory()
+        op.probe_event = torch.cuda.Event()
+    op.probe.copy_(op.workspace[:16].view(torch.int32), non_blocking=True)
+    op.probe_event.record()
+    if not getattr(op, "probe_pending", False):
+        op.probe_pending = True
+        _probed.append(op)
+
+
+def _collect(op) -> None:
+    """Look at the status a finished earlier step left (waits for that step's kernels only if they still run)."""
+    if not getattr(op, "probe_pending", False):
+        return
+    op.probe_event.synchronize()
+    op.probe_pending = False
+    if op in _probed:
+        _probed.remove(op)
+    code, where = int(op.probe[0]), int(op.probe[1])
+    if code not in (0, -10):                                      # -10: out-of-range teacher indices were ignored
+        raise B.KdklError(code, f"device status of an earlier fused_chunked_kl step, detail {where}")
+
+
+def check_status() -> None:
+    """Raises if any step whose status has not been looked at yet failed on the device (waits for those steps)."""
+    for op in list(_probed):
+        _collect(op)
 
 
 def _acquire(T, H, V, K, chunk, tau, accumulate, device):
@@ -37,6 +74,7 @@ def _acquire(T, H, V, K, chunk, tau, accumulate, device):
     pool = _free.setdefault(key, [])
     if pool:
         op = pool.pop()
+        _collect(op)                                              # the status its last step left
         if op.dweight is None:                                    # handed over to a caller last time
             op.dweight = torch.empty(V, H, dtype=torch.float32, device=device)
     else:
@@ -54,7 +92,7 @@ def _release(key, op) -> None:
 class _FusedChunkedKL(torch.autograd.Function):
     @staticmethod
     def forward(ctx, hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, chunk, temperature, dweight_out,
-                weight_grad_fp32, single_pass, expected_grad):
+                weight_grad_fp32, single_pass, expected_grad, sync_status):
         T, H = hidden.shape
         V, K = weight.shape[0], topk_idx.shape[1]
         # single pass: the gradients for an upstream gradient of 1 come out of the forward call (three projections
@@ -73,7 +111,7 @@ class _FusedChunkedKL(torch.autograd.Function):
             _release(key, op)                                     # no backward will come: the set is free again
             return loss
         ctx.op, ctx.key, ctx.generation, ctx.mask = op, key, op.generation, loss_mask
-        ctx.dweight_out, ctx.weight_grad_fp32 = dweight_out, weight_grad_fp32
+        ctx.dweight_out, ctx.weight_grad_fp32, ctx.sync_status = dweight_out, weight_grad_fp32, bool(sync_status)
         ctx.save_for_backward(hidden, weight)
         return loss
 
@@ -84,18 +122,21 @@ class _FusedChunkedKL(torch.autograd.Function):
         if op.generation != ctx.generation:
             raise RuntimeError("fused_chunked_kl: this loss's saved state has been reused by a later forward call "
                                "(backward ran twice without retain_graph semantics the buffers can honour)")
-        gl = float(grad.item())
-        if not (ctx.done and gl == ctx.expected):                 # any other upstream gradient: the recompute path
+        if not (ctx.done and float(grad.item()) == ctx.expected):   # any other upstream gradient: the recompute path
             if ctx.dweight_out is not None:
                 saved, op.dweight = op.dweight, ctx.dweight_out   # dW += into the caller's fp32 buffer
-            try:
-                op.backward(hidden, weight, loss_mask=ctx.mask, grad_loss=gl)
+            try:                                                  # the upstream gradient stays on the device
+                op.backward(hidden, weight, loss_mask=ctx.mask,
+                            grad_loss=grad.detach().to(torch.float32).contiguous())
             finally:
                 if ctx.dweight_out is not None:
                     op.dweight = saved
-        code, detail = op.status()
-        if code not in (0, -10):                                  # -10: out-of-range teacher indices were ignored
-            raise B.KdklError(code, f"device status, detail {detail}")
+        if ctx.sync_status:
+            code, detail = op.status()
+            if code not in (0, -10):                              # -10: out-of-range teacher indices were ignored
+                raise B.KdklError(code, f"device status, detail {detail}")
+        else:
+            _probe(op)
         if ctx.dweight_out is not None:
             dW = None
         elif ctx.weight_grad_fp32:
@@ -104,19 +145,19 @@ class _FusedChunkedKL(torch.autograd.Function):
             dW = op.dweight.to(weight.dtype)
         dH = op.dhidden.clone()
         _release(ctx.key, op)          # free for the next forward; a second backward of this graph before that
-        return dH, dW, None, None, None, None, None, None, None, None, None, None   # still finds its state intact
+        return dH, dW, None, None, None, None, None, None, None, None, None, None, None   # still finds its state intact
 
 
 def fused_chunked_kl(hidden, weight, topk_idx, topk_val, teacher_lse: Optional[torch.Tensor] = None,
                      loss_mask: Optional[torch.Tensor] = None, chunk: int = 4096, temperature: float = 1.0,
                      dweight_out: Optional[torch.Tensor] = None, weight_grad_fp32: bool = False,
-                     single_pass: bool = False, expected_grad: float = 1.0) -> torch.Tensor:
+                     single_pass: bool = False, expected_grad: float = 1.0, sync_status: bool = False) -> torch.Tensor:
     """Mean forward KL between the cached top-K teacher and softmax(hidden @ weight.T / temperature).
     single_pass=True computes the gradients during the forward call (kdkl_forward_backward) for an upstream
     gradient of `expected_grad` (the weight this loss carries in the total); if backward then sees another
     value, the gradients are recomputed by kdkl_backward."""
     return _FusedChunkedKL.apply(hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, chunk, temperature,
-                                 dweight_out, weight_grad_fp32, single_pass, expected_grad)
+                                 dweight_out, weight_grad_fp32, single_pass, expected_grad, sync_status)
 
 
 class _FeatureLoss(torch.autograd.Function):

@@ -47,7 +47,8 @@ class kdkl_options(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_int32), ("teacher_mode", ctypes.c_int32),
                 ("accumulate_dweight", ctypes.c_int32), ("dhidden_dtype", ctypes.c_int32),
                 ("denom_override", ctypes.c_float), ("stored_exponentials", ctypes.c_int32),
-                ("denom_device", ctypes.c_void_p), ("dw_chunks_per_pass", ctypes.c_int32)]
+                ("denom_device", ctypes.c_void_p), ("dw_chunks_per_pass", ctypes.c_int32),
+                ("grad_loss_device", ctypes.c_void_p)]
 
 
 _lib = None
@@ -177,7 +178,20 @@ def make_options(teacher_mode=0, accumulate_dweight=0, dhidden_dtype=0, denom_ov
     if denom_device is not None:
         ptr = _dptr(denom_device, torch.float64, (1,), "denom_device").value
     return kdkl_options(ctypes.sizeof(kdkl_options), teacher_mode, accumulate_dweight, dhidden_dtype, denom_override,
-                        stored_exponentials, ptr, dw_chunks_per_pass)
+                        stored_exponentials, ptr, dw_chunks_per_pass, None)
+
+
+def _grad_args(opt: Optional[kdkl_options], grad_loss):
+    """grad_loss as a number travels by value; as a CUDA float32 tensor of one element it stays on the device
+    (kdkl_options.grad_loss_device: no host read) - the options are copied with the pointer set."""
+    if not isinstance(grad_loss, torch.Tensor):
+        return opt, float(grad_loss)
+    out = kdkl_options()
+    if opt is not None:
+        ctypes.memmove(ctypes.byref(out), ctypes.byref(opt), ctypes.sizeof(kdkl_options))
+    out.struct_size = ctypes.sizeof(kdkl_options)
+    out.grad_loss_device = _dptr(grad_loss.reshape(1), _F32, (1,), "grad_loss").value
+    return out, 0.0
 
 
 def kdkl_count_tokens(loss_mask: Optional[torch.Tensor], T: int, count_out: torch.Tensor) -> None:
@@ -228,6 +242,7 @@ def kdkl_backward(hidden, weight, K, workspace, dhidden, dweight, *, loss_mask=N
     T, H = hidden.shape
     V = weight.shape[0]
     dh_dtype = _F32 if (opt is not None and opt.dhidden_dtype == 1) else _BF16
+    opt, grad_loss = _grad_args(opt, grad_loss)
     _check(lib().kdkl_backward(_dptr(hidden, _BF16, (T, H), "hidden"), _dptr(weight, _BF16, (V, H), "weight"),
                                _dptr(loss_mask, _U8, (T,), "loss_mask"), T, H, V, K, chunk, temperature,
                                _opt_ptr(opt), grad_loss, _dptr(workspace, _U8, None, "workspace"), workspace.numel(),
@@ -243,6 +258,7 @@ def kdkl_forward_backward(hidden, weight, topk_idx, topk_val, workspace, loss_ou
     V = weight.shape[0]
     K = topk_idx.shape[1]
     dh_dtype = _F32 if (opt is not None and opt.dhidden_dtype == 1) else _BF16
+    opt, grad_loss = _grad_args(opt, grad_loss)
     _check(lib().kdkl_forward_backward(
         _dptr(hidden, _BF16, (T, H), "hidden"), _dptr(weight, _BF16, (V, H), "weight"),
         _dptr(topk_idx, _I32, (T, K), "topk_idx"), _dptr(topk_val, _F32, (T, K), "topk_val"),

@@ -31,6 +31,8 @@ struct WsHeader {
   long long chunk;   // tokens per chunk of the forward call that filled the workspace
   int g_state;       // what the [chunk, V] buffer holds after forward: G_NONE, G_EXPONENTIALS (option
                      // stored_exponentials: backward converts them once), G_CONSUMED (they have been converted)
+  int neg_grad;      // 1 when the upstream gradient of the backward call in flight is negative (the recompute
+                     // GEMM carries |a_t| in the exponent and needs the sign separately)
 };
 enum { G_NONE = 0, G_EXPONENTIALS = 1, G_CONSUMED = 2 };
 
@@ -49,7 +51,7 @@ __global__ void header_reset_kernel(WsHeader* hdr) {
   if (threadIdx.x == 0 && blockIdx.x == 0) {
     hdr->status = 0; hdr->where = 0; hdr->magic = 0; hdr->go = 0;
     hdr->n_bad_idx = 0; hdr->n_tokens = 0; hdr->denom = 0.f; hdr->loss_sum = 0.0;
-    hdr->chunk = 0; hdr->g_state = G_NONE;
+    hdr->chunk = 0; hdr->g_state = G_NONE; hdr->neg_grad = 0;
   }
 }
 
@@ -203,11 +205,14 @@ count_tokens_kernel(const uint8_t* __restrict__ mask, long long T, float denom_o
 }
 
 // a_t = g_t M_t / tau, b_t = g_t / tau with g_t = grad_loss * mask_t / N (Eq. "grad"), from the header's divisor.
+// grad_dev: the upstream gradient on the device (nullptr: grad_loss).
 __global__ void step_coef_kernel(const float* __restrict__ Mv, const uint8_t* __restrict__ mask, long long T,
-                                 float grad_loss, float inv_tau, float* __restrict__ coefA,
-                                 float* __restrict__ coefB, const WsHeader* __restrict__ hdr) {
+                                 float grad_loss, const float* __restrict__ grad_dev, float inv_tau,
+                                 float* __restrict__ coefA, float* __restrict__ coefB,
+                                 const WsHeader* __restrict__ hdr) {
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= T) return;
+  if (grad_dev != nullptr) grad_loss = *grad_dev;
   const float denom = hdr->denom;
   const bool counted = mask == nullptr || mask[t] != 0;
   const float g = (counted && denom > 0.f) ? grad_loss / denom : 0.f;
@@ -525,9 +530,10 @@ loss_reduce_kernel(const float* __restrict__ loss_tok, const uint8_t* __restrict
 // nothing the verdict depends on is written by this grid.
 __global__ void bwd_coef_kernel(const float* __restrict__ Mv, const uint8_t* __restrict__ mask, long long T,
                                 long long H, long long V, int K, long long chunk, float tau, int want_exponentials,
-                                float grad_loss, float inv_tau, float* __restrict__ coefA,
-                                float* __restrict__ coefB, WsHeader* hdr) {
+                                float grad_loss, const float* __restrict__ grad_dev, float inv_tau,
+                                float* __restrict__ coefA, float* __restrict__ coefB, WsHeader* hdr) {
   __shared__ int sm_ok;
+  if (grad_dev != nullptr) grad_loss = *grad_dev;      // the upstream gradient lives on the device
   if (threadIdx.x == 0) {
     bool ok = hdr->magic == KDKL_MAGIC && hdr->T == T && hdr->H == H && hdr->V == V && hdr->K == K &&
               hdr->chunk == chunk && hdr->tau == tau;
@@ -538,6 +544,7 @@ __global__ void bwd_coef_kernel(const float* __restrict__ Mv, const uint8_t* __r
   const bool state_ok = sm_ok != 0;
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     hdr->go = state_ok ? 1 : 0;
+    hdr->neg_grad = grad_loss < 0.f ? 1 : 0;
     if (!state_ok) atomicCAS(&hdr->status, 0, -9);
   }
   if (!state_ok) return;

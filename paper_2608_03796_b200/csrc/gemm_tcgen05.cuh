@@ -109,7 +109,7 @@ struct GemmParams {
   float* zg;                 // [rows, Ktop] gathered logits, sorted order
   int* colread;              // [rows, Ktop] column actually read, sorted order
   const float* lz2;          // [rows] log2-domain log-normaliser
-  int neg_a;                 // 1 when the upstream gradient is negative (coefA <= 0 for every row)
+  const int* neg_a;          // device flag: 1 when the upstream gradient is negative (coefA <= 0 for every row)
   long long row_base;        // token index of row 0 of this launch (for error reports)
   const float* coefA;        // [rows] g_t * M_t / tau (EPI_DLOGITS; EPI_LSE_E, optional: rows with 0 store zeros)
   const float* coefB;        // [rows] g_t / tau
@@ -443,6 +443,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       bool row_zero = false;                   // EPI_LSE_E: a row without gradient stores zeros, not exponentials
       if (EPI == EPI_LSE_E) { if (row_ok && p.coefA != nullptr) row_zero = p.coefA[row] == 0.f; }
       if (EPI == EPI_TOPK) { if (row_ok) row_thr = p.thr[row]; }
+      const bool neg_a = EPI == EPI_DLOGITS && p.neg_a != nullptr && *p.neg_a != 0;   // uniform over the call
       if (kLse || EPI == EPI_DLOGITS) {
         if (row_ok) {
           idxrow = p.idx_sorted + (long long)row * p.Ktop;
@@ -574,7 +575,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               float g[32];
 #pragma unroll
               for (int j = 0; j < 32; ++j) g[j] = ex2_approx(fmaf(__uint_as_float(r[j]), p.scale_log2, row_off));
-              if (p.neg_a) {                   // uniform: the whole call has a negative upstream gradient
+              if (neg_a) {                     // the whole call has a negative upstream gradient
 #pragma unroll
                 for (int j = 0; j < 32; ++j) g[j] = -g[j];
               }

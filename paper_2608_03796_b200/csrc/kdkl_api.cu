@@ -299,16 +299,17 @@ static WsLayout ws_layout(long long T, long long H, long long V, int K, long lon
   return L;
 }
 
-// Options of this or of an earlier struct size (without dw_chunks_per_pass; without denom_device; without
-// stored_exponentials) are accepted.
+// Options of this or of an earlier struct size (without grad_loss_device; without dw_chunks_per_pass; without
+// denom_device; without stored_exponentials) are accepted.
 static int copy_options(const kdkl_options* opt, kdkl_options* eff) {
   memset(eff, 0, sizeof(*eff));
   if (!opt) return KDKL_OK;
   constexpr int32_t kSize1 = (int32_t)offsetof(kdkl_options, stored_exponentials);
   constexpr int32_t kSize2 = (int32_t)(offsetof(kdkl_options, stored_exponentials) + sizeof(int32_t));
   constexpr int32_t kSize3 = (int32_t)(offsetof(kdkl_options, denom_device) + sizeof(const double*));
+  constexpr int32_t kSize4 = (int32_t)offsetof(kdkl_options, grad_loss_device);
   if (opt->struct_size != (int32_t)sizeof(kdkl_options) && opt->struct_size != kSize1 && opt->struct_size != kSize2 &&
-      opt->struct_size != kSize3)
+      opt->struct_size != kSize3 && opt->struct_size != kSize4)
     return KDKL_ERR_ARG;
   memcpy(eff, opt, (size_t)opt->struct_size);
   eff->struct_size = (int32_t)sizeof(kdkl_options);
@@ -663,8 +664,9 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
 
   stage_mark(ST_COEF, st);
   bwd_coef_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(at<float>(ws, L.M), loss_mask, T, H, V, K, L.C, tau,
-                                                               o.stored_exponentials, grad_loss, inv_tau,
-                                                               at<float>(ws, L.coefA), at<float>(ws, L.coefB), hdr);
+                                                               o.stored_exponentials, grad_loss,
+                                                               o.grad_loss_device, inv_tau, at<float>(ws, L.coefA),
+                                                               at<float>(ws, L.coefB), hdr);
   KDKL_LAUNCHED("bwd_coef_kernel");
 
   __nv_bfloat16* Gbuf = at<__nv_bfloat16>(ws, L.G);
@@ -702,7 +704,7 @@ int kdkl_backward(const void* hidden, const void* weight, const uint8_t* loss_ma
     p.lz2 = at<float>(ws, L.lz2) + s0;
     p.coefA = at<float>(ws, L.coefA) + s0;
     p.coefB = at<float>(ws, L.coefB) + s0;
-    p.neg_a = grad_loss < 0.f ? 1 : 0;
+    p.neg_a = &hdr->neg_grad;          // written by bwd_coef_kernel above
     // dead row tiles of G are written as zeros without being computed (up to MAX_LIVE_M row tiles per chunk)
     const uint8_t* live_m = (live_c && p.m_tiles <= MAX_LIVE_M) ? live_c : nullptr;
     p.m_live = live_m;
@@ -765,8 +767,9 @@ int kdkl_forward_backward(const void* hidden, const void* weight, const int32_t*
   // the divisor of the mean and the per-token gradient coefficients are needed before the first chunk here
   count_tokens_kernel<<<1, 1024, 0, st>>>(loss_mask, T, o.denom_override, o.denom_device, hdr, nullptr);
   KDKL_LAUNCHED("count_tokens_kernel");
-  step_coef_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(at<float>(ws, L.M), loss_mask, T, grad_loss, inv_tau,
-                                                                at<float>(ws, L.coefA), at<float>(ws, L.coefB), hdr);
+  step_coef_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(at<float>(ws, L.M), loss_mask, T, grad_loss,
+                                                                o.grad_loss_device, inv_tau, at<float>(ws, L.coefA),
+                                                                at<float>(ws, L.coefB), hdr);
   KDKL_LAUNCHED("step_coef_kernel");
 
   __nv_bfloat16* Gbuf = at<__nv_bfloat16>(ws, L.G);

@@ -102,3 +102,80 @@ def test_two_live_losses_of_one_shape_do_not_share_state():
         assert _fro(h1.grad.float().cpu().double().numpy(), o1["dH"]) <= 1e-2
         assert _fro(h2.grad.float().cpu().double().numpy(), o2["dH"]) <= 1e-2
         assert _fro(W.grad.float().cpu().double().numpy(), o1["dW"] + o2["dW"]) <= 1e-2
+
+
+def test_backward_keeps_the_upstream_gradient_on_the_device_and_does_not_wait():
+    """The two-call path with a negative upstream gradient (-0.5 * loss): the value reaches the kernels through
+    kdkl_options.grad_loss_device, its sign through the workspace header. With torch's synchronisation check set to
+    raise, a whole step (forward, backward, the status probe) must not contain a blocking call."""
+    from paper_2608_03796_b200 import autograd as A
+    dev = torch.device("cuda:0")
+    cfg = I.CONFIGS["c1"]
+    d = I.make_inputs(cfg, device=dev)
+    o = kdkl_oracle(d["hidden"].cpu().double().numpy(), d["weight"].cpu().double().numpy(),
+                    d["topk_idx"].cpu().numpy(), d["topk_val"].cpu().numpy(), tau=cfg.tau, grad_loss=-0.5)
+    for step in range(2):                                   # the second step reuses pooled buffers and collects the probe
+        h = d["hidden"].clone().requires_grad_(True)
+        W = d["weight"].clone().requires_grad_(True)
+        scale = torch.full((), -0.5, device=dev)
+        torch.cuda.set_sync_debug_mode("error")
+        try:
+            loss = fused_chunked_kl(h, W, d["topk_idx"], d["topk_val"], chunk=cfg.chunk, temperature=cfg.tau)
+            (scale * loss).backward()
+        finally:
+            torch.cuda.set_sync_debug_mode("default")
+        assert _fro(h.grad.float().cpu().double().numpy(), o["dH"]) <= 1e-2
+        assert _fro(W.grad.float().cpu().double().numpy(), o["dW"]) <= 1e-2
+    A.check_status()
+
+
+def test_a_failed_step_is_reported_when_its_status_is_collected():
+    """Deferred status: the header of the workspace is wiped between forward and backward, so backward finds no
+    saved state (KDKL_ERR_STATE) and writes nothing. loss.backward() itself does not wait and does not raise;
+    check_status() - or the next step on the same buffers - does. With sync_status=True backward raises at once."""
+    from paper_2608_03796_b200 import autograd as A
+    from paper_2608_03796_b200 import binding as B
+    dev = torch.device("cuda:0")
+    cfg = I.CONFIGS["c1"]
+    d = I.make_inputs(cfg, device=dev)
+    A.clear_cache()
+    for sync in (False, True):
+        h = d["hidden"].clone().requires_grad_(True)
+        W = d["weight"].clone().requires_grad_(True)
+        loss = fused_chunked_kl(h, W, d["topk_idx"], d["topk_val"], chunk=cfg.chunk, temperature=cfg.tau,
+                                sync_status=sync)
+        loss.grad_fn.op.workspace[:64].zero_()
+        if sync:
+            with pytest.raises(B.KdklError) as e:
+                loss.backward()
+        else:
+            loss.backward()
+            with pytest.raises(B.KdklError) as e:
+                A.check_status()
+            A.check_status()                                # reported once
+        assert e.value.code == -9
+    A.clear_cache()
+
+
+def test_device_side_upstream_gradient_equals_the_by_value_argument_bitwise():
+    from paper_2608_03796_b200 import binding as B
+    dev = torch.device("cuda:0")
+    cfg = I.CONFIGS["c1"]
+    d = I.make_inputs(cfg, device=dev)
+    op = B.FusedChunkedKL(cfg.T, cfg.H, cfg.V, cfg.K, chunk=cfg.chunk, temperature=cfg.tau, device=dev,
+                          opt=B.make_options(dhidden_dtype=1))
+    for g in (1.0, -0.75, 3.0):
+        op.forward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"])
+        op.backward(d["hidden"], d["weight"], grad_loss=g)
+        want = (op.dhidden.clone(), op.dweight.clone())
+        op.dhidden.fill_(float("nan")); op.dweight.fill_(float("nan"))
+        op.backward(d["hidden"], d["weight"], grad_loss=torch.full((1,), g, device=dev))
+        assert op.status()[0] == 0
+        assert torch.equal(op.dhidden, want[0]) and torch.equal(op.dweight, want[1])
+        op.forward_backward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"], grad_loss=g)
+        want = (op.dhidden.clone(), op.dweight.clone())
+        op.dhidden.fill_(float("nan")); op.dweight.fill_(float("nan"))
+        op.forward_backward(d["hidden"], d["weight"], d["topk_idx"], d["topk_val"],
+                            grad_loss=torch.full((), g, device=dev))
+        assert op.status()[0] == 0
+        assert torch.equal(op.dhidden, want[0]) and torch.equal(op.dweight, want[1])

@@ -40,8 +40,9 @@ def test_sizes_without_a_gpu():
 
 def test_options_struct_layout():
     o = binding.make_options(teacher_mode=1, denom_override=3.0)
-    assert o.struct_size == 40 and o.teacher_mode == 1 and o.denom_override == 3.0 and o.stored_exponentials == 0
+    assert o.struct_size == 48 and o.teacher_mode == 1 and o.denom_override == 3.0 and o.stored_exponentials == 0
     assert o.denom_device is None and binding.kdkl_options.denom_device.offset == 24
+    assert o.grad_loss_device is None and binding.kdkl_options.grad_loss_device.offset == 40
 
 
 def test_host_side_argument_checks_without_a_gpu():
@@ -68,6 +69,9 @@ def test_host_side_argument_checks_without_a_gpu():
     old_size = binding.make_options()
     old_size.struct_size = 20                     # the struct before stored_exponentials was added is still accepted
     assert fwd(opt=binding._opt_ptr(old_size), wsb=ws - 1) == -4
+    for size in (24, 32, 40):                     # ... and so are the later, shorter layouts
+        old_size.struct_size = size
+        assert fwd(opt=binding._opt_ptr(old_size), wsb=ws - 1) == -4
     # stored exponentials need one chunk over all tokens
     assert fwd(opt=binding._opt_ptr(binding.make_options(stored_exponentials=1)), chunk=32) == -5
     assert fwd(opt=binding._opt_ptr(binding.make_options(stored_exponentials=2))) == -5
