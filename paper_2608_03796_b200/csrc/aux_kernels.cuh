@@ -526,8 +526,8 @@ loss_reduce_kernel(const float* __restrict__ loss_tok, const uint8_t* __restrict
 // Also checks that the workspace was filled by a forward call of the same shape, chunk size and temperature,
 // and - when backward is to convert stored exponentials instead of projecting again - that forward left
 // them and no earlier backward has converted them already (the conversion is in place: it can run once;
-// e_to_g_kernel marks them consumed). Block 0 records the verdict in `go` for the kernels that follow;
-// nothing the verdict depends on is written by this grid.
+// e_to_g_kernel marks them consumed). Block 0 records the decision in `go` for the kernels that follow;
+// nothing the decision depends on is written by this grid.
 __global__ void bwd_coef_kernel(const float* __restrict__ Mv, const uint8_t* __restrict__ mask, long long T,
                                 long long H, long long V, int K, long long chunk, float tau, int want_exponentials,
                                 float grad_loss, const float* __restrict__ grad_dev, float inv_tau,
