@@ -24,3 +24,11 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _library_is_built():
+    """The C-ABI library is compiled (or found up to date with its sources) once per session: a fresh
+    checkout carries sources only, and the tests must exercise the library built from exactly those."""
+    import __graft_entry__ as entry
+    entry.build()
