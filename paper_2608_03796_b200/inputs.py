@@ -113,6 +113,11 @@ CONFIGS = {
     "prof2": Config("prof2", T=16384, H=4096, V=32768, K=100, chunk=4096),
     "c5": Config("c5", T=32768, H=3072, V=128256, K=100, chunk=2048, tau=2.0,
                  idx_dist="zipf", tok_offset=False, packed_docs=8, pad_frac=0.05),
+    # a ragged large head (hidden 2880 = 11.25 x 256, vocabulary 201088 = 785.5 x 256: the last tile of every GEMM is
+    # partial in both directions) with a token count that leaves a short last chunk and an odd chunk out of the
+    # pairs one dW pass covers; packing mask as in c5
+    "c6": Config("c6", T=20000, H=2880, V=201088, K=100, chunk=4096,
+                 idx_dist="zipf", packed_docs=5, pad_frac=0.03),
 }
 
 

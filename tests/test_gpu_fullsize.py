@@ -37,7 +37,7 @@ def _run(cfg, d, mask, opt=None, lse=None, want_tok=True):
 
 
 @pytest.mark.parametrize("name,n_rows,partial_mass", [("c2", 48, False), ("c2", 32, True), ("c3", 48, False),
-                                                      ("c5", 64, False), ("c4c", 32, False)])
+                                                      ("c5", 64, False), ("c4c", 32, False), ("c6", 48, True)])
 def test_fullsize_sampled_parity(name, n_rows, partial_mass):
     cfg = I.CONFIGS[name]
     dev = torch.device("cuda:0")
@@ -56,7 +56,7 @@ def test_fullsize_sampled_parity(name, n_rows, partial_mass):
     mR = None if mask is None else mask[Rd].cpu().numpy()
     lseR = None if lse is None else lse[Rd].cpu().double().numpy()
     counted = np.ones(len(R), bool) if mR is None else mR != 0
-    if name == "c5":
+    if name in ("c5", "c6"):
         assert (~counted).any() and counted.any()          # the sample must see ignored rows too
 
     # ---- rows of the full run: per-token outputs and dH, with the full run's denominator
@@ -114,7 +114,7 @@ def test_fullsize_sampled_parity(name, n_rows, partial_mass):
     del oR, dW_sub
 
     # ---- additivity over a disjoint split of the mask: N dW = |R| dW_R + (N - |R|) dW_rest
-    if name in ("c2", "c5"):
+    if name in ("c2", "c5", "c6"):
         base = torch.ones(cfg.T, dtype=torch.uint8, device=dev) if mask is None else mask
         rest_mask = base & (1 - mR_full)
         sub_dW = sub.dweight.clone()
