@@ -144,6 +144,11 @@ def _dptr(t: Optional[torch.Tensor], dtype=None, shape=None, name="tensor"):
         return None
     if not t.is_cuda:
         raise TypeError(f"kdkl: {name}: expected a CUDA tensor, got a tensor on {t.device}")
+    if t.device.index != torch.cuda.current_device():
+        # the library launches on the current device and stream: a pointer into another GPU's memory would reach
+        # a kernel (and a tensor map) as it is
+        raise TypeError(f"kdkl: {name}: tensor on {t.device}, but the current device is "
+                        f"cuda:{torch.cuda.current_device()} (one process per GPU: torch.cuda.set_device first)")
     if not t.is_contiguous():
         raise TypeError(f"kdkl: {name}: expected a contiguous tensor")
     if dtype is not None and t.dtype not in (dtype if isinstance(dtype, tuple) else (dtype,)):

@@ -194,3 +194,13 @@ def test_stored_exponentials_report_rows_below_their_range():
     assert op.status()[0] == 0 and torch.isfinite(op.dweight).all()
     op.forward_backward(h, W, idx, val)
     assert op.status()[0] == -13
+
+
+def test_tensor_on_another_device_than_the_current_one_is_refused(monkeypatch):
+    """The library launches on the current device: a tensor that lives elsewhere must be refused by the binding
+    before its address reaches a kernel (shown with one GPU by making the current device look like another)."""
+    t = torch.zeros(8, device="cuda:0")
+    assert B._dptr(t).value == t.data_ptr()
+    monkeypatch.setattr(torch.cuda, "current_device", lambda: 1)
+    with pytest.raises(TypeError):
+        B._dptr(t)
