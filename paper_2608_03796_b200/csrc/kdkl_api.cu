@@ -57,6 +57,31 @@ static void stage_mark(int stage, cudaStream_t st) {
   g_timer.stage.push_back(stage);
 }
 
+static void stage_timer_start() {
+  g_timer.on = true;
+  g_timer.ev.clear();
+  g_timer.stage.clear();
+}
+// Closes the event list, waits for the stream and adds the time between consecutive events to the earlier one's stage.
+static int stage_timer_finish(int rc, cudaStream_t st, float* stage_ms, int32_t* stage_launches) {
+  stage_mark(ST_END, st);
+  g_timer.on = false;
+  cudaError_t e = cudaStreamSynchronize(st);
+  for (int i = 0; i < ST_COUNT; ++i) { stage_ms[i] = 0.f; stage_launches[i] = 0; }
+  for (size_t i = 0; e == cudaSuccess && i + 1 < g_timer.ev.size(); ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, g_timer.ev[i], g_timer.ev[i + 1]) == cudaSuccess) {
+      stage_ms[g_timer.stage[i]] += ms;
+      stage_launches[g_timer.stage[i]] += 1;
+    }
+  }
+  for (cudaEvent_t ev : g_timer.ev) cudaEventDestroy(ev);
+  g_timer.ev.clear();
+  g_timer.stage.clear();
+  if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
+  return rc;
+}
+
 // ------------------------------------------------------------------ host-buffer pipeline
 // Set (per thread) only while kdkl_forward_backward_host runs its two calls: the hidden rows of chunk i arrive on a
 // copy stream (the forward sweep of chunk i waits for in_ready[i]), and chunk i's dhidden rows leave on it as soon
@@ -1047,9 +1072,7 @@ int kdkl_profile_stages(const void* hidden, const void* weight, const int32_t* t
                         int32_t* stage_launches) {
   if (!stage_ms || !stage_launches) return KDKL_ERR_NULL;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  g_timer.on = true;
-  g_timer.ev.clear();
-  g_timer.stage.clear();
+  stage_timer_start();
   int rc = kdkl_forward(hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, T, H, V, K, chunk, tau, opt, ws,
                         ws_bytes, loss_out, nullptr, nullptr, nullptr, cuda_stream);
   const int64_t fl = g_launches;
@@ -1057,22 +1080,7 @@ int kdkl_profile_stages(const void* hidden, const void* weight, const int32_t* t
     rc = kdkl_backward(hidden, weight, loss_mask, T, H, V, K, chunk, tau, opt, grad_loss, ws, ws_bytes, dhidden,
                        dweight, cuda_stream);
   g_launches += fl;
-  stage_mark(ST_END, st);
-  g_timer.on = false;
-  cudaError_t e = cudaStreamSynchronize(st);
-  for (int i = 0; i < ST_COUNT; ++i) { stage_ms[i] = 0.f; stage_launches[i] = 0; }
-  for (size_t i = 0; e == cudaSuccess && i + 1 < g_timer.ev.size(); ++i) {
-    float ms = 0.f;
-    if (cudaEventElapsedTime(&ms, g_timer.ev[i], g_timer.ev[i + 1]) == cudaSuccess) {
-      stage_ms[g_timer.stage[i]] += ms;
-      stage_launches[g_timer.stage[i]] += 1;
-    }
-  }
-  for (cudaEvent_t ev : g_timer.ev) cudaEventDestroy(ev);
-  g_timer.ev.clear();
-  g_timer.stage.clear();
-  if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
-  return rc;
+  return stage_timer_finish(rc, st, stage_ms, stage_launches);
 }
 
 // Same measurement for the single-pass step. Stage 5 is the in-place conversion of the stored exponentials
@@ -1084,27 +1092,10 @@ int kdkl_profile_single_pass(const void* hidden, const void* weight, const int32
                              float* stage_ms, int32_t* stage_launches) {
   if (!stage_ms || !stage_launches) return KDKL_ERR_NULL;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
-  g_timer.on = true;
-  g_timer.ev.clear();
-  g_timer.stage.clear();
+  stage_timer_start();
   int rc = kdkl_forward_backward(hidden, weight, topk_idx, topk_val, teacher_lse, loss_mask, T, H, V, K, chunk, tau,
                                  opt, grad_loss, ws, ws_bytes, loss_out, nullptr, dhidden, dweight, cuda_stream);
-  stage_mark(ST_END, st);
-  g_timer.on = false;
-  cudaError_t e = cudaStreamSynchronize(st);
-  for (int i = 0; i < ST_COUNT; ++i) { stage_ms[i] = 0.f; stage_launches[i] = 0; }
-  for (size_t i = 0; e == cudaSuccess && i + 1 < g_timer.ev.size(); ++i) {
-    float ms = 0.f;
-    if (cudaEventElapsedTime(&ms, g_timer.ev[i], g_timer.ev[i + 1]) == cudaSuccess) {
-      stage_ms[g_timer.stage[i]] += ms;
-      stage_launches[g_timer.stage[i]] += 1;
-    }
-  }
-  for (cudaEvent_t ev : g_timer.ev) cudaEventDestroy(ev);
-  g_timer.ev.clear();
-  g_timer.stage.clear();
-  if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
-  return rc;
+  return stage_timer_finish(rc, st, stage_ms, stage_launches);
 }
 
 // ------------------------------------------------------------------ teacher top-K cache record
