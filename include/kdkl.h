@@ -342,6 +342,14 @@ int kdkl_feature_loss(const void* student_bf16, const void* teacher_bf16, const 
                       int32_t accumulate, void* workspace, size_t workspace_bytes, float* loss_out,
                       float* loss_per_token, void* dstudent_bf16, void* cuda_stream);
 
+/* kdkl_feature_loss with the upstream gradient read on the device when the kernels run (one float; for
+ * callers such as an autograd engine that hold it there: no host read). Always three kernels. Otherwise as above;
+ * KDKL_ERR_NULL when grad_loss_device is NULL. */
+int kdkl_feature_loss_device_grad(const void* student_bf16, const void* teacher_bf16, const uint8_t* loss_mask,
+                                  int64_t T, int64_t H, int32_t kind, float weight, const float* grad_loss_device,
+                                  float denom_override, int32_t accumulate, void* workspace, size_t workspace_bytes,
+                                  float* loss_out, float* loss_per_token, void* dstudent_bf16, void* cuda_stream);
+
 /* The same record with one projection instead of two: the first sweep also stores the fp32 logits of the pass
  * (4096 tokens at a time) and the candidates are collected from them instead of being recomputed. Costs
  * 4096 x V x 4 bytes more workspace (2 GiB at V = 131072); same results, same limits, same errors. */

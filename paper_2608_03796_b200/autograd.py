@@ -166,22 +166,20 @@ class _FeatureLoss(torch.autograd.Function):
         T, H = student.shape
         ws = torch.empty(B.kdkl_feature_loss_workspace_bytes(T), dtype=torch.uint8, device=student.device)
         loss = torch.zeros(1, dtype=torch.float32, device=student.device)
-        grad = torch.empty_like(student)
-        # loss and d loss / d student come out of the same pass, for an upstream gradient of 1
-        B.kdkl_feature_loss(student, teacher, ws, loss, kind=kind, loss_mask=loss_mask, weight=weight, dstudent=grad)
-        ctx.save_for_backward(student, teacher, grad, ws)
+        B.kdkl_feature_loss(student, teacher, ws, loss, kind=kind, loss_mask=loss_mask, weight=weight)   # loss only
+        ctx.save_for_backward(student, teacher, ws)
         ctx.args = (loss_mask, kind, weight)
         return loss.squeeze(0)
 
     @staticmethod
     def backward(ctx, g):
-        student, teacher, grad, ws = ctx.saved_tensors
-        gl = float(g.item())
-        if gl != 1.0:                              # any other upstream gradient: one more pass of the kernel
-            loss_mask, kind, weight = ctx.args
-            scratch = torch.zeros(1, dtype=torch.float32, device=student.device)
-            B.kdkl_feature_loss(student, teacher, ws, scratch, kind=kind, loss_mask=loss_mask, weight=weight,
-                                grad_loss=gl, dstudent=grad)
+        # one more pass of the same kernel writes grad * d loss / d student; the upstream gradient stays on the device
+        student, teacher, ws = ctx.saved_tensors
+        loss_mask, kind, weight = ctx.args
+        grad = torch.empty_like(student)
+        scratch = torch.zeros(1, dtype=torch.float32, device=student.device)
+        B.kdkl_feature_loss(student, teacher, ws, scratch, kind=kind, loss_mask=loss_mask, weight=weight,
+                            grad_loss=g.detach().to(torch.float32).contiguous(), dstudent=grad)
         return grad, None, None, None, None
 
 

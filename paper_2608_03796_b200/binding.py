@@ -28,7 +28,7 @@ EXPORTS = [
     "kdkl_host_arena_bytes", "kdkl_forward_backward_host", "kdkl_profile_stages", "kdkl_gemm_bf16", "kdkl_last_error",
     "kdkl_last_launch_count", "kdkl_logz_noalloc", "kdkl_forward_shard", "kdkl_forward_finish",
     "kdkl_wait_selftest", "kdkl_teacher_topk", "kdkl_teacher_topk_workspace_bytes",
-    "kdkl_feature_loss", "kdkl_feature_loss_workspace_bytes", "kdkl_step_host_record", "kdkl_record_staging_bytes",
+    "kdkl_feature_loss", "kdkl_feature_loss_device_grad", "kdkl_feature_loss_workspace_bytes", "kdkl_step_host_record", "kdkl_record_staging_bytes",
     "kdkl_forward_backward", "kdkl_profile_single_pass", "kdkl_teacher_topk_stored",
     "kdkl_teacher_topk_stored_workspace_bytes", "kdkl_workspace_layout", "kdkl_count_tokens",
     "kdkl_debug_guard_bytes",
@@ -121,6 +121,8 @@ def lib() -> ctypes.CDLL:
     L.kdkl_feature_loss_workspace_bytes.argtypes = [i64]
     L.kdkl_feature_loss.restype = ctypes.c_int
     L.kdkl_feature_loss.argtypes = [vp, vp, vp, i64, i64, i32, f32, f32, f32, i32, vp, sz, vp, vp, vp, vp]
+    L.kdkl_feature_loss_device_grad.restype = ctypes.c_int
+    L.kdkl_feature_loss_device_grad.argtypes = [vp, vp, vp, i64, i64, i32, f32, vp, f32, i32, vp, sz, vp, vp, vp, vp]
     L.kdkl_wait_selftest.restype = ctypes.c_int
     L.kdkl_wait_selftest.argtypes = [vp, i64, vp]
     L.kdkl_last_error.restype = ctypes.c_char_p
@@ -433,8 +435,17 @@ def kdkl_feature_loss_workspace_bytes(T) -> int:
 
 def kdkl_feature_loss(student, teacher, workspace, loss_out, *, kind=FEATURE_MSE, loss_mask=None, weight=1.0,
                       grad_loss=1.0, denom_override=0.0, accumulate=0, loss_per_token=None, dstudent=None) -> None:
-    """Hidden-state feature loss (MSE or cosine) and its gradient in one pass; see include/kdkl.h."""
+    """Hidden-state feature loss (MSE or cosine) and its gradient in one pass; see include/kdkl.h.
+    grad_loss: a number, or a CUDA float32 tensor of one element that is read on the device."""
     T, H = student.shape
+    if isinstance(grad_loss, torch.Tensor):
+        _check(lib().kdkl_feature_loss_device_grad(
+            _dptr(student, _BF16, (T, H), "student"), _dptr(teacher, _BF16, (T, H), "teacher"),
+            _dptr(loss_mask, _U8, (T,), "loss_mask"), T, H, kind, weight,
+            _dptr(grad_loss.reshape(1), _F32, (1,), "grad_loss"), denom_override, accumulate,
+            _dptr(workspace, _U8, None, "workspace"), workspace.numel(), _dptr(loss_out, _F32, (1,), "loss_out"),
+            _dptr(loss_per_token, _F32, (T,), "loss_per_token"), _dptr(dstudent, _BF16, (T, H), "dstudent"), _stream()))
+        return
     _check(lib().kdkl_feature_loss(_dptr(student, _BF16, (T, H), "student"), _dptr(teacher, _BF16, (T, H), "teacher"),
                                    _dptr(loss_mask, _U8, (T,), "loss_mask"), T, H, kind, weight, grad_loss,
                                    denom_override, accumulate, _dptr(workspace, _U8, None, "workspace"),

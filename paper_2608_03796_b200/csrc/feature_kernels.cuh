@@ -27,8 +27,10 @@ struct FeatHeader {
 // N = sum of the mask (or T), then the two scales every row needs. One block.
 __global__ void __launch_bounds__(1024)
 feature_count_kernel(const uint8_t* __restrict__ mask, long long T, float weight, float grad_loss,
+                     const float* __restrict__ grad_dev /* the upstream gradient on the device, or nullptr */,
                      float denom_override, FeatHeader* __restrict__ hdr) {
   __shared__ long long part[32];
+  if (grad_dev != nullptr) grad_loss = *grad_dev;
   long long c = 0;
   if (mask) {
     for (long long t = threadIdx.x; t < T; t += 1024) c += mask[t] != 0;

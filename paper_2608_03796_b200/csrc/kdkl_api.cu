@@ -1261,11 +1261,15 @@ static size_t feature_ws_bytes(long long T) { return up(256 + sizeof(float) * (s
 
 size_t kdkl_feature_loss_workspace_bytes(int64_t T) { return feature_ws_bytes(T); }
 
-int kdkl_feature_loss(const void* student, const void* teacher, const uint8_t* loss_mask, int64_t T, int64_t H,
-                      int32_t kind, float weight, float grad_loss, float denom_override, int32_t accumulate,
-                      void* workspace, size_t workspace_bytes, float* loss_out, float* loss_per_token, void* dstudent,
-                      void* cuda_stream) {
+}  // extern "C"
+
+// grad_dev: the upstream gradient on the device (then grad_loss is ignored), or nullptr.
+static int feature_loss_impl(const void* student, const void* teacher, const uint8_t* loss_mask, int64_t T, int64_t H,
+                             int32_t kind, float weight, float grad_loss, const float* grad_dev, float denom_override,
+                             int32_t accumulate, void* workspace, size_t workspace_bytes, float* loss_out,
+                             float* loss_per_token, void* dstudent, void* cuda_stream) {
   g_launches = 0;
+  if (grad_dev != nullptr) grad_loss = 1.0f;
   if (!student || !teacher || !workspace || !loss_out) return KDKL_ERR_NULL;
   if (T < 1 || H < 1 || (H % 8) != 0 || T >= (1ll << 31) || H >= (1ll << 31)) return KDKL_ERR_SHAPE;
   if (kind != KDKL_FEATURE_MSE && kind != KDKL_FEATURE_COSINE) return KDKL_ERR_ARG;
@@ -1285,9 +1289,9 @@ int kdkl_feature_loss(const void* student, const void* teacher, const uint8_t* l
   const FeatHeader* hdr = nullptr;
   FeatHeader direct;
   memset(&direct, 0, sizeof(direct));
-  if (loss_mask) {
+  if (loss_mask || grad_dev) {
     hdr = at<FeatHeader>(workspace, 0);
-    feature_count_kernel<<<1, 1024, 0, st>>>(loss_mask, T, weight, grad_loss, denom_override,
+    feature_count_kernel<<<1, 1024, 0, st>>>(loss_mask, T, weight, grad_loss, grad_dev, denom_override,
                                              at<FeatHeader>(workspace, 0));
     KDKL_LAUNCHED("feature_count_kernel");
   } else {
@@ -1322,6 +1326,25 @@ int kdkl_feature_loss(const void* student, const void* teacher, const uint8_t* l
   feature_reduce_kernel<<<1, 1024, 0, st>>>(tok, T, hdr, direct, loss_out);
   KDKL_LAUNCHED("feature_reduce_kernel");
   return KDKL_OK;
+}
+
+extern "C" {
+
+int kdkl_feature_loss(const void* student, const void* teacher, const uint8_t* loss_mask, int64_t T, int64_t H,
+                      int32_t kind, float weight, float grad_loss, float denom_override, int32_t accumulate,
+                      void* workspace, size_t workspace_bytes, float* loss_out, float* loss_per_token, void* dstudent,
+                      void* cuda_stream) {
+  return feature_loss_impl(student, teacher, loss_mask, T, H, kind, weight, grad_loss, nullptr, denom_override,
+                           accumulate, workspace, workspace_bytes, loss_out, loss_per_token, dstudent, cuda_stream);
+}
+
+int kdkl_feature_loss_device_grad(const void* student, const void* teacher, const uint8_t* loss_mask, int64_t T,
+                                  int64_t H, int32_t kind, float weight, const float* grad_loss_device,
+                                  float denom_override, int32_t accumulate, void* workspace, size_t workspace_bytes,
+                                  float* loss_out, float* loss_per_token, void* dstudent, void* cuda_stream) {
+  if (!grad_loss_device) return KDKL_ERR_NULL;
+  return feature_loss_impl(student, teacher, loss_mask, T, H, kind, weight, 1.0f, grad_loss_device, denom_override,
+                           accumulate, workspace, workspace_bytes, loss_out, loss_per_token, dstudent, cuda_stream);
 }
 
 // ------------------------------------------------------------------ bounded-wait self-test

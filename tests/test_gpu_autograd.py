@@ -114,6 +114,8 @@ def test_backward_keeps_the_upstream_gradient_on_the_device_and_does_not_wait():
     d = I.make_inputs(cfg, device=dev)
     o = kdkl_oracle(d["hidden"].cpu().double().numpy(), d["weight"].cpu().double().numpy(),
                     d["topk_idx"].cpu().numpy(), d["topk_val"].cpu().numpy(), tau=cfg.tau, grad_loss=-0.5)
+    r = I.teacher_hidden(cfg, device=dev)
+    of = feature_loss_oracle(d["hidden"].cpu().double().numpy(), r.cpu().double().numpy(), KIND_COSINE, weight=0.3)
     for step in range(2):                                   # the second step reuses pooled buffers and collects the probe
         h = d["hidden"].clone().requires_grad_(True)
         W = d["weight"].clone().requires_grad_(True)
@@ -121,10 +123,11 @@ def test_backward_keeps_the_upstream_gradient_on_the_device_and_does_not_wait():
         torch.cuda.set_sync_debug_mode("error")
         try:
             loss = fused_chunked_kl(h, W, d["topk_idx"], d["topk_val"], chunk=cfg.chunk, temperature=cfg.tau)
-            (scale * loss).backward()
+            total = scale * loss + 2.0 * feature_loss(h, r, kind=KIND_COSINE, weight=0.3)   # the recommended pair
+            total.backward()
         finally:
             torch.cuda.set_sync_debug_mode("default")
-        assert _fro(h.grad.float().cpu().double().numpy(), o["dH"]) <= 1e-2
+        assert _fro(h.grad.float().cpu().double().numpy(), o["dH"] + 2.0 * of["dS"]) <= 1e-2
         assert _fro(W.grad.float().cpu().double().numpy(), o["dW"]) <= 1e-2
     A.check_status()
 

@@ -170,3 +170,19 @@ def test_adds_onto_the_kl_gradient():
     total = op.loss.item() + floss.item()
     assert abs(total - (ok["loss"] + of["loss"])) <= 1e-3 * abs(ok["loss"] + of["loss"])
     assert _fro(op.dhidden.float().cpu().double().numpy(), ok["dH"] + of["dS"]) <= 1e-2
+
+
+@pytest.mark.parametrize("kind", [KIND_MSE, KIND_COSINE])
+@pytest.mark.parametrize("masked", [False, True])
+def test_upstream_gradient_read_on_the_device_gives_the_same_bits(kind, masked):
+    """kdkl_feature_loss_device_grad: the gradient factor comes from device memory instead of the argument list;
+    loss, per-token values and gradient must be those of the by-value call, with and without a mask (without one the
+    by-value call takes N on the host and the device-gradient call counts it on the device)."""
+    dev = torch.device("cuda:0")
+    T, H = 300, 264
+    s, r = _pair(T, H, seed=5)
+    mask = (torch.arange(T) % 5 != 0).to(torch.uint8) if masked else None
+    for g in (1.0, -2.5):
+        a = _run(s, r, kind, dev, mask=mask, weight=0.6, grad_loss=g)
+        b = _run(s, r, kind, dev, mask=mask, weight=0.6, grad_loss=torch.full((1,), g, device=dev))
+        assert a[0] == b[0] and np.array_equal(a[1], b[1]) and np.array_equal(a[2], b[2])
