@@ -33,8 +33,10 @@ _probed: list = []        # buffer sets whose last step's status has not been lo
 
 def clear_cache() -> None:
     """Drops the pooled workspaces and gradient buffers (sets in use by a live loss are unaffected)."""
-    check_status()
-    _free.clear()
+    try:
+        check_status()
+    finally:
+        _free.clear()
 
 
 def _probe(op) -> None:
@@ -64,8 +66,14 @@ def _collect(op) -> None:
 
 def check_status() -> None:
     """Raises if any step whose status has not been looked at yet failed on the device (waits for those steps)."""
-    for op in list(_probed):
-        _collect(op)
+    first = None
+    for op in list(_probed):                   # every pending status is collected, the first failure is raised
+        try:
+            _collect(op)
+        except B.KdklError as e:
+            first = first or e
+    if first is not None:
+        raise first
 
 
 def _acquire(T, H, V, K, chunk, tau, accumulate, device):
