@@ -75,9 +75,13 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
             float* __restrict__ Hent, WsHeader* hdr) {
   extern __shared__ uint8_t prep_smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  int* keys = reinterpret_cast<int*>(prep_smem) + warp * Kpad;
-  float* pv = reinterpret_cast<float*>(prep_smem + sizeof(int) * PREP_WARPS * Kpad) + warp * Kpad;
-  uint16_t* slot = reinterpret_cast<uint16_t*>(prep_smem + 2 * sizeof(int) * PREP_WARPS * Kpad) + warp * Kpad;
+  // One 64-bit word per entry is sorted: (key << 16) | slot. The probabilities stay where their slot put them and
+  // are looked up through the slot afterwards, so a compare-exchange moves 8 bytes, not three arrays; equal indices
+  // come out in slot order, which fixes the order their probabilities are added in.
+  unsigned long long* ks = reinterpret_cast<unsigned long long*>(prep_smem) + warp * Kpad;
+  float* pv = reinterpret_cast<float*>(prep_smem + sizeof(unsigned long long) * PREP_WARPS * Kpad) + warp * Kpad;
+  auto key_of = [&](int j) { return (int)(ks[j] >> 16); };
+  auto p_of = [&](int j) { return pv[(int)(ks[j] & 0xffffu)]; };
 
   const long long t = (long long)blockIdx.x * PREP_WARPS + warp;
   if (t >= T) return;
@@ -106,7 +110,8 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
         u = topk_val[t * K + k] * inv_tau;
       } else if (id >= V_total) bad++;
     }
-    keys[k] = key; pv[k] = u; slot[k] = (uint16_t)k;
+    ks[k] = ((unsigned long long)(unsigned)key << 16) | (unsigned)k;
+    pv[k] = u;
     mx = fmaxf(mx, u);
   }
   bad = (int)warp_sum((float)bad);
@@ -124,21 +129,17 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
     lam = mx + logf(s);
   }
   __syncwarp();
-  for (int k = lane; k < Kpad; k += 32) pv[k] = keys[k] < kKeyUnusable ? expf(pv[k] - lam) : 0.f;
+  for (int k = lane; k < Kpad; k += 32) pv[k] = key_of(k) < kKeyUnusable ? expf(pv[k] - lam) : 0.f;
   __syncwarp();
-  // bitonic sort by key, (p, slot) carried along
+  // bitonic sort of the (key, slot) words
   for (int size = 2; size <= Kpad; size <<= 1) {
     for (int stride = size >> 1; stride > 0; stride >>= 1) {
       for (int i = lane; i < (Kpad >> 1); i += 32) {
         const int lo = 2 * i - (i & (stride - 1));
         const int hi = lo + stride;
         const bool up = (lo & size) == 0;
-        const int a = keys[lo], b = keys[hi];
-        if ((a > b) == up) {
-          keys[lo] = b; keys[hi] = a;
-          const float pa = pv[lo]; pv[lo] = pv[hi]; pv[hi] = pa;
-          const uint16_t sa = slot[lo]; slot[lo] = slot[hi]; slot[hi] = sa;
-        }
+        const unsigned long long a = ks[lo], b = ks[hi];
+        if ((a > b) == up) { ks[lo] = b; ks[hi] = a; }
       }
       __syncwarp();
     }
@@ -146,17 +147,17 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
   // merge duplicate indices into the head of each run (scatter-add semantics). Shared memory is only
   // read from here on, so lanes may run ahead of each other.
   auto merged_p = [&](int j) -> float {
-    const int key = keys[j];
-    if (key >= kKeyUnusable || (j > 0 && keys[j - 1] == key)) return 0.f;
-    float pj = pv[j];
-    for (int q = j + 1; q < Kpad && keys[q] == key; ++q) pj += pv[q];
+    const int key = key_of(j);
+    if (key >= kKeyUnusable || (j > 0 && key_of(j - 1) == key)) return 0.f;
+    float pj = p_of(j);
+    for (int q = j + 1; q < Kpad && key_of(q) == key; ++q) pj += p_of(q);
     return pj;
   };
   // M, Hent, and the number of entries below / inside this rank's vocabulary window [v0, v0 + V)
   float msum = 0.f, hsum = 0.f;
   int lo = 0, hi = 0;
   for (int j = lane; j < Kpad; j += 32) {
-    const int key = keys[j];
+    const int key = key_of(j);
     if (key < kKeyUnusable) {
       if (key < v0) lo++;
       if (key < v0 + V) hi++;
@@ -171,12 +172,12 @@ prep_kernel(const int* __restrict__ topk_idx, const float* __restrict__ topk_val
   // entries under their local index, ascending; the rest follows (never gathered here)
   const int nv = hi - lo;
   for (int j = lane; j < K; j += 32) {
-    const int key = keys[j];
+    const int key = key_of(j);
     const bool local = j >= lo && j < hi;
     const int pos = local ? j - lo : (j < lo ? nv + j : j);
     out_idx[pos] = local ? key - v0 : key;
     out_p[pos] = merged_p(j);
-    out_perm[pos] = slot[j];
+    out_perm[pos] = (uint16_t)(ks[j] & 0xffffu);
   }
   if (lane == 0) { nvalid[t] = nv; Mout[t] = msum; Hent[t] = hsum; }
 }

@@ -387,7 +387,7 @@ static int launch_prep(const WsLayout& L, const kdkl_options& o, void* ws, const
   header_reset_kernel<<<1, 32, 0, st>>>(hdr);
   KDKL_LAUNCHED("header_reset_kernel");
   const int Kpad = next_pow2(K);
-  const size_t prep_smem = (size_t)PREP_WARPS * Kpad * (4 + 4 + 2);
+  const size_t prep_smem = (size_t)PREP_WARPS * Kpad * (8 + 4);   // (key, slot) words and probabilities
   prep_kernel<<<(unsigned)((T + PREP_WARPS - 1) / PREP_WARPS), PREP_WARPS * 32, prep_smem, st>>>(
       topk_idx, topk_val, teacher_lse, loss_mask, T, (int)V, (int)v0, (int)V_total, K, Kpad, inv_tau, o.teacher_mode,
       at<int>(ws, L.idx_sorted), at<float>(ws, L.p_sorted), at<uint16_t>(ws, L.perm), at<int>(ws, L.nvalid),
