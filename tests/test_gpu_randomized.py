@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 import torch
 
-from gradcheck import check_grad_matrix, check_support_rows, dense_dweight
+from gradcheck import check_grad_matrix, check_support_rows, dense_dweight, term_norms
 from oracle.kdkl_oracle import kdkl_oracle
 from paper_2608_03796_b200 import binding as B
 
@@ -125,10 +125,12 @@ def test_random_configuration_matches_oracle(seed, single_pass):
         # every row and every element (the single-pass step rounds its stored exponential as well: two roundings)
         nr = 2 if single_pass else 1
         b64 = base.double().numpy() if c["accumulate"] else 0.0
-        check_grad_matrix(dH, o["dH"], "dH", out_bf16=not c["dh32"], roundings=nr)
+        nH, nW = term_norms(o, c["h"].double().numpy(), c["W"].double().numpy(), idx, c["tau"])
+        check_grad_matrix(dH, o["dH"], "dH", out_bf16=not c["dh32"], roundings=nr, row_scale=nH)
         dense = dense_dweight(o, c["h"].double().numpy(), c["W"].double().numpy(), idx, c["tau"]) if single_pass else None
-        check_grad_matrix(dW - b64, o["dW"], "dW", roundings=nr, extra_tol=2.0 ** -22 * np.abs(b64), dense_mag=dense)
+        check_grad_matrix(dW - b64, o["dW"], "dW", roundings=nr, extra_tol=2.0 ** -22 * np.abs(b64), dense_mag=dense,
+                          row_scale=nW)
         check_support_rows(dW - b64, o["dW"], idx, list(np.flatnonzero(counted)[:3]), "dW", roundings=nr,
-                           dense_mag=dense)
+                           dense_mag=dense, row_scale=nW)
     else:
         assert not dH.any() and np.array_equal(dW, want_dW)

@@ -114,3 +114,54 @@ def test_cancelling_support_entry_of_a_one_token_batch():
     got[2] += 1.5 * 2.0 ** -8 * dense[2]
     with pytest.raises(AssertionError):
         check_grad_matrix(got, ref, "dW", roundings=2, dense_mag=dense)
+
+
+def test_term_norms_against_plain_loops():
+    from gradcheck import term_norms
+    from oracle.kdkl_oracle import kdkl_oracle
+    rng = np.random.default_rng(11)
+    T, H, V, K, tau = 5, 4, 9, 3, 0.8
+    h, W = rng.standard_normal((T, H)), rng.standard_normal((V, H))
+    idx = rng.integers(0, V, (T, K)); idx[1, 1] = idx[1, 0]; idx[2, 2] = -1
+    val = rng.standard_normal((T, K))
+    mask = np.array([1, 1, 1, 0, 1], np.uint8)
+    o = kdkl_oracle(h, W, idx, val, tau=tau, mask=mask, grad_loss=2.0)
+    nH, nW = term_norms(o, h, W, idx, tau)
+    # the dense dlogits through the oracle's own gradient: dH = G W with W = identity gives G
+    G = kdkl_oracle(np.concatenate([h, np.zeros((T, V))], 1)[:, :H], W, idx, val, tau=tau, mask=mask, grad_loss=2.0)
+    s = (h @ W.T) / tau
+    q = np.exp(s - s.max(1, keepdims=True)); q /= q.sum(1, keepdims=True)
+    want_H, want_W = np.zeros(T), np.zeros(V)
+    for t in range(T):
+        for v in range(V):
+            p_tv = sum(o["p_k"][t, k] for k in range(K) if idx[t, k] == v)
+            g_tv = o["g"][t] / tau * (o["M"][t] * q[t, v] - p_tv)
+            want_H[t] += g_tv ** 2 * (W[v] ** 2).sum()
+            want_W[v] += g_tv ** 2 * (h[t] ** 2).sum()
+    np.testing.assert_allclose(nH, np.sqrt(want_H), rtol=1e-12, atol=1e-18)
+    np.testing.assert_allclose(nW, np.sqrt(want_W), rtol=1e-12, atol=1e-18)
+    assert nH[3] == 0.0 and G["loss"] == o["loss"]
+
+
+def test_row_of_a_few_cancelling_terms_is_judged_against_its_terms():
+    """Three tokens with opposite signs dominate a dW row of a hidden size of 8: the row's norm is a third of the
+    root-sum-square of its terms. Every term rounded by half a bf16 step (the most one rounding can do) moves the
+    row by more than 1e-2 of its own norm, and by 2^-9 of its terms' norm."""
+    from gradcheck import check_grad_matrix
+    H = 8
+    hs = np.array([[1.0, -2.0, 0.5, 1.5, -1.0, 2.0, 0.25, -0.5],
+                   [1.1, -1.9, 0.4, 1.6, -0.9, 2.1, 0.30, -0.6],
+                   [0.9, -2.1, 0.6, 1.4, -1.1, 1.9, 0.20, -0.4]])
+    g = np.array([1.0, -1.5, 0.8])                        # dlogits of the three tokens at this vocabulary row
+    terms = g[:, None] * hs
+    ref = np.vstack([terms.sum(0), np.ones(H), np.ones(H)])
+    scale = np.array([np.sqrt((terms ** 2).sum()), 0.0, 0.0])
+    got = ref.copy()
+    got[0] = (terms * (1 + 2.0 ** -9 * np.array([[1.0], [-1.0], [1.0]]))).sum(0)
+    assert np.linalg.norm(got[0] - ref[0]) > 1e-2 * np.linalg.norm(ref[0])
+    with pytest.raises(AssertionError):
+        check_grad_matrix(got, ref, "dW")
+    check_grad_matrix(got, ref, "dW", row_scale=scale)
+    got[0] = (terms * (1 + 12 * 2.0 ** -9 * np.array([[1.0], [-1.0], [1.0]]))).sum(0)
+    with pytest.raises(AssertionError):
+        check_grad_matrix(got, ref, "dW", row_scale=scale)
