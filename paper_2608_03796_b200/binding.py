@@ -647,6 +647,7 @@ class TokenShardedFusedKL:
         kdkl_forward_backward(hidden, weight, topk_idx, topk_val, self.workspace, self.loss, self.dhidden,
                               self.dweight, teacher_lse=teacher_lse, loss_mask=loss_mask, chunk=self.chunk,
                               temperature=self.temperature, opt=self.opt, grad_loss=grad_loss)
+        self._launches[1], self._launches[2] = kdkl_last_launch_count(), 0
 
     def forward_backward(self, hidden, weight, topk_idx, topk_val, teacher_lse=None, loss_mask=None, grad_loss=1.0):
         self.count_tokens(loss_mask)
